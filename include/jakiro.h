@@ -1,0 +1,218 @@
+/*
+ * jakiro.h - C interface of the Jakiro draft-and-verify step for NVIDIA B200 (sm_100a).
+ *
+ * One speculative-decoding step of arXiv 2502.06282 has three phases (Sec. 2.1): draft,
+ * verify, refine.  This library provides the per-step kernels of each phase:
+ *
+ *   jk_draft_expand        one layer of the decoupled MoE draft head (Sec. 3.1.2, Eq. 2-5)
+ *   jk_tree_finalize       rerank the drafted candidates into the verification tree and
+ *                          build its attention mask (Sec. 3.1.2, Fig. 4)
+ *   jk_tree_verify_attn    tree-masked attention of one target layer (Sec. 2.1 step 2)
+ *   jk_accept_and_compact  acceptance walk, bonus token and KV-cache compaction
+ *                          (Sec. 2.1 steps 2-3)
+ *
+ * Conventions that hold for every call
+ *   - Returns 0 (JK_OK) or a negative jk_status.  Nothing throws or aborts.
+ *   - Pointers named "host" are host memory; every other pointer is DEVICE memory on the
+ *     current CUDA device, owned by the caller, 16-byte aligned.  The library allocates no
+ *     device memory: scratch space is the caller-provided workspace (jk_set_workspace).
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return without
+ *     synchronising.  Argument errors are reported by the return value before anything is
+ *     launched; data-dependent errors found on the device (an index out of range) are
+ *     recorded in a status word that jk_read_status returns.
+ *   - Tensors are dense, row-major, innermost index last.  "T" below is the context's
+ *     dtype (float or bfloat16).  B = batch, F = frontier nodes of this layer, H = hidden,
+ *     N = experts, K = active experts per node, I = expert inner size, V = vocabulary,
+ *     k_e = children per (node, expert), W = frontier width, M = tree nodes incl. root,
+ *     D = tree depth, Hq/Hkv/d = attention heads and head size, L = target layers.
+ *   - Same inputs give bitwise the same outputs (no floating-point atomics).
+ *   - Calls on one context must not overlap on the device: they share the workspace.
+ */
+#ifndef JAKIRO_H_
+#define JAKIRO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  JK_OK = 0,
+  JK_ERR_NULL = -1,       /* a required pointer is NULL                                  */
+  JK_ERR_SHAPE = -2,      /* a size is outside the supported range                       */
+  JK_ERR_ALIGN = -3,      /* a pointer or stride is not 16-byte aligned                  */
+  JK_ERR_DTYPE = -4,      /* unknown dtype                                               */
+  JK_ERR_CAPACITY = -5,   /* more rows than the context was created for                  */
+  JK_ERR_WORKSPACE = -6,  /* workspace missing or too small                              */
+  JK_ERR_CUDA = -7,       /* a CUDA runtime call failed (see jk_last_cuda_error)         */
+  JK_ERR_TIMEOUT = -8,    /* a bounded device-side wait ran out                          */
+  JK_ERR_BOUNDS = -9      /* device status: an input index was out of range              */
+} jk_status;
+
+typedef enum { JK_F32 = 0, JK_BF16 = 1 } jk_dtype;
+
+/* Limits: top_k <= n_experts <= 8, k_per_expert <= 16, max_tree <= 128,
+ * max_batch * max_frontier <= 128, head_dim 64 or 128, hidden/inter multiples of 8. */
+typedef struct {
+  int32_t hidden, n_experts, top_k, inter, vocab;
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  int32_t max_batch, max_tree, max_depth, max_frontier, k_per_expert;
+  int32_t dtype;            /* jk_dtype of weights, hidden states, Q and the KV cache    */
+  float rms_eps;            /* epsilon of the pre-MoE RMSNorm                            */
+  int32_t use_pre_norm;     /* 1: router and experts see RMSNorm(u) * norm_weight (the
+                               normalisation Sec. 3.1.2 leaves out of Eq. 1-5); 0: u     */
+  int32_t branch_residual;  /* 1: branch feature = g_r * Expert_r(x) + u; 0: g_r * Expert_r(x) */
+} jk_config;
+
+typedef struct jk_ctx jk_ctx;
+
+/* Host-only bookkeeping; no CUDA call is made.  *out is owned by the caller until jk_destroy. */
+int jk_create(jk_ctx** out, const jk_config* host_cfg);
+int jk_destroy(jk_ctx* ctx);
+/* Bytes of device scratch the context needs (a multiple of 256). */
+size_t jk_workspace_bytes(const jk_ctx* ctx);
+/* dev_ptr: device memory, 256-byte aligned, at least jk_workspace_bytes(ctx) bytes, owned by
+ * the caller and kept alive while the context is used.  Clears the device status word on
+ * `stream`. */
+int jk_set_workspace(jk_ctx* ctx, void* stream, void* dev_ptr, size_t bytes);
+const char* jk_strerror(int code);
+/* Text of the last CUDA runtime error seen by this context ("" if none). */
+const char* jk_last_cuda_error(const jk_ctx* ctx);
+/* Synchronises `stream`, copies the device status word to *host_status (0 or a jk_status)
+ * and clears it. */
+int jk_read_status(jk_ctx* ctx, void* stream, int32_t* host_status);
+/* Which kernels run the dense contractions: 0 = CUDA-core kernels, 1 = tensor-core
+ * (tcgen05) kernels where the dtype allows.  Default 1 for bf16, always 0 for f32. */
+int jk_set_tensor_path(jk_ctx* ctx, int32_t enable);
+
+/* Draft weights (Sec. 3.1.1-3.1.2): device pointers, read-only, output-major. */
+typedef struct {
+  const void* router;       /* T [N, H]     expert centroids e_j (Eq. 2)                 */
+  const void* w_gate;       /* T [N, I, H]  SiLU branch of Expert_j                      */
+  const void* w_up;         /* T [N, I, H]  linear branch of Expert_j                    */
+  const void* w_down;       /* T [N, H, I]  output projection of Expert_j                */
+  const void* lm_head;      /* T [V, H]     the target model's LM head (shared, Eq. 4)   */
+  const void* norm_weight;  /* T [H] or NULL (= ones)                                    */
+} jk_draft_weights;
+
+/* Candidate pool of one step: every child proposed by any jk_draft_expand call, in
+ * generation order (layer, frontier slot, branch, rank).  Arrays are [B, *] with
+ * `stride_b` elements between sequences; jk_draft_expand fills entries
+ * gidx_base .. gidx_base + F*K*k_e - 1 of each sequence. */
+typedef struct {
+  int32_t* tok;             /* token id                                                  */
+  float* score;             /* cumulative log-probability from the root                  */
+  int32_t* parent;          /* generation index of the parent, -1 = root                 */
+  int32_t* qslot;           /* row of the stored draft logits if the node was expanded, else -1 */
+  int32_t* branch;          /* 0 = left (larger router score), 1 = right, ...            */
+  int64_t stride_b;
+} jk_pool;
+
+/*
+ * One draft layer for F frontier nodes per sequence (Sec. 3.1.2).
+ *   x = RMSNorm(u) * norm_weight; s = softmax_N(x E^T) (Eq. 2); the K largest s keep their
+ *   value as gates, larger one first = left (Eq. 5); y_r = Expert_{j_r}(x);
+ *   f = sum_r g_r y_r + u (Eq. 3); branch feature b_r = g_r y_r (+ u);
+ *   logits_r = b_r W_head^T (Eq. 4); per branch the k_e largest logits (ties: lower id)
+ *   become children with score = parent_score + logit - logsumexp(logits_r); the W best
+ *   children of the layer (ties: lower index) form the next frontier.
+ * Inputs
+ *   u            T   [B, F, H]   hidden state of each frontier node after draft attention (Eq. 1)
+ *   parent_score f32 [B, F]      cumulative score of each frontier node (0 for the root)
+ *   parent_gidx  i32 [B, F]      generation index of each frontier node (-1 for the root)
+ *   gidx_base    generation index of this call's first child; slot_base: row index of this
+ *                call's first node among all expanded nodes of the step (root = 0)
+ * Outputs (any marked "opt" may be NULL)
+ *   out_probs    f32 [B, F, N]   router scores s (opt)
+ *   out_expert   i32 [B, F, K]   selected experts, left first
+ *   out_gate     f32 [B, F, K]
+ *   pool         children appended as described at jk_pool; qslot is set for the children
+ *                chosen as next frontier (slot_base + F + position), -1 for the others
+ *   out_lse      f32 [B, F, K]   logsumexp of each logits row (opt)
+ *   out_feat     T   [B, F, H]   combined feature f (Eq. 3)
+ *   out_logits   f32 [B, F, K, V] (opt; needed later for sampling acceptance)
+ *   next_frontier      i32 [B, W'] flat child index (f*K + r)*k_e + j of the chosen children,
+ *                      best first, W' = min(width, F*K*k_e) (opt, with the two arrays below);
+ *                      width = 0 skips the selection (last layer)
+ *   next_parent_score  f32 [B, W'] their scores
+ *   next_parent_gidx   i32 [B, W'] their generation indices
+ * Errors: NULL/ALIGN/SHAPE/CAPACITY (B > max_batch, F > max_frontier)/WORKSPACE/CUDA.
+ */
+int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* host_w,
+                    int32_t batch, int32_t n_frontier, int32_t width,
+                    const void* u, const float* parent_score, const int32_t* parent_gidx,
+                    int32_t gidx_base, int32_t slot_base,
+                    float* out_probs, int32_t* out_expert, float* out_gate,
+                    const jk_pool* host_pool, float* out_lse, void* out_feat, float* out_logits,
+                    int32_t* next_frontier, float* next_parent_score, int32_t* next_parent_gidx);
+
+/*
+ * Build the verification tree from the pool (Sec. 3.1.2; mask as in Fig. 4): node 0 is the
+ * root (root_tok[b]); nodes 1..M-1 are the M-1 best pool entries by (score descending,
+ * generation index ascending), listed in ascending generation index, so parent[i] < i.
+ *   pool_n <= 4096 entries per sequence; tree_size = M <= max_tree, pool_n >= M-1.
+ *   root_tok i32 [B]; outputs i32 [B, M]: tok, parent (-1 for the root), depth, branch, qslot
+ *   (root: 0); anc u64 [B, M, 2]: bit t of the 128-bit set is 1 iff t is the node itself or
+ *   one of its ancestors.
+ */
+int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const jk_pool* host_pool,
+                     int32_t pool_n, const int32_t* root_tok, int32_t tree_size,
+                     int32_t* tok, int32_t* parent, int32_t* depth, int32_t* branch,
+                     int32_t* qslot, uint64_t* anc);
+
+/*
+ * Tree-masked attention of one target layer over all M tree tokens (Sec. 2.1 step 2):
+ *   out[b,i,h] = sum_c softmax_c(softmax_scale * q[b,i,h] . K[b,h/G,c] + mask) V[b,h/G,c],
+ *   c < kv_len[b] + M, G = Hq/Hkv; column c is visible to node i iff c < kv_len[b] or
+ *   c - kv_len[b] is i or an ancestor of i.
+ *   q, out       T [B, M, Hq, d]
+ *   k_cache, v_cache  T [B, Hkv, cap, d] addressed with cache_stride_b / cache_stride_h
+ *                (elements); rows 0..kv_len[b]-1 hold the committed prefix, the caller has
+ *                written the tree tokens' K/V at rows kv_len[b] .. kv_len[b]+M-1
+ *   kv_len       i32 [B]; parent i32 [B, M] with parent[i] < i, -1 for the root
+ *   cache_rows   rows addressable in each cache (cap); kv_len[b] + M > cap sets JK_ERR_BOUNDS
+ */
+int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
+                        const void* q, const void* k_cache, const void* v_cache,
+                        int64_t cache_stride_b, int64_t cache_stride_h, int32_t cache_rows,
+                        const int32_t* kv_len, const int32_t* parent, float softmax_scale,
+                        void* out);
+
+/*
+ * Acceptance walk and KV compaction (Sec. 2.1 steps 2-3).
+ *   mode 0 (greedy): from the root, follow the first child whose token equals the target's
+ *     top-1 token (ties: lower id) at the current node; stop when none does; the bonus token
+ *     is the top-1 at the stop node.
+ *   mode 1 (sampling, temperature > 0): p = softmax(target/T) at the current node, q_r =
+ *     softmax(draft/T) of branch r; children in order: accept iff u_accept[c] <
+ *     min(1, p[x]/q_r[x]); on rejection p <- norm(max(0, p - q_r)), q_r[x] <- 0 and q_r is
+ *     renormalised; if no child is accepted the bonus token is the inverse-CDF draw from p with
+ *     u_bonus[depth].
+ *   Then, for every layer l < n_layers and both caches, row kv_len+acc_idx[j] moves to row
+ *   kv_len+1+j (j < n_acc) and kv_len[b] becomes kv_len[b] + 1 + n_acc[b].
+ *   target_logits  [B, M, V] of tl_dtype (f32 or bf16)
+ *   tok, parent, depth, branch, qslot   i32 [B, M] as written by jk_tree_finalize
+ *   draft_logits   f32 [B, S, K, V], S = n_slots (mode 1; NULL in mode 0)
+ *   u_accept       f32 [B, M], u_bonus f32 [B, max_depth+1], uniform in [0,1) (mode 1)
+ *   k_caches, v_caches   device arrays of n_layers device pointers (may be NULL if n_layers = 0)
+ *   outputs: n_acc i32 [B], acc_idx i32 [B, max_depth], acc_tok i32 [B, max_depth] (entries
+ *   past n_acc are -1), bonus_tok i32 [B]
+ */
+int jk_accept_and_compact(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
+                          int32_t mode, float temperature,
+                          const void* target_logits, int32_t tl_dtype,
+                          const int32_t* tok, const int32_t* parent, const int32_t* depth,
+                          const int32_t* branch, const int32_t* qslot,
+                          const float* draft_logits, int32_t n_slots,
+                          const float* u_accept, const float* u_bonus,
+                          int32_t n_layers, void* const* k_caches, void* const* v_caches,
+                          int64_t cache_stride_b, int64_t cache_stride_h, int32_t cache_rows,
+                          int32_t* kv_len, int32_t* n_acc, int32_t* acc_idx, int32_t* acc_tok,
+                          int32_t* bonus_tok);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JAKIRO_H_ */
