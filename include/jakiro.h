@@ -132,7 +132,9 @@ typedef struct {
  *                chosen as next frontier (slot_base + F + position), -1 for the others
  *   out_lse      f32 [B, F, K]   logsumexp of each logits row (opt)
  *   out_feat     T   [B, F, H]   combined feature f (Eq. 3)
- *   out_logits   f32 [B, F, K, V] (opt; needed later for sampling acceptance)
+ *   out_logits   f32 [B, F, K, V] (opt; needed later for sampling acceptance), with
+ *                logits_stride_b elements between sequences (0 = dense, F*K*V), so that a call
+ *                can write rows slot_base..slot_base+F-1 of a [B, S, K, V] buffer directly
  *   next_frontier      i32 [B, W'] flat child index (f*K + r)*k_e + j of the chosen children,
  *                      best first, W' = min(width, F*K*k_e) (opt, with the two arrays below);
  *                      width = 0 skips the selection (last layer)
@@ -146,7 +148,7 @@ int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* host_w,
                     int32_t gidx_base, int32_t slot_base,
                     float* out_probs, int32_t* out_expert, float* out_gate,
                     const jk_pool* host_pool, float* out_lse, void* out_feat, float* out_logits,
-                    int32_t* next_frontier, float* next_parent_score, int32_t* next_parent_gidx);
+                    int64_t logits_stride_b, int32_t* next_frontier, float* next_parent_score, int32_t* next_parent_gidx);
 
 /*
  * Build the verification tree from the pool (Sec. 3.1.2; mask as in Fig. 4): node 0 is the

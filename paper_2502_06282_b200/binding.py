@@ -1,0 +1,288 @@
+"""ctypes binding of libjakiro.so: same entry points as include/jakiro.h.
+
+Argument marshalling only.  Every arithmetic step runs in the CUDA kernels of
+the library; torch is used for device memory and for the current stream.  If
+the shared library has not been built the import of the library raises; there
+is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libjakiro.so")
+
+JK_F32, JK_BF16 = 0, 1
+JK_OK = 0
+ERR = {"NULL": -1, "SHAPE": -2, "ALIGN": -3, "DTYPE": -4, "CAPACITY": -5, "WORKSPACE": -6,
+       "CUDA": -7, "TIMEOUT": -8, "BOUNDS": -9}
+
+EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", "jk_strerror",
+           "jk_last_cuda_error", "jk_read_status", "jk_set_tensor_path", "jk_draft_expand",
+           "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact"]
+
+
+class JkConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "hidden", "n_experts", "top_k", "inter", "vocab", "n_q_heads", "n_kv_heads", "head_dim",
+        "max_batch", "max_tree", "max_depth", "max_frontier", "k_per_expert", "dtype")] + [
+        ("rms_eps", C.c_float), ("use_pre_norm", C.c_int32), ("branch_residual", C.c_int32)]
+
+
+class JkDraftWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("router", "w_gate", "w_up", "w_down", "lm_head",
+                                          "norm_weight")]
+
+
+class JkPool(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("tok", "score", "parent", "qslot", "branch")] + [
+        ("stride_b", C.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2502_06282_b200.build` "
+                "(needs nvcc); there is no fallback implementation")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+        L.jk_create.argtypes = [C.POINTER(vp), C.POINTER(JkConfig)]
+        L.jk_destroy.argtypes = [vp]
+        L.jk_workspace_bytes.argtypes = [vp]
+        L.jk_workspace_bytes.restype = C.c_size_t
+        L.jk_set_workspace.argtypes = [vp, vp, vp, C.c_size_t]
+        L.jk_strerror.argtypes = [C.c_int]
+        L.jk_strerror.restype = C.c_char_p
+        L.jk_last_cuda_error.argtypes = [vp]
+        L.jk_last_cuda_error.restype = C.c_char_p
+        L.jk_read_status.argtypes = [vp, vp, C.POINTER(i32)]
+        L.jk_set_tensor_path.argtypes = [vp, i32]
+        L.jk_draft_expand.argtypes = [vp, vp, C.POINTER(JkDraftWeights), i32, i32, i32, vp, vp,
+                                      vp, i32, i32, vp, vp, vp, C.POINTER(JkPool), vp, vp, vp,
+                                      i64, vp, vp, vp]
+        L.jk_tree_finalize.argtypes = [vp, vp, i32, C.POINTER(JkPool), i32, vp, i32, vp, vp, vp,
+                                       vp, vp, vp]
+        L.jk_tree_verify_attn.argtypes = [vp, vp, i32, i32, vp, vp, vp, i64, i64, i32, vp, vp,
+                                          f32, vp]
+        L.jk_accept_and_compact.argtypes = [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, vp, vp,
+                                            vp, vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp,
+                                            vp, vp, vp, vp]
+        for name in EXPORTS:
+            if name not in ("jk_workspace_bytes", "jk_strerror", "jk_last_cuda_error"):
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+class JakiroError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        msg = lib().jk_strerror(code).decode()
+        super().__init__(f"{where}: {msg} ({code}) {detail}".strip())
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def torch_dtype(dtype: str) -> torch.dtype:
+    return torch.bfloat16 if dtype == "bf16" else torch.float32
+
+
+class Context:
+    """Owns a jk_ctx and its device workspace (a torch allocation)."""
+
+    def __init__(self, *, hidden, n_experts, top_k, inter, vocab, n_q_heads, n_kv_heads,
+                 head_dim, max_batch, max_tree, max_depth, max_frontier, k_per_expert, dtype,
+                 rms_eps=1e-5, use_pre_norm=True, branch_residual=True, device="cuda",
+                 allocate=True):
+        self.cfg = JkConfig(hidden, n_experts, top_k, inter, vocab, n_q_heads, n_kv_heads,
+                            head_dim, max_batch, max_tree, max_depth, max_frontier,
+                            k_per_expert, JK_BF16 if dtype == "bf16" else JK_F32, rms_eps,
+                            int(use_pre_norm), int(branch_residual))
+        self.dtype = dtype
+        self.tdtype = torch_dtype(dtype)
+        self._h = C.c_void_p()
+        rc = lib().jk_create(C.byref(self._h), C.byref(self.cfg))
+        if rc != JK_OK:
+            self._h = C.c_void_p()
+            raise JakiroError(rc, "jk_create")
+        self.workspace = None
+        self.device = device
+        if allocate:
+            n = lib().jk_workspace_bytes(self._h)
+            self.workspace = torch.empty(n + 256, dtype=torch.uint8, device=device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            self._check(lib().jk_set_workspace(self._h, _stream(), base, n), "jk_set_workspace")
+
+    @classmethod
+    def for_workload(cls, w, **kw) -> "Context":
+        return cls(hidden=w.hidden, n_experts=w.n_experts, top_k=w.top_k, inter=w.inter,
+                   vocab=w.vocab, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                   head_dim=w.head_dim, max_batch=w.batch, max_tree=w.tree_size,
+                   max_depth=w.depth, max_frontier=max(w.frontier_sizes),
+                   k_per_expert=w.k_per_expert, dtype=w.dtype, **kw)
+
+    def _check(self, rc: int, where: str):
+        if rc != JK_OK:
+            detail = lib().jk_last_cuda_error(self._h).decode() if rc == ERR["CUDA"] else ""
+            raise JakiroError(rc, where, detail)
+
+    @property
+    def workspace_bytes(self) -> int:
+        return lib().jk_workspace_bytes(self._h)
+
+    def close(self):
+        if self._h:
+            lib().jk_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_tensor_path(self, enable: bool):
+        self._check(lib().jk_set_tensor_path(self._h, int(enable)), "jk_set_tensor_path")
+
+    def read_status(self) -> int:
+        out = C.c_int32(0)
+        self._check(lib().jk_read_status(self._h, _stream(), C.byref(out)), "jk_read_status")
+        return out.value
+
+    # ------------------------------------------------------------------ calls
+    @staticmethod
+    def weights_struct(w: Dict[str, torch.Tensor]) -> JkDraftWeights:
+        return JkDraftWeights(_ptr(w["router"]), _ptr(w["w_gate"]), _ptr(w["w_up"]),
+                              _ptr(w["w_down"]), _ptr(w["lm_head"]), _ptr(w.get("norm_weight")))
+
+    @staticmethod
+    def pool_struct(pool: Dict[str, torch.Tensor]) -> JkPool:
+        return JkPool(_ptr(pool["tok"]), _ptr(pool["score"]), _ptr(pool["parent"]),
+                      _ptr(pool["qslot"]), _ptr(pool["branch"]), pool["tok"].stride(0))
+
+    def draft_expand(self, weights, batch, n_frontier, width, u, parent_score, parent_gidx,
+                     gidx_base, slot_base, out_probs, out_expert, out_gate, pool, out_lse,
+                     out_feat, out_logits, next_frontier, next_parent_score, next_parent_gidx):
+        ws = weights if isinstance(weights, JkDraftWeights) else self.weights_struct(weights)
+        ps = pool if isinstance(pool, JkPool) else self.pool_struct(pool)
+        rc = lib().jk_draft_expand(
+            self._h, _stream(), C.byref(ws), batch, n_frontier, width, _ptr(u),
+            _ptr(parent_score), _ptr(parent_gidx), gidx_base, slot_base, _ptr(out_probs),
+            _ptr(out_expert), _ptr(out_gate), C.byref(ps), _ptr(out_lse), _ptr(out_feat),
+            _ptr(out_logits), 0 if out_logits is None else out_logits.stride(0),
+            _ptr(next_frontier), _ptr(next_parent_score),
+            _ptr(next_parent_gidx))
+        self._check(rc, "jk_draft_expand")
+
+    def tree_finalize(self, batch, pool, pool_n, root_tok, tree_size, tok, parent, depth, branch,
+                      qslot, anc):
+        ps = pool if isinstance(pool, JkPool) else self.pool_struct(pool)
+        rc = lib().jk_tree_finalize(self._h, _stream(), batch, C.byref(ps), pool_n,
+                                    _ptr(root_tok), tree_size, _ptr(tok), _ptr(parent),
+                                    _ptr(depth), _ptr(branch), _ptr(qslot), _ptr(anc))
+        self._check(rc, "jk_tree_finalize")
+
+    def tree_verify_attn(self, batch, tree_size, q, k_cache, v_cache, kv_len, parent, scale, out,
+                         cache_rows=None):
+        rows = k_cache.shape[2] if cache_rows is None else cache_rows
+        rc = lib().jk_tree_verify_attn(self._h, _stream(), batch, tree_size, _ptr(q),
+                                       _ptr(k_cache), _ptr(v_cache), k_cache.stride(0),
+                                       k_cache.stride(1), rows, _ptr(kv_len), _ptr(parent),
+                                       float(scale), _ptr(out))
+        self._check(rc, "jk_tree_verify_attn")
+
+    def accept_and_compact(self, batch, tree_size, mode, temperature, target_logits, tree,
+                           draft_logits, n_slots, u_accept, u_bonus, n_layers, k_ptrs, v_ptrs,
+                           cache_stride_b, cache_stride_h, cache_rows, kv_len, n_acc, acc_idx,
+                           acc_tok, bonus_tok):
+        tl_dtype = JK_BF16 if target_logits.dtype == torch.bfloat16 else JK_F32
+        rc = lib().jk_accept_and_compact(
+            self._h, _stream(), batch, tree_size, mode, float(temperature), _ptr(target_logits),
+            tl_dtype, _ptr(tree["tok"]), _ptr(tree["parent"]), _ptr(tree["depth"]),
+            _ptr(tree["branch"]), _ptr(tree["qslot"]), _ptr(draft_logits), n_slots,
+            _ptr(u_accept), _ptr(u_bonus), n_layers, _ptr(k_ptrs), _ptr(v_ptrs), cache_stride_b,
+            cache_stride_h, cache_rows, _ptr(kv_len), _ptr(n_acc), _ptr(acc_idx), _ptr(acc_tok),
+            _ptr(bonus_tok))
+        self._check(rc, "jk_accept_and_compact")
+
+
+class StepBuffers:
+    """Device buffers of one draft-and-verify step for a workload, allocated once."""
+
+    def __init__(self, ctx: Context, w, keep_logits: bool = True, device="cuda"):
+        B, K, ke, V, H = w.batch, w.top_k, w.k_per_expert, w.vocab, w.hidden
+        fs = w.frontier_sizes
+        Fm = max(fs)
+        i32 = dict(dtype=torch.int32, device=device)
+        f32 = dict(dtype=torch.float32, device=device)
+        self.w = w
+        self.pool = {"tok": torch.empty(B, w.pool_size, **i32),
+                     "score": torch.empty(B, w.pool_size, **f32),
+                     "parent": torch.empty(B, w.pool_size, **i32),
+                     "qslot": torch.empty(B, w.pool_size, **i32),
+                     "branch": torch.empty(B, w.pool_size, **i32)}
+        self.pool_struct = ctx.pool_struct(self.pool)
+        self.probs = [torch.empty(B, F, w.n_experts, **f32) for F in fs]
+        self.expert = [torch.empty(B, F, K, **i32) for F in fs]
+        self.gate = [torch.empty(B, F, K, **f32) for F in fs]
+        self.lse = [torch.empty(B, F, K, **f32) for F in fs]
+        self.feat = [torch.empty(B, F, H, dtype=ctx.tdtype, device=device) for F in fs]
+        self.logits = torch.empty(B, w.n_slots, K, V, **f32) if keep_logits else None
+        self.frontier = [torch.empty(B, min(w.width, F * K * ke), **i32) for F in fs]
+        self.parent_score = [torch.zeros(B, 1, **f32)] + [
+            torch.empty(B, min(w.width, F * K * ke), **f32) for F in fs]
+        self.parent_gidx = [torch.full((B, 1), -1, **i32)] + [
+            torch.empty(B, min(w.width, F * K * ke), **i32) for F in fs]
+        M = w.tree_size
+        self.tree = {k: torch.empty(B, M, **i32) for k in ("tok", "parent", "depth", "branch",
+                                                           "qslot")}
+        self.anc = torch.empty(B, M, 2, dtype=torch.int64, device=device)
+        self.n_acc = torch.empty(B, **i32)
+        self.acc_idx = torch.empty(B, w.depth, **i32)
+        self.acc_tok = torch.empty(B, w.depth, **i32)
+        self.bonus = torch.empty(B, **i32)
+
+
+def run_draft(ctx: Context, bufs: StepBuffers, weights, u_layers: Sequence[torch.Tensor],
+              root_tok: torch.Tensor, finalize: bool = True):
+    """D calls of jk_draft_expand, one per tree layer, then jk_tree_finalize.  The expanded
+    nodes' logits are kept in bufs.logits at slot order when that buffer exists."""
+    w = bufs.w
+    fs = w.frontier_sizes
+    B, K, ke = w.batch, w.top_k, w.k_per_expert
+    gidx_base = 0
+    slot_base = 0
+    for l, F in enumerate(fs):
+        last = l == len(fs) - 1
+        out_logits = None
+        if bufs.logits is not None:      # rows slot_base..slot_base+F-1 of every sequence
+            out_logits = bufs.logits[:, slot_base:slot_base + F]
+        ctx.draft_expand(weights, B, F, 0 if last else w.width, u_layers[l],
+                         bufs.parent_score[l], bufs.parent_gidx[l], gidx_base, slot_base,
+                         bufs.probs[l], bufs.expert[l], bufs.gate[l], bufs.pool_struct,
+                         bufs.lse[l], bufs.feat[l], out_logits,
+                         None if last else bufs.frontier[l],
+                         None if last else bufs.parent_score[l + 1],
+                         None if last else bufs.parent_gidx[l + 1])
+        gidx_base += F * K * ke
+        slot_base += F
+    if finalize:
+        ctx.tree_finalize(B, bufs.pool_struct, w.pool_size, root_tok, w.tree_size,
+                          bufs.tree["tok"], bufs.tree["parent"], bufs.tree["depth"],
+                          bufs.tree["branch"], bufs.tree["qslot"], bufs.anc)

@@ -1,0 +1,371 @@
+// jk_accept_and_compact: per-node statistics of the target logits, the acceptance walk (greedy
+// path match or speculative sampling, arXiv 2502.06282 Sec. 2.1 steps 2-3) and the compaction of
+// the accepted nodes' KV rows.
+#include <limits.h>
+#include <math.h>
+
+#include "jk_common.cuh"
+
+// ------------------------------------------------------------------------------------------
+// Row statistics: top-1 token (ties: lower id), max and sum exp((x - max)/T).  One block per
+// tree node.
+// ------------------------------------------------------------------------------------------
+template <typename TL>
+__global__ void __launch_bounds__(512) k_row_stats(const TL* __restrict__ tl, int V, float inv_t,
+                                                   int32_t* __restrict__ rs_arg,
+                                                   float* __restrict__ rs_max,
+                                                   float* __restrict__ rs_sum) {
+  constexpr int VN = jk_vec<TL>::N;
+  __shared__ float red[33];
+  __shared__ float wv[16];
+  __shared__ int wi[16];
+  const size_t row = blockIdx.x;
+  const TL* r = tl + row * V;
+  float bv = -INFINITY;
+  int bi = INT_MAX;
+  const int vmain = V / VN * VN;
+  for (int k = threadIdx.x * VN; k < vmain; k += blockDim.x * VN) {
+    float v[VN];
+    jk_vec<TL>::load(r + k, v);
+#pragma unroll
+    for (int i = 0; i < VN; ++i)
+      if (jk_better(v[i], k + i, bv, bi)) { bv = v[i]; bi = k + i; }
+  }
+  for (int k = vmain + threadIdx.x; k < V; k += blockDim.x) {
+    const float v = jk_to_float(r[k]);
+    if (jk_better(v, k, bv, bi)) { bv = v; bi = k; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (jk_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
+  __syncthreads();
+  float mx = wv[0];
+  int am = wi[0];
+  for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+    if (jk_better(wv[w], wi[w], mx, am)) { mx = wv[w]; am = wi[w]; }
+  float s = 0.f;
+  for (int k = threadIdx.x * VN; k < vmain; k += blockDim.x * VN) {
+    float v[VN];
+    jk_vec<TL>::load(r + k, v);
+#pragma unroll
+    for (int i = 0; i < VN; ++i) s += expf((v[i] - mx) * inv_t);
+  }
+  for (int k = vmain + threadIdx.x; k < V; k += blockDim.x)
+    s += expf((jk_to_float(r[k]) - mx) * inv_t);
+  s = jk_block_sum(s, red);
+  if (threadIdx.x == 0) { rs_arg[row] = am; rs_max[row] = mx; rs_sum[row] = s; }
+}
+
+// ------------------------------------------------------------------------------------------
+// The walk.  One block per sequence.
+// ------------------------------------------------------------------------------------------
+struct walk_out {
+  int32_t* kv_len;
+  int32_t* p_old;
+  int32_t* n_acc;
+  int32_t* acc_idx;
+  int32_t* acc_tok;
+  int32_t* bonus_tok;
+};
+
+__device__ __forceinline__ void walk_finish(const walk_out& o, int b, int max_depth, int n,
+                                            const int* path, const int* path_tok, int bonus,
+                                            int cache_rows, int M, int32_t* status) {
+  // thread 0 only
+  const int P = o.kv_len[b];
+  o.p_old[b] = P;
+  o.n_acc[b] = n;
+  for (int j = 0; j < max_depth; ++j) {
+    o.acc_idx[(size_t)b * max_depth + j] = j < n ? path[j] : -1;
+    o.acc_tok[(size_t)b * max_depth + j] = j < n ? path_tok[j] : -1;
+  }
+  o.bonus_tok[b] = bonus;
+  if (P < 0 || P + M > cache_rows) jk_set_status(status, JK_ERR_BOUNDS);
+  o.kv_len[b] = P + 1 + n;
+}
+
+__global__ void __launch_bounds__(128) k_walk_greedy(
+    int M, int max_depth, int V, const int32_t* __restrict__ tok,
+    const int32_t* __restrict__ parent, const int32_t* __restrict__ rs_arg, walk_out o,
+    int cache_rows, int32_t* status) {
+  __shared__ int s_next;
+  __shared__ int path[16], path_tok[16];
+  const int b = blockIdx.x;
+  const int t = threadIdx.x;                         // one thread per tree node
+  int cur = 0, n = 0;
+  for (int level = 0; level < max_depth; ++level) {
+    const int want = rs_arg[(size_t)b * M + cur];
+    if (t == 0) s_next = INT_MAX;
+    __syncthreads();
+    if (t < M && t > 0 && parent[(size_t)b * M + t] == cur && tok[(size_t)b * M + t] == want)
+      atomicMin(&s_next, t);                         // first matching child in child order
+    __syncthreads();
+    const int nxt = s_next;
+    __syncthreads();
+    if (nxt == INT_MAX) break;
+    if (t == 0) { path[n] = nxt; path_tok[n] = want; }
+    ++n;
+    cur = nxt;
+  }
+  __syncthreads();
+  if (t == 0)
+    walk_finish(o, b, max_depth, n, path, path_tok, rs_arg[(size_t)b * M + cur], cache_rows, M,
+                status);
+}
+
+// Sampling walk.  p and the q_r start "lazy" (read from the logits with the row's max and sum)
+// and are written out to pbuf/qbuf the first time a rejection changes them.
+__global__ void __launch_bounds__(1024) k_walk_sample(
+    int M, int max_depth, int V, int K, int n_slots, float inv_t,
+    const void* __restrict__ tl_raw, int tl_bf16, const int32_t* __restrict__ tok,
+    const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
+    const int32_t* __restrict__ branch, const int32_t* __restrict__ qslot,
+    const float* __restrict__ draft_logits, const float* __restrict__ u_accept,
+    const float* __restrict__ u_bonus, const float* __restrict__ rs_max,
+    const float* __restrict__ rs_sum, float* __restrict__ pbuf_all, float* __restrict__ qbuf_all,
+    walk_out o, int cache_rows, int32_t* status) {
+  __shared__ float red[33];
+  __shared__ int kids[JK_MAX_TREE];
+  __shared__ int n_kids;
+  __shared__ int path[16], path_tok[16];
+  __shared__ int s_decision;
+  __shared__ float scan_s[1024];
+  __shared__ int s_found;
+  const int b = blockIdx.x, t = threadIdx.x, nt = blockDim.x;
+  float* pbuf = pbuf_all + (size_t)b * V;
+  const float* tlf = (const float*)tl_raw;
+  const __nv_bfloat16* tlh = (const __nv_bfloat16*)tl_raw;
+  int cur = 0, n = 0;
+  bool p_mat = false;                 // p lives in pbuf (scaled by p_scale) instead of the logits
+  float p_scale = 1.f, p_max = 0.f, p_isum = 1.f;
+  size_t tl_row = 0;
+  auto tl_at = [&](size_t row, int v) -> float {
+    return tl_bf16 ? __bfloat162float(tlh[row * V + v]) : tlf[row * V + v];
+  };
+  auto p_at = [&](int v) -> float {
+    return p_mat ? pbuf[v] * p_scale : expf((tl_at(tl_row, v) - p_max) * inv_t) * p_isum;
+  };
+  while (true) {
+    tl_row = (size_t)b * M + cur;
+    p_mat = false;
+    p_max = rs_max[tl_row];
+    p_isum = 1.f / rs_sum[tl_row];
+    // children of cur in child order (= ascending node index)
+    if (t == 0) {
+      int c = 0;
+      for (int i = 1; i < M; ++i)
+        if (parent[(size_t)b * M + i] == cur) kids[c++] = i;
+      n_kids = c;
+    }
+    __syncthreads();
+    const int nk = n_kids;
+    const int slot = qslot[(size_t)b * M + cur];
+    int accepted = -1;
+    if (nk > 0 && n < max_depth && slot >= 0 && slot < n_slots) {
+      // per-branch draft distributions: lazy (max, 1/sum) until a rejection touches them
+      float q_max[JK_MAX_EXPERTS], q_isum[JK_MAX_EXPERTS], q_scale[JK_MAX_EXPERTS];
+      bool q_mat[JK_MAX_EXPERTS];
+      for (int r = 0; r < K; ++r) {
+        const float* dl = draft_logits + (((size_t)b * n_slots + slot) * K + r) * V;
+        float mx = -INFINITY;
+        for (int v = t; v < V; v += nt) mx = fmaxf(mx, dl[v]);
+        mx = jk_block_max(mx, red);
+        float s = 0.f;
+        for (int v = t; v < V; v += nt) s += expf((dl[v] - mx) * inv_t);
+        s = jk_block_sum(s, red);
+        q_max[r] = mx; q_isum[r] = 1.f / s; q_scale[r] = 1.f; q_mat[r] = false;
+      }
+      for (int ci = 0; ci < nk; ++ci) {
+        const int c = kids[ci];
+        const int x = tok[(size_t)b * M + c];
+        int r = branch[(size_t)b * M + c];
+        if (x < 0 || x >= V || r < 0 || r >= K) {
+          if (t == 0) jk_set_status(status, JK_ERR_BOUNDS);
+          break;
+        }
+        const float* dl = draft_logits + (((size_t)b * n_slots + slot) * K + r) * V;
+        float* qbuf = qbuf_all + ((size_t)b * K + r) * V;
+        if (t == 0) {
+          const float px = p_at(x);
+          const float qx = q_mat[r] ? qbuf[x] * q_scale[r]
+                                    : expf((dl[x] - q_max[r]) * inv_t) * q_isum[r];
+          bool acc;
+          if (qx > 0.f) acc = u_accept[(size_t)b * M + c] < fminf(1.f, px / qx);
+          else acc = px > 0.f;
+          s_decision = acc ? 1 : 0;
+        }
+        __syncthreads();
+        const int dec = s_decision;
+        __syncthreads();
+        if (dec) { accepted = c; break; }
+        // rejection: p <- max(0, p - q_r) (normalised through p_scale); q_r[x] <- 0, renormalised
+        float sp = 0.f, sq = 0.f;
+        for (int v = t; v < V; v += nt) {
+          const float pv = p_at(v);
+          const float qv = q_mat[r] ? qbuf[v] * q_scale[r]
+                                    : expf((dl[v] - q_max[r]) * inv_t) * q_isum[r];
+          const float res = fmaxf(0.f, pv - qv);
+          const float qn = (v == x) ? 0.f : qv;
+          pbuf[v] = res;
+          qbuf[v] = qn;
+          sp += res;
+          sq += qn;
+        }
+        sp = jk_block_sum(sp, red);
+        sq = jk_block_sum(sq, red);
+        q_mat[r] = true;
+        q_scale[r] = sq > 0.f ? 1.f / sq : 1.f;
+        if (!(sp > 0.f)) {            // residual vanished: keep the node's own p for the bonus
+          p_mat = false;
+          break;
+        }
+        p_mat = true;
+        p_scale = 1.f / sp;
+      }
+    }
+    if (accepted >= 0) {
+      if (t == 0) { path[n] = accepted; path_tok[n] = tok[(size_t)b * M + accepted]; }
+      ++n;
+      cur = accepted;
+      __syncthreads();
+      continue;
+    }
+    // bonus token: inverse CDF of the current p at u_bonus[depth]
+    const int dcur = depth[(size_t)b * M + cur];
+    const float ub = u_bonus[(size_t)b * (max_depth + 1) + min(max(dcur, 0), max_depth)];
+    const int per = (V + nt - 1) / nt;
+    const int v0 = t * per, v1 = min(V, v0 + per);
+    float loc = 0.f;
+    for (int v = v0; v < v1; ++v) loc += p_at(v);
+    scan_s[t] = loc;
+    if (t == 0) s_found = INT_MAX;
+    __syncthreads();
+    for (int off = 1; off < nt; off <<= 1) {
+      const float add = t >= off ? scan_s[t - off] : 0.f;
+      __syncthreads();
+      scan_s[t] += add;
+      __syncthreads();
+    }
+    const float total = scan_s[nt - 1];
+    const float thr = ub * total;
+    float run = scan_s[t] - loc;
+    for (int v = v0; v < v1; ++v) {
+      run += p_at(v);
+      if (run > thr) { atomicMin(&s_found, v); break; }
+    }
+    __syncthreads();
+    if (s_found == INT_MAX) {            // rounding left no bin: last token with p > 0
+      __syncthreads();
+      if (t == 0) s_found = -1;
+      __syncthreads();
+      for (int v = v1 - 1; v >= v0; --v)
+        if (p_at(v) > 0.f) { atomicMax(&s_found, v); break; }
+      __syncthreads();
+    }
+    if (t == 0)
+      walk_finish(o, b, max_depth, n, path, path_tok, max(s_found, 0), cache_rows, M, status);
+    return;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// KV compaction: row P + acc_idx[j] -> row P + 1 + j.  One block per (cache, sequence, kv head);
+// all source rows are loaded before any row is stored (a destination can be a later source).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_compact(
+    void* const* __restrict__ k_caches, void* const* __restrict__ v_caches, int n_layers,
+    long long stride_b, long long stride_h, int row_bytes, int cache_rows, int max_depth, int M,
+    const int32_t* __restrict__ p_old, const int32_t* __restrict__ n_acc,
+    const int32_t* __restrict__ acc_idx, int elem_size) {
+  const int which = blockIdx.z;                  // layer*2 + (0 = K, 1 = V)
+  const int b = blockIdx.y, kvh = blockIdx.x;
+  const int n = n_acc[b];
+  const int P = p_old[b];
+  if (n <= 0 || P < 0 || P + M > cache_rows) return;
+  char* base = (char*)((which & 1) ? v_caches[which >> 1] : k_caches[which >> 1]) +
+               ((size_t)b * stride_b + (size_t)kvh * stride_h) * elem_size;
+  const int chunks = row_bytes / 16;
+  const int total = n * chunks;
+  uint4 held[2];                                 // up to 2 chunks per thread (16 rows * 32 chunks)
+  int cnt = 0;
+  for (int idx = threadIdx.x; idx < total && cnt < 2; idx += blockDim.x, ++cnt) {
+    const int j = idx / chunks, c = idx % chunks;
+    const int a = acc_idx[(size_t)b * max_depth + j];
+    held[cnt] = *reinterpret_cast<const uint4*>(base + (size_t)(P + a) * row_bytes + c * 16);
+  }
+  __syncthreads();
+  cnt = 0;
+  for (int idx = threadIdx.x; idx < total && cnt < 2; idx += blockDim.x, ++cnt) {
+    const int j = idx / chunks, c = idx % chunks;
+    *reinterpret_cast<uint4*>(base + (size_t)(P + 1 + j) * row_bytes + c * 16) = held[cnt];
+  }
+}
+
+extern "C" int jk_accept_and_compact(
+    jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size, int32_t mode, float temperature,
+    const void* target_logits, int32_t tl_dtype, const int32_t* tok, const int32_t* parent,
+    const int32_t* depth, const int32_t* branch, const int32_t* qslot, const float* draft_logits,
+    int32_t n_slots, const float* u_accept, const float* u_bonus, int32_t n_layers,
+    void* const* k_caches, void* const* v_caches, int64_t cache_stride_b, int64_t cache_stride_h,
+    int32_t cache_rows, int32_t* kv_len, int32_t* n_acc, int32_t* acc_idx, int32_t* acc_tok,
+    int32_t* bonus_tok) {
+  if (!ctx || !target_logits || !tok || !parent || !depth || !branch || !qslot || !kv_len ||
+      !n_acc || !acc_idx || !acc_tok || !bonus_tok)
+    return JK_ERR_NULL;
+  if (mode != 0 && mode != 1) return JK_ERR_SHAPE;
+  if (mode == 1 && (!draft_logits || !u_accept || !u_bonus)) return JK_ERR_NULL;
+  if (mode == 1 && (!(temperature > 0.f) || n_slots < 1)) return JK_ERR_SHAPE;
+  if (n_layers < 0 || (n_layers > 0 && (!k_caches || !v_caches))) return JK_ERR_NULL;
+  if (tl_dtype != JK_F32 && tl_dtype != JK_BF16) return JK_ERR_DTYPE;
+  const jk_config& c = ctx->cfg;
+  if (batch < 1 || tree_size < 1 || cache_rows < tree_size) return JK_ERR_SHAPE;
+  if (batch > c.max_batch || tree_size > c.max_tree) return JK_ERR_CAPACITY;
+  if (!jk_aligned16(target_logits) || (draft_logits && !jk_aligned16(draft_logits)))
+    return JK_ERR_ALIGN;
+  const int es = jk_elem_size(c.dtype);
+  const int row_bytes = c.head_dim * es;
+  if (n_layers > 0 && ((cache_stride_b * es) % 16 || (cache_stride_h * es) % 16))
+    return JK_ERR_ALIGN;
+  // the vectorised row scan needs 16-byte aligned rows
+  if (((size_t)c.vocab * jk_elem_size(tl_dtype)) % 16) return JK_ERR_ALIGN;
+  if (!ctx->ws) return JK_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const jk_ws_layout& L = ctx->lay;
+  char* ws = ctx->ws;
+  int32_t* rs_arg = (int32_t*)(ws + L.rs_arg);
+  float* rs_max = (float*)(ws + L.rs_max);
+  float* rs_sum = (float*)(ws + L.rs_sum);
+  int32_t* status = (int32_t*)(ws + L.status);
+  const float inv_t = mode == 1 ? 1.f / temperature : 1.f;
+  const int rows = batch * tree_size;
+  if (tl_dtype == JK_BF16)
+    k_row_stats<__nv_bfloat16><<<rows, 512, 0, st>>>((const __nv_bfloat16*)target_logits, c.vocab,
+                                                     inv_t, rs_arg, rs_max, rs_sum);
+  else
+    k_row_stats<float><<<rows, 512, 0, st>>>((const float*)target_logits, c.vocab, inv_t, rs_arg,
+                                             rs_max, rs_sum);
+  JK_LAUNCH_CHECK(ctx);
+  walk_out o{kv_len, (int32_t*)(ws + L.p_old), n_acc, acc_idx, acc_tok, bonus_tok};
+  if (mode == 0) {
+    k_walk_greedy<<<batch, 128, 0, st>>>(tree_size, c.max_depth, c.vocab, tok, parent, rs_arg, o,
+                                         cache_rows, status);
+  } else {
+    k_walk_sample<<<batch, 1024, 0, st>>>(
+        tree_size, c.max_depth, c.vocab, c.top_k, n_slots, inv_t, target_logits,
+        tl_dtype == JK_BF16, tok, parent, depth, branch, qslot, draft_logits, u_accept, u_bonus,
+        rs_max, rs_sum, (float*)(ws + L.pbuf), (float*)(ws + L.qbuf), o, cache_rows, status);
+  }
+  JK_LAUNCH_CHECK(ctx);
+  if (n_layers > 0) {
+    k_compact<<<dim3(c.n_kv_heads, batch, 2 * n_layers), 256, 0, st>>>(
+        k_caches, v_caches, n_layers, cache_stride_b, cache_stride_h, row_bytes, cache_rows,
+        c.max_depth, tree_size, (const int32_t*)(ws + L.p_old), n_acc, acc_idx, es);
+    JK_LAUNCH_CHECK(ctx);
+  }
+  return JK_OK;
+}

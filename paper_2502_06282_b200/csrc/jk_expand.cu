@@ -1,0 +1,624 @@
+// jk_draft_expand and jk_tree_finalize: router, expert FFNs, shared LM head, per-expert top-k,
+// frontier selection and tree finalisation (arXiv 2502.06282, Sec. 3.1.2, Eq. 2-5).
+//
+// The dense contractions have two implementations: CUDA-core kernels in this file (exact fp32
+// accumulation, used for the f32 dtype and as a cross-check), and tcgen05 tensor-core kernels in
+// jk_gemm_tc.cu (bf16).  Everything around them (router, activation, residuals, top-k, frontier)
+// is shared.
+#include <limits.h>
+#include <math.h>
+
+#include "jk_common.cuh"
+
+// tensor-core path (jk_gemm_tc.cu)
+int jk_tc_expert_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
+                     const int32_t* expert, int do_lm_head, float* logits, int RK,
+                     int rows_per_b, long long logits_stride_b);
+int jk_tc_available(const jk_ctx* ctx);
+
+// ------------------------------------------------------------------------------------------
+// Router: RMSNorm, Eq. 2 softmax over the N centroids, Eq. 5 top-K gate.  One block per row.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) k_router(
+    const T* __restrict__ u, const T* __restrict__ router, const T* __restrict__ norm_w,
+    int H, int N, int K, float eps, int use_norm, T* __restrict__ xn,
+    float* __restrict__ out_probs, int32_t* __restrict__ out_expert, float* __restrict__ out_gate) {
+  constexpr int VN = jk_vec<T>::N;
+  __shared__ float red[33];
+  __shared__ float zs[JK_MAX_EXPERTS];
+  const int row = blockIdx.x;
+  const T* ur = u + (size_t)row * H;
+  float ss = 0.f;
+  for (int k = threadIdx.x * VN; k < H; k += blockDim.x * VN) {
+    float v[VN];
+    jk_vec<T>::load(ur + k, v);
+#pragma unroll
+    for (int i = 0; i < VN; ++i) ss += v[i] * v[i];
+  }
+  ss = jk_block_sum(ss, red);
+  const float rinv = use_norm ? rsqrtf(ss / (float)H + eps) : 1.f;
+  float z[JK_MAX_EXPERTS];
+#pragma unroll
+  for (int j = 0; j < JK_MAX_EXPERTS; ++j) z[j] = 0.f;
+  for (int k = threadIdx.x * VN; k < H; k += blockDim.x * VN) {
+    float v[VN], g[VN];
+    jk_vec<T>::load(ur + k, v);
+    if (use_norm && norm_w) {
+      jk_vec<T>::load(norm_w + k, g);
+#pragma unroll
+      for (int i = 0; i < VN; ++i) v[i] = v[i] * rinv * g[i];
+    } else {
+#pragma unroll
+      for (int i = 0; i < VN; ++i) v[i] = v[i] * rinv;
+    }
+#pragma unroll
+    for (int i = 0; i < VN; ++i) xn[(size_t)row * H + k + i] = jk_from_float<T>(v[i]);
+#pragma unroll
+    for (int j = 0; j < JK_MAX_EXPERTS; ++j) {
+      if (j < N) {
+        float e[VN];
+        jk_vec<T>::load(router + (size_t)j * H + k, e);
+#pragma unroll
+        for (int i = 0; i < VN; ++i) z[j] += v[i] * e[i];
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < JK_MAX_EXPERTS; ++j) {
+    if (j < N) {
+      float t = jk_block_sum(z[j], red);
+      if (threadIdx.x == 0) zs[j] = t;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = -INFINITY;
+    for (int j = 0; j < N; ++j) m = fmaxf(m, zs[j]);
+    float s[JK_MAX_EXPERTS], tot = 0.f;
+    for (int j = 0; j < N; ++j) { s[j] = expf(zs[j] - m); tot += s[j]; }
+    for (int j = 0; j < N; ++j) {
+      s[j] = s[j] / tot;
+      if (out_probs) out_probs[(size_t)row * N + j] = s[j];
+    }
+    unsigned taken = 0;
+    for (int r = 0; r < K; ++r) {
+      int best = -1;
+      for (int j = 0; j < N; ++j) {
+        if (taken & (1u << j)) continue;
+        if (best < 0 || s[j] > s[best]) best = j;     // ties: lower expert id stays
+      }
+      taken |= 1u << best;
+      out_expert[(size_t)row * K + r] = best;
+      out_gate[(size_t)row * K + r] = s[best];
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// CUDA-core contractions: one warp per weight row, RB activation rows at a time.
+// ------------------------------------------------------------------------------------------
+template <typename T, int RB>
+__device__ __forceinline__ void warp_rows_dot(const T* __restrict__ w, const T* __restrict__ x0,
+                                              size_t ldx, const int* rows, int nr, int Kdim,
+                                              float (&acc)[RB]) {
+  constexpr int VN = jk_vec<T>::N;
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int rb = 0; rb < RB; ++rb) acc[rb] = 0.f;
+  for (int k = lane * VN; k < Kdim; k += 32 * VN) {
+    float wv[VN];
+    jk_vec<T>::load(w + k, wv);
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) {
+      if (rb < nr) {
+        float xv[VN];
+        jk_vec<T>::load(x0 + (size_t)rows[rb] * ldx + k, xv);
+#pragma unroll
+        for (int i = 0; i < VN; ++i) acc[rb] = fmaf(wv[i], xv[i], acc[rb]);
+      }
+    }
+  }
+#pragma unroll
+  for (int rb = 0; rb < RB; ++rb) acc[rb] = jk_warp_sum(acc[rb]);
+}
+
+// rows routed to expert e, ascending
+__device__ __forceinline__ int build_expert_rows(const int32_t* expert, int R, int K, int e,
+                                                 int* list, int* count) {
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int r = 0; r < R; ++r)
+      for (int k = 0; k < K; ++k)
+        if (expert[r * K + k] == e) { list[n++] = r; break; }
+    *count = n;
+  }
+  __syncthreads();
+  return *count;
+}
+
+// h[e, r, i] = SiLU(W_gate[e, i] . x_r) * (W_up[e, i] . x_r) for the rows r routed to expert e
+template <typename T>
+__global__ void __launch_bounds__(256) k_gateup(
+    const T* __restrict__ w_gate, const T* __restrict__ w_up, const T* __restrict__ xn,
+    const int32_t* __restrict__ expert, int R, int K, int H, int I, int Rp, T* __restrict__ hbuf) {
+  constexpr int RB = 4;
+  __shared__ int list[JK_MAX_ROWS];
+  __shared__ int count;
+  const int e = blockIdx.y;
+  const int n = build_expert_rows(expert, R, K, e, list, &count);
+  if (n == 0) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int rows_per_block = 32;
+  const int i0 = blockIdx.x * rows_per_block;
+  for (int ii = warp; ii < rows_per_block; ii += nw) {
+    const int i = i0 + ii;
+    if (i >= I) break;
+    const T* wg = w_gate + ((size_t)e * I + i) * H;
+    const T* wu = w_up + ((size_t)e * I + i) * H;
+    for (int p = 0; p < n; p += RB) {
+      const int nr = min(RB, n - p);
+      float ag[RB], au[RB];
+      warp_rows_dot<T, RB>(wg, xn, H, list + p, nr, H, ag);
+      warp_rows_dot<T, RB>(wu, xn, H, list + p, nr, H, au);
+      if (lane < nr) {
+        float g = 0.f, a = 0.f;
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) if (rb == lane) { g = ag[rb]; a = au[rb]; }
+        const float hval = g / (1.f + expf(-g)) * a;
+        hbuf[((size_t)e * Rp + list[p + lane]) * I + i] = jk_from_float<T>(hval);
+      }
+    }
+  }
+}
+
+// y[e, r, o] = W_down[e, o] . h[e, r]
+template <typename T>
+__global__ void __launch_bounds__(256) k_down(
+    const T* __restrict__ w_down, const T* __restrict__ hbuf, const int32_t* __restrict__ expert,
+    int R, int K, int H, int I, int Rp, float* __restrict__ ybuf) {
+  constexpr int RB = 4;
+  __shared__ int list[JK_MAX_ROWS];
+  __shared__ int count;
+  const int e = blockIdx.y;
+  const int n = build_expert_rows(expert, R, K, e, list, &count);
+  if (n == 0) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int rows_per_block = 16;
+  const int o0 = blockIdx.x * rows_per_block;
+  const T* x0 = hbuf + (size_t)e * Rp * I;
+  for (int oo = warp; oo < rows_per_block; oo += nw) {
+    const int o = o0 + oo;
+    if (o >= H) break;
+    const T* wd = w_down + ((size_t)e * H + o) * I;
+    for (int p = 0; p < n; p += RB) {
+      const int nr = min(RB, n - p);
+      float acc[RB];
+      warp_rows_dot<T, RB>(wd, x0, I, list + p, nr, I, acc);
+      if (lane < nr) {
+        float v = 0.f;
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) if (rb == lane) v = acc[rb];
+        ybuf[((size_t)e * Rp + list[p + lane]) * H + o] = v;
+      }
+    }
+  }
+}
+
+// Eq. 3 and the branch features: f = u + sum_r g_r y_r; b_r = g_r y_r (+ u)
+template <typename T>
+__global__ void __launch_bounds__(256) k_branch(
+    const T* __restrict__ u, const float* __restrict__ ybuf, const int32_t* __restrict__ expert,
+    const float* __restrict__ gate, int K, int H, int Rp, int branch_residual,
+    T* __restrict__ bbuf, T* __restrict__ out_feat) {
+  const int r = blockIdx.x;
+  for (int h = threadIdx.x; h < H; h += blockDim.x) {
+    const float uv = jk_to_float(u[(size_t)r * H + h]);
+    float f = uv;
+    for (int k = 0; k < K; ++k) {
+      const int e = expert[r * K + k];
+      const float gy = gate[r * K + k] * ybuf[((size_t)e * Rp + r) * H + h];
+      f += gy;
+      bbuf[((size_t)r * K + k) * H + h] = jk_from_float<T>(branch_residual ? gy + uv : gy);
+    }
+    out_feat[(size_t)r * H + h] = jk_from_float<T>(f);
+  }
+}
+
+// offset of logits row rk = (b*F + f)*K + r when sequences are stride_b elements apart
+__host__ __device__ __forceinline__ size_t logit_row_off(int rk, int rows_per_b, long long stride_b,
+                                                         int V) {
+  return (size_t)(rk / rows_per_b) * (size_t)stride_b + (size_t)(rk % rows_per_b) * V;
+}
+
+// logits[rk, v] = b[rk] . W_head[v]   (Eq. 4)
+template <typename T>
+__global__ void __launch_bounds__(256) k_lmhead(
+    const T* __restrict__ lm_head, const T* __restrict__ bbuf, int RK, int H, int V,
+    float* __restrict__ logits, int rows_per_b, long long stride_b) {
+  constexpr int RB = 8;
+  __shared__ int ident[JK_MAX_ROWS * JK_MAX_EXPERTS];
+  for (int i = threadIdx.x; i < RK; i += blockDim.x) ident[i] = i;
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int rows_per_block = 32;
+  const int v0 = blockIdx.x * rows_per_block;
+  for (int vv = warp; vv < rows_per_block; vv += nw) {
+    const int v = v0 + vv;
+    if (v >= V) break;
+    const T* wr = lm_head + (size_t)v * H;
+    for (int p = 0; p < RK; p += RB) {
+      const int nr = min(RB, RK - p);
+      float acc[RB];
+      warp_rows_dot<T, RB>(wr, bbuf, H, ident + p, nr, H, acc);
+      if (lane < nr) {
+        float val = 0.f;
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) if (rb == lane) val = acc[rb];
+        logits[logit_row_off(p + lane, rows_per_b, stride_b, V) + v] = val;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-expert top-k over the vocabulary: partial pass per 4096-entry chunk, then a merge.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_topk_partial(
+    const float* __restrict__ logits, int rows_per_b, long long stride_b, int V, int k_e,
+    int chunks, float* __restrict__ tk_val, int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
+  constexpr int PER = JK_TOPK_CHUNK / 256;
+  __shared__ float red[33];
+  __shared__ float wv[8];
+  __shared__ int wi[8];
+  __shared__ int win_idx;
+  const int chunk = blockIdx.x, row = blockIdx.y;
+  const float* lr = logits + logit_row_off(row, rows_per_b, stride_b, V);
+  const int base = chunk * JK_TOPK_CHUNK;
+  float vals[PER];
+  float lmax = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int idx = base + threadIdx.x + j * 256;
+    vals[j] = idx < V ? lr[idx] : -INFINITY;
+    lmax = fmaxf(lmax, vals[j]);
+  }
+  const float bmax = jk_block_max(lmax, red);
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) {
+    const int idx = base + threadIdx.x + j * 256;
+    if (idx < V) s += expf(vals[j] - bmax);
+  }
+  const float bsum = jk_block_sum(s, red);
+  const size_t prow = (size_t)row * chunks + chunk;
+  if (threadIdx.x == 0) { tk_ms[prow * 2] = bmax; tk_ms[prow * 2 + 1] = bsum; }
+  unsigned taken = 0;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int it = 0; it < k_e; ++it) {
+    float bv = -INFINITY;
+    int bi = INT_MAX;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+      const int idx = base + threadIdx.x + j * 256;
+      if (!(taken & (1u << j)) && idx < V && jk_better(vals[j], idx, bv, bi)) { bv = vals[j]; bi = idx; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (jk_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float fv = wv[0];
+      int fi = wi[0];
+      for (int w = 1; w < 8; ++w)
+        if (jk_better(wv[w], wi[w], fv, fi)) { fv = wv[w]; fi = wi[w]; }
+      tk_val[prow * k_e + it] = fv;
+      tk_idx[prow * k_e + it] = fi;
+      win_idx = fi;
+    }
+    __syncthreads();
+    const int wsel = win_idx;
+    if (wsel != INT_MAX) {
+#pragma unroll
+      for (int j = 0; j < PER; ++j)
+        if (base + threadIdx.x + j * 256 == wsel) taken |= 1u << j;
+    }
+    __syncthreads();
+  }
+}
+
+// Merge the chunk partials of every logits row of one sequence, append the children to the
+// pool, then pick the next frontier.  One block per sequence.
+__global__ void __launch_bounds__(256) k_expand_finish(
+    int F, int K, int k_e, int chunks, int width,
+    const float* __restrict__ tk_val, const int32_t* __restrict__ tk_idx,
+    const float* __restrict__ tk_ms, const float* __restrict__ parent_score,
+    const int32_t* __restrict__ parent_gidx, int gidx_base, int slot_base,
+    jk_pool pool, float* __restrict__ out_lse, int32_t* __restrict__ next_frontier,
+    float* __restrict__ next_parent_score, int32_t* __restrict__ next_parent_gidx) {
+  __shared__ float sc[JK_MAX_POOL];
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int rows = F * K;
+  const size_t pb = (size_t)b * pool.stride_b;
+  for (int lr = warp; lr < rows; lr += nw) {
+    const int f = lr / K, r = lr % K;
+    const size_t row = (size_t)b * rows + lr;
+    // log-sum-exp over the chunk statistics
+    float m = -INFINITY;
+    for (int c = lane; c < chunks; c += 32) m = fmaxf(m, tk_ms[(row * chunks + c) * 2]);
+    m = jk_warp_max(m);
+    float s = 0.f;
+    for (int c = lane; c < chunks; c += 32)
+      s += tk_ms[(row * chunks + c) * 2 + 1] * expf(tk_ms[(row * chunks + c) * 2] - m);
+    s = jk_warp_sum(s);
+    const float lse = m + logf(s);
+    if (out_lse && lane == 0) out_lse[row] = lse;
+    // top-k_e of the chunks * k_e partial winners
+    const int nc = chunks * k_e;
+    const int per = (nc + 31) / 32;            // <= 16 with <= 32 chunks; more chunks loop below
+    unsigned long long taken = 0ull;
+    const float ps = parent_score[(size_t)b * F + f];
+    const int pg = parent_gidx[(size_t)b * F + f];
+    for (int it = 0; it < k_e; ++it) {
+      float bv = -INFINITY;
+      int bi = INT_MAX, bj = -1;
+      for (int j = 0; j < per && j < 64; ++j) {
+        const int c = lane + j * 32;
+        if (c < nc && !(taken & (1ull << j))) {
+          const float v = tk_val[row * nc + c];
+          const int i = tk_idx[row * nc + c];
+          if (jk_better(v, i, bv, bi)) { bv = v; bi = i; bj = j; }
+        }
+      }
+      float wv = bv;
+      int wi = bi;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+        if (jk_better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
+      }
+      if (wi == bi && bj >= 0 && wi != INT_MAX) taken |= 1ull << bj;
+      if (lane == 0) {
+        const int flat = lr * k_e + it;
+        const int g = gidx_base + flat;
+        const float score = ps + (wv - lse);
+        pool.tok[pb + g] = wi;
+        pool.score[pb + g] = score;
+        pool.parent[pb + g] = pg;
+        pool.qslot[pb + g] = -1;
+        pool.branch[pb + g] = r;
+        sc[flat] = score;
+      }
+    }
+  }
+  __syncthreads();
+  if (width <= 0 || !next_frontier) return;
+  const int n = rows * k_e;
+  const int wsel = min(width, n);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const float v = sc[i];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) rank += jk_better(sc[j], j, v, i) ? 1 : 0;
+    if (rank < wsel) {
+      next_frontier[(size_t)b * wsel + rank] = i;
+      next_parent_score[(size_t)b * wsel + rank] = v;
+      next_parent_gidx[(size_t)b * wsel + rank] = gidx_base + i;
+      pool.qslot[pb + gidx_base + i] = slot_base + F + rank;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Tree finalisation: top (M-1) of the pool, ascending generation order, ancestor bitsets.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) k_tree_finalize(
+    jk_pool pool, int pool_n, const int32_t* __restrict__ root_tok, int M,
+    int32_t* __restrict__ tok, int32_t* __restrict__ parent, int32_t* __restrict__ depth,
+    int32_t* __restrict__ branch, int32_t* __restrict__ qslot, unsigned long long* __restrict__ anc,
+    int32_t* status) {
+  __shared__ float sc[JK_MAX_POOL];
+  __shared__ short newid[JK_MAX_POOL];      // 0 = dropped, else node index
+  __shared__ int par_s[JK_MAX_TREE];
+  __shared__ int scan[1024];
+  const int b = blockIdx.x;
+  const size_t pb = (size_t)b * pool.stride_b;
+  const int t = threadIdx.x;
+  for (int g = t; g < pool_n; g += blockDim.x) sc[g] = pool.score[pb + g];
+  __syncthreads();
+  const int m1 = M - 1;
+  // each thread owns a contiguous slice so that the prefix sum runs in generation order
+  const int per = (pool_n + blockDim.x - 1) / blockDim.x;
+  const int g0 = t * per, g1 = min(pool_n, g0 + per);
+  int cnt = 0;
+  unsigned keepmask = 0;                     // per <= 4 for pool_n <= 4096
+  for (int g = g0; g < g1; ++g) {
+    const float v = sc[g];
+    int rank = 0;
+    for (int j = 0; j < pool_n; ++j) rank += jk_better(sc[j], j, v, g) ? 1 : 0;
+    if (rank < m1) { keepmask |= 1u << (g - g0); ++cnt; }
+  }
+  scan[t] = cnt;
+  __syncthreads();
+  for (int off = 1; off < (int)blockDim.x; off <<= 1) {
+    int v = t >= off ? scan[t - off] : 0;
+    __syncthreads();
+    scan[t] += v;
+    __syncthreads();
+  }
+  int id = 1 + scan[t] - cnt;
+  for (int g = g0; g < g1; ++g) newid[g] = (keepmask >> (g - g0)) & 1u ? (short)(id++) : (short)0;
+  __syncthreads();
+  const size_t ob = (size_t)b * M;
+  if (t == 0) {
+    tok[ob] = root_tok[b];
+    parent[ob] = -1;
+    depth[ob] = 0;
+    branch[ob] = 0;
+    qslot[ob] = 0;
+    par_s[0] = -1;
+  }
+  for (int g = g0; g < g1; ++g) {
+    const int i = newid[g];
+    if (!i) continue;
+    const int pg = pool.parent[pb + g];
+    int p = 0;
+    if (pg >= 0) {
+      p = (pg < pool_n) ? newid[pg] : 0;
+      if (p == 0 || p >= i) { jk_set_status(status, JK_ERR_BOUNDS); p = 0; }
+    }
+    tok[ob + i] = pool.tok[pb + g];
+    parent[ob + i] = p;
+    par_s[i] = p;
+    branch[ob + i] = pool.branch[pb + g];
+    qslot[ob + i] = pool.qslot[pb + g];
+  }
+  __syncthreads();
+  if (t < M) {
+    unsigned long long lo = 0ull, hi = 0ull;
+    int d = -1, c = t;
+    for (int guard = 0; c >= 0 && guard <= JK_MAX_TREE; ++guard) {
+      if (c < 64) lo |= 1ull << c; else hi |= 1ull << (c - 64);
+      ++d;
+      c = par_s[c];
+    }
+    depth[ob + t] = d;
+    anc[(ob + t) * 2] = lo;
+    anc[(ob + t) * 2 + 1] = hi;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+template <typename T>
+static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int B, int F,
+                       int width, const void* u, const float* parent_score,
+                       const int32_t* parent_gidx, int gidx_base, int slot_base, float* out_probs,
+                       int32_t* out_expert, float* out_gate, const jk_pool* pool, float* out_lse,
+                       void* out_feat, float* out_logits, int64_t logits_stride_b,
+                       int32_t* next_frontier, float* next_parent_score,
+                       int32_t* next_parent_gidx) {
+  const jk_config& c = ctx->cfg;
+  const jk_ws_layout& L = ctx->lay;
+  const int R = B * F, K = c.top_k, RK = R * K, H = c.hidden, I = c.inter, V = c.vocab;
+  const int Rp = L.rows_pad;
+  char* ws = ctx->ws;
+  T* xn = (T*)(ws + L.xn);
+  T* hbuf = (T*)(ws + L.hbuf);
+  float* ybuf = (float*)(ws + L.ybuf);
+  T* bbuf = (T*)(ws + L.bbuf);
+  float* logits = out_logits ? out_logits : (float*)(ws + L.logits);
+  const int rows_per_b = F * K;
+  const long long lsb = (out_logits && logits_stride_b) ? logits_stride_b : (long long)rows_per_b * V;
+
+  k_router<T><<<R, 256, 0, st>>>((const T*)u, (const T*)w->router, (const T*)w->norm_weight, H,
+                                 c.n_experts, K, c.rms_eps, c.use_pre_norm, xn, out_probs,
+                                 out_expert, out_gate);
+  JK_LAUNCH_CHECK(ctx);
+  const bool tc = ctx->tensor_path && c.dtype == JK_BF16 && jk_tc_available(ctx);
+  if (tc) {
+    int rc = jk_tc_expert_ffn(ctx, st, w, R, out_expert, 0, nullptr, RK, rows_per_b, lsb);
+    if (rc != JK_OK) return rc;
+  } else {
+    k_gateup<T><<<dim3((I + 31) / 32, c.n_experts), 256, 0, st>>>(
+        (const T*)w->w_gate, (const T*)w->w_up, xn, out_expert, R, K, H, I, Rp, hbuf);
+    JK_LAUNCH_CHECK(ctx);
+    k_down<T><<<dim3((H + 15) / 16, c.n_experts), 256, 0, st>>>(
+        (const T*)w->w_down, hbuf, out_expert, R, K, H, I, Rp, ybuf);
+    JK_LAUNCH_CHECK(ctx);
+  }
+  k_branch<T><<<R, 256, 0, st>>>((const T*)u, ybuf, out_expert, out_gate, K, H, Rp,
+                                 c.branch_residual, bbuf, (T*)out_feat);
+  JK_LAUNCH_CHECK(ctx);
+  if (tc) {
+    int rc = jk_tc_expert_ffn(ctx, st, w, R, out_expert, 1, logits, RK, rows_per_b, lsb);
+    if (rc != JK_OK) return rc;
+  } else {
+    k_lmhead<T><<<(V + 31) / 32, 256, 0, st>>>((const T*)w->lm_head, bbuf, RK, H, V, logits,
+                                               rows_per_b, lsb);
+    JK_LAUNCH_CHECK(ctx);
+  }
+  k_topk_partial<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
+      logits, rows_per_b, lsb, V, c.k_per_expert, L.topk_chunks, (float*)(ws + L.tk_val),
+      (int32_t*)(ws + L.tk_idx), (float*)(ws + L.tk_ms));
+  JK_LAUNCH_CHECK(ctx);
+  k_expand_finish<<<B, 256, 0, st>>>(F, K, c.k_per_expert, L.topk_chunks, width,
+                                     (const float*)(ws + L.tk_val),
+                                     (const int32_t*)(ws + L.tk_idx),
+                                     (const float*)(ws + L.tk_ms), parent_score, parent_gidx,
+                                     gidx_base, slot_base, *pool, out_lse, next_frontier,
+                                     next_parent_score, next_parent_gidx);
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
+
+extern "C" int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* w,
+                               int32_t batch, int32_t n_frontier, int32_t width, const void* u,
+                               const float* parent_score, const int32_t* parent_gidx,
+                               int32_t gidx_base, int32_t slot_base, float* out_probs,
+                               int32_t* out_expert, float* out_gate, const jk_pool* pool,
+                               float* out_lse, void* out_feat, float* out_logits,
+                               int64_t logits_stride_b, int32_t* next_frontier,
+                               float* next_parent_score, int32_t* next_parent_gidx) {
+  if (!ctx || !w || !u || !parent_score || !parent_gidx || !out_expert || !out_gate || !pool ||
+      !out_feat)
+    return JK_ERR_NULL;
+  if (!w->router || !w->w_gate || !w->w_up || !w->w_down || !w->lm_head) return JK_ERR_NULL;
+  if (!pool->tok || !pool->score || !pool->parent || !pool->qslot || !pool->branch)
+    return JK_ERR_NULL;
+  if (width > 0 && (!next_frontier || !next_parent_score || !next_parent_gidx)) return JK_ERR_NULL;
+  const jk_config& c = ctx->cfg;
+  if (batch < 1 || n_frontier < 1 || width < 0 || gidx_base < 0 || slot_base < 0)
+    return JK_ERR_SHAPE;
+  if (batch > c.max_batch || n_frontier > c.max_frontier) return JK_ERR_CAPACITY;
+  const int n_cand = n_frontier * c.top_k * c.k_per_expert;
+  if (n_cand > JK_MAX_POOL) return JK_ERR_SHAPE;
+  if (pool->stride_b < (int64_t)gidx_base + n_cand) return JK_ERR_SHAPE;
+  if (logits_stride_b < 0 || logits_stride_b % 4 ||
+      (logits_stride_b && logits_stride_b < (int64_t)n_frontier * c.top_k * c.vocab))
+    return JK_ERR_SHAPE;
+  if (!ctx->ws) return JK_ERR_WORKSPACE;
+  const void* ptrs[] = {u, w->router, w->w_gate, w->w_up, w->w_down, w->lm_head, w->norm_weight,
+                        out_feat, out_logits};
+  for (const void* p : ptrs)
+    if (p && !jk_aligned16(p)) return JK_ERR_ALIGN;
+  int rc = jk_ensure_device_info(ctx);
+  if (rc != JK_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (c.dtype == JK_BF16)
+    return expand_impl<__nv_bfloat16>(ctx, st, w, batch, n_frontier, width, u, parent_score,
+                                      parent_gidx, gidx_base, slot_base, out_probs, out_expert,
+                                      out_gate, pool, out_lse, out_feat, out_logits,
+                                      logits_stride_b, next_frontier, next_parent_score,
+                                      next_parent_gidx);
+  return expand_impl<float>(ctx, st, w, batch, n_frontier, width, u, parent_score, parent_gidx,
+                            gidx_base, slot_base, out_probs, out_expert, out_gate, pool, out_lse,
+                            out_feat, out_logits, logits_stride_b, next_frontier,
+                            next_parent_score, next_parent_gidx);
+}
+
+extern "C" int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const jk_pool* pool,
+                                int32_t pool_n, const int32_t* root_tok, int32_t tree_size,
+                                int32_t* tok, int32_t* parent, int32_t* depth, int32_t* branch,
+                                int32_t* qslot, uint64_t* anc) {
+  if (!ctx || !pool || !root_tok || !tok || !parent || !depth || !branch || !qslot || !anc)
+    return JK_ERR_NULL;
+  if (!pool->tok || !pool->score || !pool->parent || !pool->qslot || !pool->branch)
+    return JK_ERR_NULL;
+  if (batch < 1 || tree_size < 1 || pool_n < 0) return JK_ERR_SHAPE;
+  if (batch > ctx->cfg.max_batch || tree_size > ctx->cfg.max_tree) return JK_ERR_CAPACITY;
+  if (pool_n > JK_MAX_POOL || pool_n < tree_size - 1 || pool->stride_b < pool_n)
+    return JK_ERR_SHAPE;
+  if (!ctx->ws) return JK_ERR_WORKSPACE;
+  k_tree_finalize<<<batch, 1024, 0, (cudaStream_t)stream>>>(
+      *pool, pool_n, root_tok, tree_size, tok, parent, depth, branch, qslot,
+      (unsigned long long*)anc, (int32_t*)(ctx->ws + ctx->lay.status));
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
