@@ -583,11 +583,11 @@ extern "C" int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights
   if (logits_stride_b < 0 || logits_stride_b % 4 ||
       (logits_stride_b && logits_stride_b < (int64_t)n_frontier * c.top_k * c.vocab))
     return JK_ERR_SHAPE;
-  if (!ctx->ws) return JK_ERR_WORKSPACE;
   const void* ptrs[] = {u, w->router, w->w_gate, w->w_up, w->w_down, w->lm_head, w->norm_weight,
                         out_feat, out_logits};
   for (const void* p : ptrs)
     if (p && !jk_aligned16(p)) return JK_ERR_ALIGN;
+  if (!ctx->ws) return JK_ERR_WORKSPACE;
   int rc = jk_ensure_device_info(ctx);
   if (rc != JK_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;

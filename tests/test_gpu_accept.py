@@ -1,0 +1,201 @@
+"""GPU parity of jk_accept_and_compact: bit-exact paths, tokens, lengths and caches."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import jakiro_oracle as orc
+from paper_2502_06282_b200 import binding as jk
+from paper_2502_06282_b200 import synth
+from tests.jk_testutil import dev, host
+
+pytestmark = pytest.mark.gpu
+
+
+def _tree_arrays(w, kind, seed):
+    B, M = w.batch, w.tree_size
+    if kind == "random":
+        parent = np.stack([synth.random_tree(M, w.depth, seed + b) for b in range(B)])
+    elif kind == "chain":
+        parent = np.stack([synth.chain_tree(M)] * B)
+    else:
+        parent = np.stack([synth.star_tree(M)] * B)
+    depth = np.stack([synth.tree_depths(p) for p in parent])
+    rng = np.random.default_rng(seed)
+    tok = rng.integers(0, w.vocab, size=(B, M)).astype(np.int32)
+    branch = rng.integers(0, w.top_k, size=(B, M)).astype(np.int32)
+    # children of one parent: left branch first, as the expand step orders them
+    for b in range(B):
+        for i in range(M):
+            kids = orc.children_of(parent[b], i)
+            branch[b, kids] = np.sort(branch[b, kids])
+    branch[:, 0] = 0
+    # internal nodes own a slot of draft logits
+    qslot = np.full((B, M), -1, dtype=np.int32)
+    n_slots = 0
+    for b in range(B):
+        s = 0
+        for i in range(M):
+            if orc.children_of(parent[b], i):
+                qslot[b, i] = s
+                s += 1
+        n_slots = max(n_slots, s)
+    return {"tok": tok, "parent": parent.astype(np.int32), "depth": depth.astype(np.int32),
+            "branch": branch, "qslot": qslot}, n_slots
+
+
+def _caches(w, L, dtype, seed):
+    out = []
+    for l in range(L):
+        _, k, v, _ = synth.attn_inputs(synth.scaled(w, dtype=dtype, seed=seed), layer=l)
+        out.append((k, v))
+    return out
+
+
+def _call(w, tree, mode, T, tl, dl, n_slots, ua, ub, caches, kv_len, dtype, tl_bf16=False):
+    ctx = jk.Context.for_workload(synth.scaled(w, dtype=dtype))
+    B, M, D = w.batch, w.tree_size, w.depth
+    tr = {k: dev(v) for k, v in tree.items()}
+    kd = [dev(k, dtype) for k, _ in caches]
+    vd = [dev(v, dtype) for _, v in caches]
+    kp = torch.tensor([t.data_ptr() for t in kd], dtype=torch.int64, device="cuda")
+    vp = torch.tensor([t.data_ptr() for t in vd], dtype=torch.int64, device="cuda")
+    kvl = dev(kv_len.copy())
+    i32 = dict(dtype=torch.int32, device="cuda")
+    n_acc, bonus = torch.empty(B, **i32), torch.empty(B, **i32)
+    acc_idx, acc_tok = torch.empty(B, D, **i32), torch.empty(B, D, **i32)
+    tld = dev(tl, "bf16" if tl_bf16 else None)
+    L = len(caches)
+    ctx.accept_and_compact(B, M, mode, T, tld, tr, None if dl is None else dev(dl), n_slots,
+                           None if ua is None else dev(ua), None if ub is None else dev(ub), L,
+                           kp if L else None, vp if L else None,
+                           kd[0].stride(0) if L else 0, kd[0].stride(1) if L else 0,
+                           w.kv_capacity, kvl, n_acc, acc_idx, acc_tok, bonus)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    return (host(n_acc), host(acc_idx), host(acc_tok), host(bonus), host(kvl),
+            [host(t) for t in kd], [host(t) for t in vd])
+
+
+def _check_compaction(w, caches, kv_len, paths, got_k, got_v):
+    for l, (k, v) in enumerate(caches):
+        for b in range(w.batch):
+            assert np.array_equal(got_k[l][b], orc.compact_kv(k[b], int(kv_len[b]), paths[b]))
+            assert np.array_equal(got_v[l][b], orc.compact_kv(v[b], int(kv_len[b]), paths[b]))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("alpha", [0.0, 0.8, 1.0])
+@pytest.mark.parametrize("kind", ["random", "chain", "star"])
+def test_greedy_accept_and_compaction(dtype, alpha, kind):
+    w = synth.scaled(synth.WORKLOADS["tiny"], batch=3, vocab=4100 if dtype == "f32" else 4096)
+    tree, n_slots = _tree_arrays(w, kind, 11)
+    tl = synth.target_logits(w, tree["tok"], tree["parent"], alpha)
+    caches = _caches(w, 2, dtype, 500)
+    kv_len = np.array([w.prefix, w.prefix - 7, 3], dtype=np.int32)
+    n_acc, acc_idx, acc_tok, bonus, kvl, gk, gv = _call(w, tree, 0, 0.0, tl, None, 0, None, None,
+                                                        caches, kv_len, dtype)
+    paths = []
+    for b in range(w.batch):
+        path, toks, bo = orc.accept_greedy(tl[b], tree["tok"][b], tree["parent"][b])
+        paths.append(path)
+        assert n_acc[b] == len(path) and bonus[b] == bo
+        assert acc_idx[b, :len(path)].tolist() == path and acc_tok[b, :len(path)].tolist() == toks
+        assert np.all(acc_idx[b, len(path):] == -1)
+        assert kvl[b] == kv_len[b] + 1 + len(path)
+    if alpha == 1.0 and kind == "chain":
+        assert all(len(p) == w.depth for p in paths) or w.tree_size - 1 < w.depth
+    _check_compaction(w, caches, kv_len, paths, gk, gv)
+
+
+def test_greedy_bf16_target_logits_and_ties():
+    w = synth.scaled(synth.WORKLOADS["tiny"], batch=2)
+    tree, _ = _tree_arrays(w, "random", 12)
+    tl = synth.bf16_round(synth.target_logits(w, tree["tok"], tree["parent"], 0.8))
+    tl[0, 0, :] = 0.0                      # an all-equal row: top-1 must be token 0
+    n_acc, acc_idx, acc_tok, bonus, *_ = _call(w, tree, 0, 0.0, tl, None, 0, None, None, [],
+                                               np.array([5, 5], np.int32), "f32", tl_bf16=True)
+    for b in range(2):
+        path, toks, bo = orc.accept_greedy(tl[b], tree["tok"][b], tree["parent"][b])
+        assert acc_idx[b, :n_acc[b]].tolist() == path and bonus[b] == bo
+
+
+def _near_tie(trace, ua):
+    """True if some decision of the oracle's walk sits within rounding of its threshold."""
+    for t in trace:
+        if "child" in t and abs(float(ua[t["child"]]) - t["ratio"]) <= 1e-4 * max(t["ratio"], 1e-30):
+            return True
+    return False
+
+
+@pytest.mark.parametrize("kind,alpha,agree", [("random", 0.8, 0.0), ("random", 0.0, 0.0),
+                                              ("chain", 0.8, 1.0), ("star", 0.8, 0.5),
+                                              ("random", 1.0, 1.0)])
+def test_sampling_accept(kind, alpha, agree):
+    w = synth.scaled(synth.WORKLOADS["tiny"], batch=4, vocab=2000, seed=1234)
+    tree, n_slots = _tree_arrays(w, kind, 21)
+    tl = synth.target_logits(w, tree["tok"], tree["parent"], alpha, boost=6.0)
+    rng = np.random.default_rng(5)
+    dl = (rng.standard_normal((w.batch, n_slots, w.top_k, w.vocab)) * 2).astype(np.float32)
+    # `agree` blends the target's row into the draft rows so that acceptances happen
+    for b in range(w.batch):
+        for i in range(w.tree_size):
+            s = tree["qslot"][b, i]
+            if s >= 0:
+                dl[b, s] = (1 - agree) * dl[b, s] + agree * tl[b, i][None]
+                for c in orc.children_of(tree["parent"][b], i):
+                    dl[b, s, tree["branch"][b, c], tree["tok"][b, c]] += 4.0
+    ua, ub = synth.uniforms(w)
+    caches = _caches(w, 1, "bf16", 600)
+    kv_len = np.array([w.prefix, 9, 64, 1], dtype=np.int32)
+    n_acc, acc_idx, acc_tok, bonus, kvl, gk, gv = _call(w, tree, 1, 1.0, tl, dl, n_slots, ua, ub,
+                                                        caches, kv_len, "bf16")
+    paths = []
+    ties = 0
+    for b in range(w.batch):
+        trace = []
+        path, toks, bo = orc.accept_sampling(tl[b], tree["tok"][b], tree["parent"][b],
+                                             tree["depth"][b], tree["branch"][b],
+                                             tree["qslot"][b], dl[b], ua[b], ub[b], 1.0,
+                                             trace=trace)
+        got_path = acc_idx[b, :n_acc[b]].tolist()
+        if got_path != path or bonus[b] != bo:
+            # only acceptable inside the tie band: the GPU decides in fp32
+            cdf_edge = False
+            if got_path == path:
+                p = orc.softmax(tl[b, path[-1] if path else 0])   # coarse: only no-reject walks
+                c = np.cumsum(p)
+                u = float(ub[b, tree["depth"][b][path[-1]] if path else 0])
+                cdf_edge = np.min(np.abs(c - u)) < 1e-5
+            assert _near_tie(trace, ua[b]) or cdf_edge, (b, got_path, path, bonus[b], bo)
+            ties += 1
+            paths.append(got_path)
+            continue
+        paths.append(path)
+        assert acc_tok[b, :len(path)].tolist() == toks
+        assert kvl[b] == kv_len[b] + 1 + len(path)
+    assert ties <= 1
+    _check_compaction(w, caches, kv_len, paths, gk, gv)
+
+
+def test_accept_llama2_7b_shape():
+    """Benchmark shape: M = 60, V = 32000, 32 layers of bf16 caches; greedy and sampling."""
+    w = synth.scaled(synth.WORKLOADS["llama2_7b"], n_layers=4)
+    tree, n_slots = _tree_arrays(w, "random", 31)
+    tl = synth.target_logits(w, tree["tok"], tree["parent"], 0.8)
+    caches = _caches(w, 4, "bf16", 700)
+    kv_len = np.array([w.prefix], dtype=np.int32)
+    n_acc, acc_idx, acc_tok, bonus, kvl, gk, gv = _call(w, tree, 0, 0.0, tl, None, 0, None, None,
+                                                        caches, kv_len, "bf16")
+    path, toks, bo = orc.accept_greedy(tl[0], tree["tok"][0], tree["parent"][0])
+    assert acc_idx[0, :n_acc[0]].tolist() == path and bonus[0] == bo
+    _check_compaction(w, caches, kv_len, [path], gk, gv)
+    rng = np.random.default_rng(6)
+    dl = rng.standard_normal((1, n_slots, 2, w.vocab)).astype(np.float32)
+    ua, ub = synth.uniforms(w)
+    n_acc, acc_idx, acc_tok, bonus, *_ = _call(w, tree, 1, 1.0, tl, dl, n_slots, ua, ub, [],
+                                               kv_len, "bf16")
+    trace = []
+    path, toks, bo = orc.accept_sampling(tl[0], tree["tok"][0], tree["parent"][0],
+                                         tree["depth"][0], tree["branch"][0], tree["qslot"][0],
+                                         dl[0], ua[0], ub[0], 1.0, trace=trace)
+    assert (acc_idx[0, :n_acc[0]].tolist() == path and bonus[0] == bo) or _near_tie(trace, ua[0])

@@ -1,0 +1,194 @@
+"""GPU parity of jk_draft_expand / jk_tree_finalize against the CPU oracle.
+
+Floating stages are compared by tolerance with the oracle's own computation on the same inputs;
+every discrete decision (experts, top-k tokens, frontier, final tree) is re-derived by the oracle
+from the GPU's floating inputs to that decision and compared exactly.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import jakiro_oracle as orc
+from paper_2502_06282_b200 import binding as jk
+from paper_2502_06282_b200 import synth
+from tests.jk_testutil import TOL, dev, host, rel_err, weights_to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_gpu(w, wts_np, us_np, tensor_path=None, root_tok=5):
+    ctx = jk.Context.for_workload(w)
+    if tensor_path is not None:
+        ctx.set_tensor_path(tensor_path)
+    bufs = jk.StepBuffers(ctx, w)
+    wts = weights_to_device(wts_np, w.dtype)
+    us = [dev(u, w.dtype) for u in us_np]
+    root = torch.full((w.batch,), root_tok, dtype=torch.int32, device="cuda")
+    jk.run_draft(ctx, bufs, wts, us, root)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    return ctx, bufs
+
+
+def _check_layers(w, wts_np, us_np, bufs):
+    tol = TOL[w.dtype]
+    fs = w.frontier_sizes
+    K, ke = w.top_k, w.k_per_expert
+    gidx_base, slot_base = 0, 0
+    pool = {k: host(v) for k, v in bufs.pool.items()}
+    logits_all = host(bufs.logits)
+    for l, F in enumerate(fs):
+        u = us_np[l].astype(np.float64)
+        pscore = host(bufs.parent_score[l]).astype(np.float64)
+        pgidx = host(bufs.parent_gidx[l])
+        probs_g, exp_g, gate_g = host(bufs.probs[l]), host(bufs.expert[l]), host(bufs.gate[l])
+        feat_g, lse_g = host(bufs.feat[l]), host(bufs.lse[l])
+        x = orc.rmsnorm(u, wts_np["norm_weight"], 1e-5)
+        probs_o = orc.router_scores(x, wts_np["router"])
+        assert rel_err(probs_g, probs_o) <= tol
+        n_cand = F * K * ke
+        for b in range(w.batch):
+            for f in range(F):
+                # experts: replayed from the GPU's own scores, exact
+                ids_r, g_r = orc.topk_gate(probs_g[b, f], K)
+                assert exp_g[b, f].tolist() == ids_r.tolist()
+                assert np.array_equal(gate_g[b, f], probs_g[b, f][ids_r])
+                ids_o, _ = orc.topk_gate(probs_o[b, f], K)
+                margin = np.sort(probs_o[b, f])[::-1]
+                if margin[K - 1] - margin[K] > 1e-3 and (K < 2 or margin[0] - margin[1] > 1e-3):
+                    assert ids_o.tolist() == ids_r.tolist()
+                _, br, ff = orc.moe_features(u[b, f], x[b, f], ids_r, probs_o[b, f][ids_r], wts_np)
+                assert rel_err(feat_g[b, f], ff) <= tol
+                lg_o = orc.head_logits(br, wts_np["lm_head"])
+                lg_g = logits_all[b, slot_base + f]
+                assert rel_err(lg_g, lg_o) <= tol
+                for r in range(K):
+                    # top-k tokens and scores: replayed from the GPU's logits
+                    ids_t, sc_t, lse_t = orc.branch_topk(lg_g[r], ke, pscore[b, f])
+                    g0 = gidx_base + (f * K + r) * ke
+                    assert pool["tok"][b, g0:g0 + ke].tolist() == ids_t.tolist()
+                    assert np.allclose(pool["score"][b, g0:g0 + ke], sc_t, rtol=1e-5, atol=2e-5)
+                    assert abs(lse_g[b, f, r] - lse_t) <= 2e-5 * max(1.0, abs(lse_t))
+                    assert np.all(pool["parent"][b, g0:g0 + ke] == pgidx[b, f])
+                    assert np.all(pool["branch"][b, g0:g0 + ke] == r)
+            if l < len(fs) - 1:
+                sel = orc.frontier_select(pool["score"][b, gidx_base:gidx_base + n_cand],
+                                          min(w.width, n_cand))
+                assert host(bufs.frontier[l])[b].tolist() == sel.tolist()
+                assert np.array_equal(host(bufs.parent_score[l + 1])[b],
+                                      pool["score"][b, gidx_base + sel])
+                assert host(bufs.parent_gidx[l + 1])[b].tolist() == (gidx_base + sel).tolist()
+                q = np.full(n_cand, -1)
+                q[sel] = slot_base + F + np.arange(len(sel))
+                assert pool["qslot"][b, gidx_base:gidx_base + n_cand].tolist() == q.tolist()
+            else:
+                assert np.all(pool["qslot"][b, gidx_base:gidx_base + n_cand] == -1)
+        gidx_base += n_cand
+        slot_base += F
+    return pool
+
+
+def _check_tree(w, pool, bufs, root_tok):
+    for b in range(w.batch):
+        t = orc.tree_finalize(pool["tok"][b], pool["score"][b], pool["parent"][b],
+                              pool["qslot"][b], root_tok, w.tree_size,
+                              pool_branch=pool["branch"][b])
+        for key in ("tok", "parent", "depth", "branch", "qslot"):
+            assert host(bufs.tree[key])[b].tolist() == t[key].tolist(), key
+        anc = orc.ancestor_mask(t["parent"])
+        bits = host(bufs.anc)[b].astype(np.uint64)
+        for i in range(w.tree_size):
+            got = [(int(bits[i, c >> 6]) >> (c & 63)) & 1 for c in range(w.tree_size)]
+            assert got == anc[i].astype(int).tolist()
+
+
+def _inputs(w):
+    wts = synth.draft_weights(w)
+    us = [synth.layer_hidden(w, l, F) for l, F in enumerate(w.frontier_sizes)]
+    return wts, us
+
+
+@pytest.mark.parametrize("name,tensor_path", [("tiny", None), ("tiny_bf16", False),
+                                              ("tiny_bf16", True)])
+def test_expand_tiny_full_parity(name, tensor_path):
+    w = synth.WORKLOADS[name]
+    wts, us = _inputs(w)
+    ctx, bufs = _run_gpu(w, wts, us, tensor_path)
+    pool = _check_layers(w, wts, us, bufs)
+    _check_tree(w, pool, bufs, 5)
+    if w.dtype == "f32":
+        # no near-ties in this seeded case: the oracle's own tree is the same tree
+        ref = orc.grow_tree(us, wts, w.k_per_expert, w.width)
+        t = orc.tree_finalize(ref["tok"][0], ref["score"][0], ref["parent"][0], ref["qslot"][0],
+                              5, w.tree_size, frontier_sizes=w.frontier_sizes,
+                              top_k=w.top_k, k_e=w.k_per_expert)
+        assert host(bufs.tree["tok"])[0].tolist() == t["tok"].tolist()
+        assert host(bufs.tree["parent"])[0].tolist() == t["parent"].tolist()
+
+
+@pytest.mark.parametrize("tensor_path", [False, True])
+def test_expand_batched_ragged_shapes(tensor_path):
+    # batch 3, vocabulary and inner size that end in partial tiles, N = 3 experts, k_e = 3
+    w = synth.scaled(synth.WORKLOADS["tiny_bf16"], name="ragged", batch=3, vocab=5000,
+                     inter=1000, hidden=264, n_experts=3, k_per_expert=3, width=5,
+                     tree_size=20, depth=3, seed=77)
+    wts, us = _inputs(w)
+    ctx, bufs = _run_gpu(w, wts, us, tensor_path)
+    pool = _check_layers(w, wts, us, bufs)
+    _check_tree(w, pool, bufs, 5)
+
+
+def test_expand_f32_ragged_and_flags():
+    w = synth.scaled(synth.WORKLOADS["tiny"], name="ragged32", batch=2, vocab=4100, inter=520,
+                     hidden=136, n_experts=5, k_per_expert=4, width=6, tree_size=25, depth=3,
+                     seed=78)
+    wts, us = _inputs(w)
+    ctx, bufs = _run_gpu(w, wts, us)
+    pool = _check_layers(w, wts, us, bufs)
+    _check_tree(w, pool, bufs, 5)
+
+
+def test_expand_is_deterministic():
+    w = synth.WORKLOADS["tiny_bf16"]
+    wts, us = _inputs(w)
+    _, a = _run_gpu(w, wts, us)
+    _, b = _run_gpu(w, wts, us)
+    assert torch.equal(a.logits, b.logits)
+    for k in a.pool:
+        assert torch.equal(a.pool[k], b.pool[k])
+
+
+def test_expand_llama2_7b_shape_sampled_rows():
+    """Full-size shapes of the benchmark configuration, launch configuration as benchmarked;
+    the oracle recomputes two frontier rows of layer 2 and the root row of layer 1."""
+    w = synth.WORKLOADS["llama2_7b"]
+    wts = synth.draft_weights(w)
+    fs = w.frontier_sizes[:2]
+    us = [synth.layer_hidden(w, l, F) for l, F in enumerate(fs)]
+    w2 = synth.scaled(w, depth=2, tree_size=30)
+    ctx, bufs = _run_gpu(w2, wts, us)
+    tol = TOL[w.dtype]
+    head64 = wts["lm_head"].astype(np.float64)
+    slot_base = 0
+    for l, F in enumerate(fs):
+        rows = [0] if F == 1 else [3, 8]
+        u = us[l].astype(np.float64)
+        probs_g = host(bufs.probs[l])
+        for f in rows:
+            x = orc.rmsnorm(u[0, f], wts["norm_weight"], 1e-5)
+            probs_o = orc.router_scores(x, wts["router"])
+            assert rel_err(probs_g[0, f], probs_o) <= tol
+            ids, _ = orc.topk_gate(probs_g[0, f], w.top_k)
+            assert host(bufs.expert[l])[0, f].tolist() == ids.tolist()
+            _, br, ff = orc.moe_features(u[0, f], x, ids, probs_o[ids], wts)
+            assert rel_err(host(bufs.feat[l])[0, f], ff) <= tol
+            lg_o = br @ head64.T
+            lg_g = host(bufs.logits)[0, slot_base + f]
+            assert rel_err(lg_g, lg_o) <= tol
+            for r in range(w.top_k):
+                ids_t, sc_t, _ = orc.branch_topk(lg_g[r], w.k_per_expert,
+                                                 float(host(bufs.parent_score[l])[0, f]))
+                g0 = (0 if l == 0 else fs[0] * w.top_k * w.k_per_expert) + \
+                    (f * w.top_k + r) * w.k_per_expert
+                assert host(bufs.pool["tok"])[0, g0:g0 + w.k_per_expert].tolist() == ids_t.tolist()
+        slot_base += F
