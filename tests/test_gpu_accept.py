@@ -88,6 +88,8 @@ def _check_compaction(w, caches, kv_len, paths, got_k, got_v):
 @pytest.mark.parametrize("kind", ["random", "chain", "star"])
 def test_greedy_accept_and_compaction(dtype, alpha, kind):
     w = synth.scaled(synth.WORKLOADS["tiny"], batch=3, vocab=4100 if dtype == "f32" else 4096)
+    if kind == "chain":
+        w = synth.scaled(w, depth=w.tree_size - 1)      # a chain is as deep as it is long
     tree, n_slots = _tree_arrays(w, kind, 11)
     tl = synth.target_logits(w, tree["tok"], tree["parent"], alpha)
     caches = _caches(w, 2, dtype, 500)
@@ -103,7 +105,7 @@ def test_greedy_accept_and_compaction(dtype, alpha, kind):
         assert np.all(acc_idx[b, len(path):] == -1)
         assert kvl[b] == kv_len[b] + 1 + len(path)
     if alpha == 1.0 and kind == "chain":
-        assert all(len(p) == w.depth for p in paths) or w.tree_size - 1 < w.depth
+        assert all(len(p) == w.tree_size - 1 for p in paths)
     _check_compaction(w, caches, kv_len, paths, gk, gv)
 
 
@@ -132,6 +134,8 @@ def _near_tie(trace, ua):
                                               ("random", 1.0, 1.0)])
 def test_sampling_accept(kind, alpha, agree):
     w = synth.scaled(synth.WORKLOADS["tiny"], batch=4, vocab=2000, seed=1234)
+    if kind == "chain":
+        w = synth.scaled(w, depth=w.tree_size - 1)
     tree, n_slots = _tree_arrays(w, kind, 21)
     tl = synth.target_logits(w, tree["tok"], tree["parent"], alpha, boost=6.0)
     rng = np.random.default_rng(5)
