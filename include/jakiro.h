@@ -87,6 +87,17 @@ int jk_read_status(jk_ctx* ctx, void* stream, int32_t* host_status);
  * (tcgen05) kernels where the dtype allows.  Default 1 for bf16, always 0 for f32. */
 int jk_set_tensor_path(jk_ctx* ctx, int32_t enable);
 
+/* Diagnostics (the paper has no counterpart): with max_launches > 0 every kernel launch of this
+ * context is bracketed by a pair of CUDA events on its stream (up to max_launches launches
+ * between two collects); 0 switches it off.  jk_profile_collect synchronises `stream`, writes
+ * the summed milliseconds and the launch count of every stage to the two host arrays of
+ * jk_profile_stage_count() entries and starts over.  Event handles are host resources; no
+ * device memory is allocated. */
+int jk_profile_enable(jk_ctx* ctx, int32_t max_launches);
+int jk_profile_collect(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count);
+int32_t jk_profile_stage_count(void);
+const char* jk_profile_stage_name(int32_t stage);
+
 /* Draft weights (Sec. 3.1.1-3.1.2): device pointers, read-only, output-major. */
 typedef struct {
   const void* router;       /* T [N, H]     expert centroids e_j (Eq. 2)                 */

@@ -23,7 +23,9 @@ ERR = {"NULL": -1, "SHAPE": -2, "ALIGN": -3, "DTYPE": -4, "CAPACITY": -5, "WORKS
 
 EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", "jk_strerror",
            "jk_last_cuda_error", "jk_read_status", "jk_set_tensor_path", "jk_draft_expand",
-           "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact"]
+           "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
+           "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
+           "jk_profile_stage_name"]
 
 
 class JkConfig(C.Structure):
@@ -77,8 +79,14 @@ def lib() -> C.CDLL:
         L.jk_accept_and_compact.argtypes = [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, vp, vp,
                                             vp, vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp,
                                             vp, vp, vp, vp]
+        L.jk_profile_enable.argtypes = [vp, i32]
+        L.jk_profile_collect.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
+        L.jk_profile_stage_count.argtypes = []
+        L.jk_profile_stage_name.argtypes = [i32]
+        L.jk_profile_stage_name.restype = C.c_char_p
         for name in EXPORTS:
-            if name not in ("jk_workspace_bytes", "jk_strerror", "jk_last_cuda_error"):
+            if name not in ("jk_workspace_bytes", "jk_strerror", "jk_last_cuda_error",
+                            "jk_profile_stage_name"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -164,6 +172,18 @@ class Context:
         out = C.c_int32(0)
         self._check(lib().jk_read_status(self._h, _stream(), C.byref(out)), "jk_read_status")
         return out.value
+
+    def profile_enable(self, max_launches: int):
+        self._check(lib().jk_profile_enable(self._h, max_launches), "jk_profile_enable")
+
+    def profile_collect(self) -> Dict[str, tuple]:
+        """{stage name: (total ms, launches)} since the last collect; synchronises."""
+        n = lib().jk_profile_stage_count()
+        ms = (C.c_float * n)()
+        cnt = (C.c_int32 * n)()
+        self._check(lib().jk_profile_collect(self._h, _stream(), ms, cnt), "jk_profile_collect")
+        return {lib().jk_profile_stage_name(i).decode(): (float(ms[i]), int(cnt[i]))
+                for i in range(n) if cnt[i]}
 
     # ------------------------------------------------------------------ calls
     @staticmethod

@@ -343,6 +343,7 @@ extern "C" int jk_accept_and_compact(
   int32_t* status = (int32_t*)(ws + L.status);
   const float inv_t = mode == 1 ? 1.f / temperature : 1.f;
   const int rows = batch * tree_size;
+  JK_PROF(ctx, st, JK_ST_ROWSTATS);
   if (tl_dtype == JK_BF16)
     k_row_stats<__nv_bfloat16><<<rows, 512, 0, st>>>((const __nv_bfloat16*)target_logits, c.vocab,
                                                      inv_t, rs_arg, rs_max, rs_sum);
@@ -351,6 +352,7 @@ extern "C" int jk_accept_and_compact(
                                              rs_max, rs_sum);
   JK_LAUNCH_CHECK(ctx);
   walk_out o{kv_len, (int32_t*)(ws + L.p_old), n_acc, acc_idx, acc_tok, bonus_tok};
+  JK_PROF(ctx, st, JK_ST_WALK);
   if (mode == 0) {
     k_walk_greedy<<<batch, 128, 0, st>>>(tree_size, c.max_depth, c.vocab, tok, parent, rs_arg, o,
                                          cache_rows, status);
@@ -362,6 +364,7 @@ extern "C" int jk_accept_and_compact(
   }
   JK_LAUNCH_CHECK(ctx);
   if (n_layers > 0) {
+    JK_PROF(ctx, st, JK_ST_COMPACT);
     k_compact<<<dim3(c.n_kv_heads, batch, 2 * n_layers), 256, 0, st>>>(
         k_caches, v_caches, n_layers, cache_stride_b, cache_stride_h, row_bytes, cache_rows,
         c.max_depth, tree_size, (const int32_t*)(ws + L.p_old), n_acc, acc_idx, es);

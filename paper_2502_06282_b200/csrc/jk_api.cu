@@ -6,6 +6,7 @@
 
 size_t jk_tc_partial_bytes(const jk_config& c);   // jk_gemm_tc.cu
 void jk_tc_destroy(jk_ctx* ctx);                  // jk_gemm_tc.cu
+static void prof_free(jk_ctx* ctx);
 
 static int validate_config(const jk_config& c) {
   if (c.dtype != JK_F32 && c.dtype != JK_BF16) return JK_ERR_DTYPE;
@@ -85,6 +86,7 @@ extern "C" int jk_create(jk_ctx** out, const jk_config* cfg) {
 extern "C" int jk_destroy(jk_ctx* ctx) {
   if (!ctx) return JK_ERR_NULL;
   jk_tc_destroy(ctx);
+  if (ctx->prof.cap) prof_free(ctx);
   free(ctx);
   return JK_OK;
 }
@@ -135,6 +137,69 @@ extern "C" int jk_read_status(jk_ctx* ctx, void* stream, int32_t* host_status) {
   JK_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 16, st));
   JK_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
   return JK_OK;
+}
+
+// ---------------------------------------------------------------- per-kernel timing
+void jk_prof_begin(jk_ctx* ctx, cudaStream_t st, int stage) {
+  jk_prof& p = ctx->prof;
+  if (p.n >= p.cap) return;
+  p.stage[p.n] = stage;
+  p.stream = st;
+  if (cudaEventRecord(p.ev[2 * p.n], st) == cudaSuccess) p.open = 1;
+}
+
+void jk_prof_end(jk_ctx* ctx) {
+  jk_prof& p = ctx->prof;
+  p.open = 0;
+  if (cudaEventRecord(p.ev[2 * p.n + 1], p.stream) == cudaSuccess) ++p.n;
+}
+
+static void prof_free(jk_ctx* ctx) {
+  jk_prof& p = ctx->prof;
+  for (int i = 0; i < 2 * p.cap; ++i) cudaEventDestroy(p.ev[i]);
+  free(p.ev);
+  free(p.stage);
+  memset(&p, 0, sizeof(p));
+}
+
+extern "C" int jk_profile_enable(jk_ctx* ctx, int32_t max_launches) {
+  if (!ctx) return JK_ERR_NULL;
+  if (max_launches < 0 || max_launches > (1 << 20)) return JK_ERR_SHAPE;
+  if (ctx->prof.cap) prof_free(ctx);
+  if (max_launches == 0) return JK_OK;
+  jk_prof& p = ctx->prof;
+  p.ev = (cudaEvent_t*)calloc(2 * (size_t)max_launches, sizeof(cudaEvent_t));
+  p.stage = (int*)calloc(max_launches, sizeof(int));
+  if (!p.ev || !p.stage) return JK_ERR_CUDA;
+  for (int i = 0; i < 2 * max_launches; ++i) JK_CUDA_CHECK(ctx, cudaEventCreate(&p.ev[i]));
+  p.cap = max_launches;
+  return JK_OK;
+}
+
+extern "C" int jk_profile_collect(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count) {
+  if (!ctx || !host_ms || !host_count) return JK_ERR_NULL;
+  for (int s = 0; s < JK_N_STAGES; ++s) { host_ms[s] = 0.f; host_count[s] = 0; }
+  jk_prof& p = ctx->prof;
+  if (!p.cap) return JK_OK;
+  JK_CUDA_CHECK(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+  for (int i = 0; i < p.n; ++i) {
+    float ms = 0.f;
+    JK_CUDA_CHECK(ctx, cudaEventElapsedTime(&ms, p.ev[2 * i], p.ev[2 * i + 1]));
+    host_ms[p.stage[i]] += ms;
+    host_count[p.stage[i]] += 1;
+  }
+  p.n = 0;
+  return JK_OK;
+}
+
+extern "C" int32_t jk_profile_stage_count(void) { return JK_N_STAGES; }
+
+extern "C" const char* jk_profile_stage_name(int32_t stage) {
+  static const char* names[JK_N_STAGES] = {
+      "router", "expert_gate_up", "expert_down", "branch_features", "lm_head", "topk_partial",
+      "expand_finish", "tree_finalize", "tree_attn", "attn_combine", "row_stats", "accept_walk",
+      "kv_compact", "gemm_fixup"};
+  return (stage >= 0 && stage < JK_N_STAGES) ? names[stage] : "?";
 }
 
 int jk_ensure_device_info(jk_ctx* ctx) {

@@ -196,12 +196,14 @@ static int attn_impl(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, 
   }
   float* part_o = (float*)(ctx->ws + L.attn_o);
   float* part_ml = (float*)(ctx->ws + L.attn_ml);
+  JK_PROF(ctx, st, JK_ST_ATTN);
   kern<<<dim3(n_split * n_qblk, c.n_kv_heads, B), 256, smem, st>>>(
       (const T*)q, (const T*)kc, (const T*)vc, sb, sh, cache_rows, kv_len, parent, scale, M,
       c.n_q_heads, c.n_kv_heads, n_split, n_qblk, part_o, part_ml,
       (int32_t*)(ctx->ws + L.status));
   JK_LAUNCH_CHECK(ctx);
   const size_t n_out = (size_t)B * M * c.n_q_heads;
+  JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
   k_attn_combine<T, D><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
                                                                     n_out, (T*)out);
   JK_LAUNCH_CHECK(ctx);

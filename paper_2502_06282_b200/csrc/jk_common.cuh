@@ -48,6 +48,19 @@ struct jk_ws_layout {
   size_t gemm_part_bytes;
 };
 
+// Optional per-kernel timing: a pair of CUDA events around every launch, summed per stage.
+enum jk_stage {
+  JK_ST_ROUTER = 0, JK_ST_GATEUP, JK_ST_DOWN, JK_ST_BRANCH, JK_ST_LMHEAD, JK_ST_TOPK,
+  JK_ST_FINISH, JK_ST_FINALIZE, JK_ST_ATTN, JK_ST_ATTN_COMBINE, JK_ST_ROWSTATS, JK_ST_WALK,
+  JK_ST_COMPACT, JK_ST_GEMM_FIXUP, JK_N_STAGES
+};
+struct jk_prof {
+  cudaEvent_t* ev;        // 2 * cap events
+  int* stage;             // stage of each recorded pair
+  int cap, n, open;
+  cudaStream_t stream;
+};
+
 struct jk_ctx {
   jk_config cfg;
   jk_ws_layout lay;
@@ -58,7 +71,15 @@ struct jk_ctx {
   int attn_smem_set;
   char cuda_err[256];
   void* tc_state;         // tensor-core path bookkeeping (tensor maps), host memory
+  jk_prof prof;
 };
+
+void jk_prof_begin(jk_ctx* ctx, cudaStream_t st, int stage);
+void jk_prof_end(jk_ctx* ctx);
+#define JK_PROF(ctx, st, stage)                                  \
+  do {                                                           \
+    if ((ctx)->prof.cap) jk_prof_begin(ctx, st, stage);          \
+  } while (0)
 
 static inline size_t jk_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int jk_elem_size(int dtype) { return dtype == JK_BF16 ? 2 : 4; }
@@ -75,6 +96,7 @@ static inline int jk_elem_size(int dtype) { return dtype == JK_BF16 ? 2 : 4; }
 
 #define JK_LAUNCH_CHECK(ctx)                                                         \
   do {                                                                               \
+    if ((ctx)->prof.open) jk_prof_end(ctx);                                          \
     cudaError_t e_ = cudaGetLastError();                                             \
     if (e_ != cudaSuccess) {                                                         \
       snprintf((ctx)->cuda_err, sizeof((ctx)->cuda_err), "launch at %s:%d: %s",      \

@@ -517,6 +517,7 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
   const int rows_per_b = F * K;
   const long long lsb = (out_logits && logits_stride_b) ? logits_stride_b : (long long)rows_per_b * V;
 
+  JK_PROF(ctx, st, JK_ST_ROUTER);
   k_router<T><<<R, 256, 0, st>>>((const T*)u, (const T*)w->router, (const T*)w->norm_weight, H,
                                  c.n_experts, K, c.rms_eps, c.use_pre_norm, xn, out_probs,
                                  out_expert, out_gate);
@@ -526,13 +527,16 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
     int rc = jk_tc_expert_ffn(ctx, st, w, R, out_expert, 0, nullptr, RK, rows_per_b, lsb);
     if (rc != JK_OK) return rc;
   } else {
+    JK_PROF(ctx, st, JK_ST_GATEUP);
     k_gateup<T><<<dim3((I + 31) / 32, c.n_experts), 256, 0, st>>>(
         (const T*)w->w_gate, (const T*)w->w_up, xn, out_expert, R, K, H, I, Rp, hbuf);
     JK_LAUNCH_CHECK(ctx);
+    JK_PROF(ctx, st, JK_ST_DOWN);
     k_down<T><<<dim3((H + 15) / 16, c.n_experts), 256, 0, st>>>(
         (const T*)w->w_down, hbuf, out_expert, R, K, H, I, Rp, ybuf);
     JK_LAUNCH_CHECK(ctx);
   }
+  JK_PROF(ctx, st, JK_ST_BRANCH);
   k_branch<T><<<R, 256, 0, st>>>((const T*)u, ybuf, out_expert, out_gate, K, H, Rp,
                                  c.branch_residual, bbuf, (T*)out_feat);
   JK_LAUNCH_CHECK(ctx);
@@ -540,14 +544,17 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
     int rc = jk_tc_expert_ffn(ctx, st, w, R, out_expert, 1, logits, RK, rows_per_b, lsb);
     if (rc != JK_OK) return rc;
   } else {
+    JK_PROF(ctx, st, JK_ST_LMHEAD);
     k_lmhead<T><<<(V + 31) / 32, 256, 0, st>>>((const T*)w->lm_head, bbuf, RK, H, V, logits,
                                                rows_per_b, lsb);
     JK_LAUNCH_CHECK(ctx);
   }
+  JK_PROF(ctx, st, JK_ST_TOPK);
   k_topk_partial<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
       logits, rows_per_b, lsb, V, c.k_per_expert, L.topk_chunks, (float*)(ws + L.tk_val),
       (int32_t*)(ws + L.tk_idx), (float*)(ws + L.tk_ms));
   JK_LAUNCH_CHECK(ctx);
+  JK_PROF(ctx, st, JK_ST_FINISH);
   k_expand_finish<<<B, 256, 0, st>>>(F, K, c.k_per_expert, L.topk_chunks, width,
                                      (const float*)(ws + L.tk_val),
                                      (const int32_t*)(ws + L.tk_idx),
@@ -616,7 +623,9 @@ extern "C" int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const 
   if (pool_n > JK_MAX_POOL || pool_n < tree_size - 1 || pool->stride_b < pool_n)
     return JK_ERR_SHAPE;
   if (!ctx->ws) return JK_ERR_WORKSPACE;
-  k_tree_finalize<<<batch, 1024, 0, (cudaStream_t)stream>>>(
+  cudaStream_t st = (cudaStream_t)stream;
+  JK_PROF(ctx, st, JK_ST_FINALIZE);
+  k_tree_finalize<<<batch, 1024, 0, st>>>(
       *pool, pool_n, root_tok, tree_size, tok, parent, depth, branch, qslot,
       (unsigned long long*)anc, (int32_t*)(ctx->ws + ctx->lay.status));
   JK_LAUNCH_CHECK(ctx);
