@@ -194,6 +194,38 @@ int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_s
                         void* out);
 
 /*
+ * jk_tree_verify_attn for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same arithmetic.)
+ *
+ * Meant for processes that have given all free HBM to their own pools at start-up, so that a
+ * later cudaMalloc for a workspace fails, and for decode loops that cannot afford the
+ * device-wide synchronisation of cudaMalloc/cudaFree.  It needs no jk_set_workspace: the split-KV
+ * partials go to a fixed 8 MiB (+256 B) array compiled into the library, which every GPU that
+ * loads the library holds until the process exits.  The call makes no cudaMalloc/cudaFree and
+ * uses no allocating library routine.
+ *
+ *   Arguments as jk_tree_verify_attn, plus
+ *   status   i32 [1] device, optional: receives JK_ERR_BOUNDS if kv_len[b] + M > cache_rows
+ *            (atomic compare-and-swap on 0, so the caller clears it); with NULL the error is
+ *            only recorded inside the built-in array, which the next call clears.
+ *   Limit    batch * tree_size * n_q_heads * (head_dim + 2) * 4 bytes <= 8 MiB (e.g. 60 nodes x
+ *            32 heads x 128 uses 1 MiB per key slice); beyond it the call returns
+ *            JK_ERR_CAPACITY, launches nothing, and jk_last_cuda_error(ctx) says why.
+ *   Set-up   the first call on each device (with that device current) looks up the array's
+ *            device address; make that first call before starting any stream capture.
+ *   Sharing  all contexts, streams and threads of the process share the one array per GPU, and
+ *            it keeps the previous call's contents.  Nothing in it has to start at zero except
+ *            the internal status word, which the call clears itself; but two of these calls
+ *            that overlap on the same GPU race on the partials and give wrong results: run
+ *            them one after the other.
+ */
+int jk_tree_verify_attn_static(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
+                               const void* q, const void* k_cache, const void* v_cache,
+                               int64_t cache_stride_b, int64_t cache_stride_h, int32_t cache_rows,
+                               const int32_t* kv_len, const int32_t* parent, float softmax_scale,
+                               void* out, int32_t* status);
+
+/*
  * Acceptance walk and KV compaction (Sec. 2.1 steps 2-3).
  *   mode 0 (greedy): from the root, follow the first child whose token equals the target's
  *     top-1 token (ties: lower id) at the current node; stop when none does; the bonus token

@@ -25,7 +25,7 @@ EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", 
            "jk_last_cuda_error", "jk_read_status", "jk_set_tensor_path", "jk_draft_expand",
            "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
            "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
-           "jk_profile_stage_name"]
+           "jk_profile_stage_name", "jk_tree_verify_attn_static"]
 
 
 class JkConfig(C.Structure):
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
                                        vp, vp, vp]
         L.jk_tree_verify_attn.argtypes = [vp, vp, i32, i32, vp, vp, vp, i64, i64, i32, vp, vp,
                                           f32, vp]
+        L.jk_tree_verify_attn_static.argtypes = L.jk_tree_verify_attn.argtypes + [vp]
         L.jk_accept_and_compact.argtypes = [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, vp, vp,
                                             vp, vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp,
                                             vp, vp, vp, vp]
@@ -226,6 +227,20 @@ class Context:
                                        k_cache.stride(1), rows, _ptr(kv_len), _ptr(parent),
                                        float(scale), _ptr(out))
         self._check(rc, "jk_tree_verify_attn")
+
+    def tree_verify_attn_static(self, batch, tree_size, q, k_cache, v_cache, kv_len, parent,
+                                scale, out, status=None, cache_rows=None):
+        """jk_tree_verify_attn_static: the same attention without any workspace, for callers
+        that cannot allocate device memory; scratch is the library's built-in 8 MiB array."""
+        rows = k_cache.shape[2] if cache_rows is None else cache_rows
+        rc = lib().jk_tree_verify_attn_static(self._h, _stream(), batch, tree_size, _ptr(q),
+                                              _ptr(k_cache), _ptr(v_cache), k_cache.stride(0),
+                                              k_cache.stride(1), rows, _ptr(kv_len),
+                                              _ptr(parent), float(scale), _ptr(out),
+                                              _ptr(status))
+        if rc != JK_OK:
+            detail = lib().jk_last_cuda_error(self._h).decode()
+            raise JakiroError(rc, "jk_tree_verify_attn_static", detail)
 
     def accept_and_compact(self, batch, tree_size, mode, temperature, target_logits, tree,
                            draft_logits, n_slots, u_accept, u_bonus, n_layers, k_ptrs, v_ptrs,

@@ -239,3 +239,113 @@ extern "C" int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int
   JK_ATTN_CASE(float, 64);
 #undef JK_ATTN_CASE
 }
+
+// ------------------------------------------------------------------------------------------
+// jk_tree_verify_attn_static: the same attention for callers that cannot allocate.
+//
+// Who they are: a serving process that handed every free byte of HBM to its KV-cache pool at
+// start-up (a cudaMalloc for a workspace then simply fails), and a decode loop that must not
+// stall, since cudaMalloc and cudaFree synchronise the whole device.  Such a caller cannot give
+// this library the workspace that jk_set_workspace wants, so here the split-KV partials live in
+// an array that is part of the library image itself.  Cost: every GPU that loads the library
+// carries these JK_ATTN_STATIC_BYTES (+256) until the process exits, used or not.
+//
+// The array's name is only a handle in host code, not a device address; the address the kernels
+// need comes from cudaGetSymbolAddress, asked once per device with that device current.
+// ------------------------------------------------------------------------------------------
+#define JK_ATTN_STATIC_BYTES (8u << 20)
+#define JK_ATTN_STATIC_MAX_DEVICES 64
+static __device__ __align__(256) unsigned char g_attn_static_scratch[JK_ATTN_STATIC_BYTES + 256];
+static void* g_attn_static_ptr[JK_ATTN_STATIC_MAX_DEVICES];   // device address, per device
+
+template <typename T, int D>
+static int attn_static_impl(jk_ctx* ctx, cudaStream_t st, unsigned char* scratch, int B, int M,
+                            const void* q, const void* kc, const void* vc, int64_t sb, int64_t sh,
+                            int cache_rows, const int32_t* kv_len, const int32_t* parent,
+                            float scale, void* out, int32_t* status) {
+  const jk_config& c = ctx->cfg;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int n_qblk = (G * M + JK_ATTN_QB - 1) / JK_ATTN_QB;
+  const int base_ctas = n_qblk * c.n_kv_heads * B;
+  const size_t n_out = (size_t)B * M * c.n_q_heads;
+  const size_t per_split = n_out * (D + 2) * sizeof(float);
+  if (per_split > JK_ATTN_STATIC_BYTES) {
+    snprintf(ctx->cuda_err, sizeof(ctx->cuda_err),
+             "jk_tree_verify_attn_static: B*M*Hq*(d+2)*4 = %zu bytes exceeds the %u-byte scratch",
+             per_split, JK_ATTN_STATIC_BYTES);
+    return JK_ERR_CAPACITY;
+  }
+  int n_split = (2 * ctx->sm_count + base_ctas - 1) / base_ctas;
+  const int max_by_len = (cache_rows / 64) > 0 ? (cache_rows / 64) : 1;
+  const int max_by_mem = (int)(JK_ATTN_STATIC_BYTES / per_split);
+  if (n_split > max_by_len) n_split = max_by_len;
+  if (n_split > max_by_mem) n_split = max_by_mem;
+  if (n_split > JK_ATTN_MAX_SPLIT) n_split = JK_ATTN_MAX_SPLIT;
+  if (n_split < 1) n_split = 1;
+  // first 256 bytes: a status word for callers that pass none; it must start at zero
+  int32_t* status_word = status ? status : reinterpret_cast<int32_t*>(scratch);
+  if (!status) JK_CUDA_CHECK(ctx, cudaMemsetAsync(scratch, 0, 16, st));
+  float* part_o = reinterpret_cast<float*>(scratch + 256);
+  float* part_ml = part_o + (size_t)n_split * n_out * D;
+  const size_t smem = sizeof(attn_smem<D>);
+  auto kern = k_tree_attn<T, D>;
+  JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)smem));
+  kern<<<dim3(n_split * n_qblk, c.n_kv_heads, B), 256, smem, st>>>(
+      (const T*)q, (const T*)kc, (const T*)vc, sb, sh, cache_rows, kv_len, parent, scale, M,
+      c.n_q_heads, c.n_kv_heads, n_split, n_qblk, part_o, part_ml, status_word);
+  JK_LAUNCH_CHECK(ctx);
+  k_attn_combine<T, D><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
+                                                                    n_out, (T*)out);
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
+
+extern "C" int jk_tree_verify_attn_static(jk_ctx* ctx, void* stream, int32_t batch,
+                                          int32_t tree_size, const void* q, const void* k_cache,
+                                          const void* v_cache, int64_t cache_stride_b,
+                                          int64_t cache_stride_h, int32_t cache_rows,
+                                          const int32_t* kv_len, const int32_t* parent,
+                                          float softmax_scale, void* out, int32_t* status) {
+  if (!ctx || !q || !k_cache || !v_cache || !kv_len || !parent || !out) return JK_ERR_NULL;
+  const jk_config& c = ctx->cfg;
+  if (batch < 1 || tree_size < 1 || cache_rows < tree_size) return JK_ERR_SHAPE;
+  if (batch > c.max_batch || tree_size > c.max_tree) return JK_ERR_CAPACITY;
+  if (cache_stride_h < (int64_t)cache_rows * c.head_dim) return JK_ERR_SHAPE;
+  if (!jk_aligned16(q) || !jk_aligned16(k_cache) || !jk_aligned16(v_cache) || !jk_aligned16(out))
+    return JK_ERR_ALIGN;
+  const int es = jk_elem_size(c.dtype);
+  if ((cache_stride_b * es) % 16 || (cache_stride_h * es) % 16) return JK_ERR_ALIGN;
+  if ((size_t)batch * tree_size * c.n_q_heads * (c.head_dim + 2) * sizeof(float) >
+      JK_ATTN_STATIC_BYTES) {
+    snprintf(ctx->cuda_err, sizeof(ctx->cuda_err),
+             "jk_tree_verify_attn_static: batch*tree_size*n_q_heads*(head_dim+2)*4 exceeds the "
+             "%u-byte built-in scratch", JK_ATTN_STATIC_BYTES);
+    return JK_ERR_CAPACITY;
+  }
+  int rc = jk_ensure_device_info(ctx);
+  if (rc != JK_OK) return rc;
+  // once per device: turn the symbol into the device address the kernels can use
+  int dev = -1;
+  JK_CUDA_CHECK(ctx, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= JK_ATTN_STATIC_MAX_DEVICES) return JK_ERR_SHAPE;
+  if (!g_attn_static_ptr[dev]) {
+    void* p = nullptr;
+    JK_CUDA_CHECK(ctx, cudaGetSymbolAddress(&p, g_attn_static_scratch));
+    if (!p) return JK_ERR_CUDA;
+    g_attn_static_ptr[dev] = p;
+  }
+  unsigned char* scratch = static_cast<unsigned char*>(g_attn_static_ptr[dev]);
+  cudaStream_t st = (cudaStream_t)stream;
+#define JK_ATTN_STATIC_CASE(T, D)                                                             \
+  return attn_static_impl<T, D>(ctx, st, scratch, batch, tree_size, q, k_cache, v_cache,      \
+                                cache_stride_b, cache_stride_h, cache_rows, kv_len, parent,   \
+                                softmax_scale, out, status)
+  if (c.dtype == JK_BF16) {
+    if (c.head_dim == 128) JK_ATTN_STATIC_CASE(__nv_bfloat16, 128);
+    JK_ATTN_STATIC_CASE(__nv_bfloat16, 64);
+  }
+  if (c.head_dim == 128) JK_ATTN_STATIC_CASE(float, 128);
+  JK_ATTN_STATIC_CASE(float, 64);
+#undef JK_ATTN_STATIC_CASE
+}
