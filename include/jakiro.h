@@ -86,6 +86,9 @@ int jk_read_status(jk_ctx* ctx, void* stream, int32_t* host_status);
 /* Which kernels run the dense contractions: 0 = CUDA-core kernels, 1 = tensor-core
  * (tcgen05) kernels where the dtype allows.  Default 1 for bf16, always 0 for f32. */
 int jk_set_tensor_path(jk_ctx* ctx, int32_t enable);
+/* 1 if the tensor-core kernels will run the contractions of this context (bf16, enabled, rows
+ * within their limit, driver entry point for tensor maps found), else 0. */
+int jk_tensor_path_active(jk_ctx* ctx);
 
 /* Diagnostics (the paper has no counterpart): with max_launches > 0 every kernel launch of this
  * context is bracketed by a pair of CUDA events on its stream (up to max_launches launches

@@ -25,7 +25,7 @@ EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", 
            "jk_last_cuda_error", "jk_read_status", "jk_set_tensor_path", "jk_draft_expand",
            "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
            "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
-           "jk_profile_stage_name", "jk_tree_verify_attn_static"]
+           "jk_profile_stage_name", "jk_tree_verify_attn_static", "jk_tensor_path_active"]
 
 
 class JkConfig(C.Structure):
@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
         L.jk_last_cuda_error.restype = C.c_char_p
         L.jk_read_status.argtypes = [vp, vp, C.POINTER(i32)]
         L.jk_set_tensor_path.argtypes = [vp, i32]
+        L.jk_tensor_path_active.argtypes = [vp]
         L.jk_draft_expand.argtypes = [vp, vp, C.POINTER(JkDraftWeights), i32, i32, i32, vp, vp,
                                       vp, i32, i32, vp, vp, vp, C.POINTER(JkPool), vp, vp, vp,
                                       i64, vp, vp, vp]
@@ -168,6 +169,10 @@ class Context:
 
     def set_tensor_path(self, enable: bool):
         self._check(lib().jk_set_tensor_path(self._h, int(enable)), "jk_set_tensor_path")
+
+    @property
+    def tensor_path_active(self) -> bool:
+        return bool(lib().jk_tensor_path_active(self._h))
 
     def read_status(self) -> int:
         out = C.c_int32(0)

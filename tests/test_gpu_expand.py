@@ -20,6 +20,7 @@ def _run_gpu(w, wts_np, us_np, tensor_path=None, root_tok=5):
     ctx = jk.Context.for_workload(w)
     if tensor_path is not None:
         ctx.set_tensor_path(tensor_path)
+        assert ctx.tensor_path_active == bool(tensor_path)
     bufs = jk.StepBuffers(ctx, w)
     wts = weights_to_device(wts_np, w.dtype)
     us = [dev(u, w.dtype) for u in us_np]
