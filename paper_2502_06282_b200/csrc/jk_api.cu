@@ -7,6 +7,7 @@
 size_t jk_tc_partial_bytes(const jk_config& c);   // jk_gemm_tc.cu
 void jk_tc_destroy(jk_ctx* ctx);                  // jk_gemm_tc.cu
 static void prof_free(jk_ctx* ctx);
+void jk_attn_tc_destroy(jk_ctx* ctx);             // jk_attn_tc.cu
 
 static int validate_config(const jk_config& c) {
   if (c.dtype != JK_F32 && c.dtype != JK_BF16) return JK_ERR_DTYPE;
@@ -86,6 +87,7 @@ extern "C" int jk_create(jk_ctx** out, const jk_config* cfg) {
 extern "C" int jk_destroy(jk_ctx* ctx) {
   if (!ctx) return JK_ERR_NULL;
   jk_tc_destroy(ctx);
+  jk_attn_tc_destroy(ctx);
   if (ctx->prof.cap) prof_free(ctx);
   free(ctx);
   return JK_OK;

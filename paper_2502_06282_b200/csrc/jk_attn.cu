@@ -210,6 +210,28 @@ static int attn_impl(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, 
   return JK_OK;
 }
 
+// tensor-core kernel (jk_attn_tc.cu)
+int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
+               const void* vc, int64_t sb, int64_t sh, int cache_rows, const int32_t* kv_len,
+               const int32_t* parent, float scale, void* out);
+int jk_tc_available(const jk_ctx* ctx);
+
+// Merge launch shared with the tensor-core kernel (bf16 output).
+int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_out, void* out) {
+  const jk_ws_layout& L = ctx->lay;
+  const float* part_o = (const float*)(ctx->ws + L.attn_o);
+  const float* part_ml = (const float*)(ctx->ws + L.attn_ml);
+  JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
+  if (ctx->cfg.head_dim == 128)
+    k_attn_combine<__nv_bfloat16, 128><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(
+        part_o, part_ml, n_split, n_out, (__nv_bfloat16*)out);
+  else
+    k_attn_combine<__nv_bfloat16, 64><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(
+        part_o, part_ml, n_split, n_out, (__nv_bfloat16*)out);
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
+
 extern "C" int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
                                    const void* q, const void* k_cache, const void* v_cache,
                                    int64_t cache_stride_b, int64_t cache_stride_h,
@@ -228,7 +250,10 @@ extern "C" int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int
   int rc = jk_ensure_device_info(ctx);
   if (rc != JK_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-#define JK_ATTN_CASE(T, D)                                                                  \
+  if (c.dtype == JK_BF16 && ctx->tensor_path && softmax_scale > 0.f && jk_tc_available(ctx))
+    return jk_attn_tc(ctx, st, batch, tree_size, q, k_cache, v_cache, cache_stride_b,
+                      cache_stride_h, cache_rows, kv_len, parent, softmax_scale, out);
+#define JK_ATTN_CASE(T, D)                                                                \
   return attn_impl<T, D>(ctx, st, batch, tree_size, q, k_cache, v_cache, cache_stride_b,    \
                          cache_stride_h, cache_rows, kv_len, parent, softmax_scale, out)
   if (c.dtype == JK_BF16) {

@@ -1,0 +1,374 @@
+// Tensor-core (tcgen05) kernel of jk_tree_verify_attn for bf16 (arXiv 2502.06282, Sec. 2.1 step 2,
+// mask of Fig. 4).
+//
+// One CTA = (sequence, kv head, block of 128 query rows, slice of the key range).  Query rows are
+// (q head of the group, tree node) pairs, so for GQA the heads that share a kv head share its K/V
+// tiles.  Per tile of 128 keys:
+//   TMA brings K [128 keys x d] and V [128 keys x d] into swizzled shared memory;
+//   S = Q K^T on the tensor core into tensor memory (128 x 128 fp32);
+//   every thread owns one query row: it reads its row of S, applies the tree mask (a 128-bit
+//   visibility word built from the node's ancestor set and the prefix length), keeps a running
+//   max and sum, and writes P = exp(S - max) as bf16 into the shared memory K just left;
+//   O (+)= P V on the tensor core, V taken MN-major straight from its row-major tile; when the
+//   running max moved, O is first rescaled in tensor memory.
+// The CTA writes an unnormalised partial (max, sum, O) per row; the merge kernel of jk_attn.cu
+// combines the slices.  96 KB of shared memory and 256 tensor-memory columns per CTA, so two CTAs
+// share an SM and overlap each other's copy and math phases.  All mbarrier waits are bounded.
+#include <math.h>
+#include <stdlib.h>
+
+#include "jk_common.cuh"
+#include "jk_tcgen05.cuh"
+
+#define ATC_ROWS 128
+#define ATC_KEYS 128
+
+struct atc_tail {
+  uint64_t bar_k, bar_v, bar_s, bar_o;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128) k_tree_attn_tc(
+    const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+    const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ kv_len,
+    const int32_t* __restrict__ parent, float scale, int M, int Hq, int Hkv, int n_split,
+    int cache_rows, float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status) {
+  constexpr int KB = D / 64;                       // 64-element blocks along d
+  constexpr int Q_BYTES = ATC_ROWS * D * 2;
+  constexpr int KP_BYTES = 2 * ATC_ROWS * 64 * 2;  // K tile (KB blocks) or P tile (2 blocks)
+  constexpr int V_BYTES = ATC_KEYS * D * 2;
+  constexpr uint32_t TMEM_COLS = 256;
+  constexpr uint32_t O_COL = 128;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* sq = smem;
+  unsigned char* skp = smem + Q_BYTES;
+  unsigned char* sv = skp + KP_BYTES;
+  atc_tail& T = *reinterpret_cast<atc_tail*>(sv + V_BYTES);
+  volatile int* abort_flag = &T.abort_flag;
+
+  const int split = blockIdx.x % n_split, qblk = blockIdx.x / n_split;
+  const int kvh = blockIdx.y, b = blockIdx.z;
+  const int G = Hq / Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int P = kv_len[b];
+  const int Ltot = P + M;
+  if (P < 0 || Ltot > cache_rows) {
+    if (tid == 0) jk_set_status(status, JK_ERR_BOUNDS);
+    return;
+  }
+  const int n_rows = G * M;
+  const int row0 = qblk * ATC_ROWS;
+  const bool row_valid = row0 + tid < n_rows;
+  const int g_idx = row_valid ? (row0 + tid) / M : 0;
+  const int node = row_valid ? (row0 + tid) % M : 0;
+  const size_t n_out = (size_t)gridDim.z * M * Hq;
+  const size_t orow = ((size_t)b * M + node) * Hq + kvh * G + g_idx;
+  const int tiles_total = (Ltot + ATC_KEYS - 1) / ATC_KEYS;
+  const int tiles_per = (tiles_total + n_split - 1) / n_split;
+  const int t0 = split * tiles_per;
+  const int t1 = min(tiles_total, t0 + tiles_per);
+  if (t0 >= t1) {                                  // no keys in this slice
+    if (row_valid) {
+      part_ml[((size_t)split * n_out + orow) * 2] = -INFINITY;
+      part_ml[((size_t)split * n_out + orow) * 2 + 1] = 0.f;
+    }
+    return;
+  }
+
+  auto issue_kv = [&](int tile) {
+    mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb)
+      tma_load_4d(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k);
+    mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb)
+      tma_load_4d(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v);
+  };
+
+  if (tid == 0) {
+    mbar_init(&T.bar_k, 1); mbar_init(&T.bar_v, 1); mbar_init(&T.bar_s, 1); mbar_init(&T.bar_o, 1);
+    T.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    issue_kv(t0);
+  }
+  if (warp == 0) {
+    tmem_alloc(&T.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  // Q block -> shared memory in the K-major 128-byte-swizzled layout the MMA reads
+  for (int idx = tid; idx < ATC_ROWS * (D / 8); idx += 128) {
+    const int rr = idx / (D / 8), ch = idx % (D / 8);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row0 + rr < n_rows) {
+      const int gg = (row0 + rr) / M, ii = (row0 + rr) % M;
+      v = *reinterpret_cast<const uint4*>(q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8);
+    }
+    const int kb = ch >> 3, cb = ch & 7;
+    *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = v;
+  }
+  // ancestor set of this thread's node (Fig. 4)
+  unsigned long long anc_lo = 0ull, anc_hi = 0ull;
+  if (row_valid) {
+    int c = node;
+    for (int guard = 0; c >= 0 && guard <= JK_MAX_TREE; ++guard) {
+      if (c < 64) anc_lo |= 1ull << c; else anc_hi |= 1ull << (c - 64);
+      const int pp = parent[(size_t)b * M + c];
+      c = (pp < c) ? pp : -1;
+    }
+  }
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = T.tmem_base;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  const uint32_t idesc_s = instr_desc_bf16_ex(ATC_KEYS, 0);
+  const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
+  const float sl2 = scale * 1.4426950408889634f;
+
+  float m_run = -INFINITY, l_run = 0.f;
+  bool ok = true;
+  for (int tile = t0; tile < t1; ++tile) {
+    const uint32_t ph = (uint32_t)(tile - t0) & 1u;
+    if (tid == 0) {
+      ok = mbar_wait(&T.bar_k, ph, abort_flag, status);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t qa = smem_u32(sq), ka = smem_u32(skp);
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            tc_mma_bf16(tmem_base, smem_desc_sw128(qa + kb * 16384 + k * 32),
+                        smem_desc_sw128(ka + kb * 16384 + k * 32), idesc_s, (kb | k) ? 1u : 0u);
+        tc_commit(&T.bar_s);
+      }
+    }
+    ok = ok && mbar_wait(&T.bar_s, ph, abort_flag, status);
+    if (!__syncthreads_and(ok)) { ok = false; break; }
+    tc_fence_after();
+
+    // visibility of keys key0 .. key0+127 for this row: prefix keys, then the ancestor set
+    unsigned long long vis_lo = 0ull, vis_hi = 0ull;
+    if (row_valid) {
+      const int s = P - tile * ATC_KEYS;
+      if (s >= 128) { vis_lo = ~0ull; vis_hi = ~0ull; }
+      else if (s >= 0) {
+        if (s >= 64) { vis_lo = ~0ull; vis_hi = (s == 64) ? 0ull : ((1ull << (s - 64)) - 1ull); }
+        else { vis_lo = (s == 0) ? 0ull : ((1ull << s) - 1ull); }
+        unsigned long long a_lo, a_hi;
+        if (s == 0) { a_lo = anc_lo; a_hi = anc_hi; }
+        else if (s < 64) { a_lo = anc_lo << s; a_hi = (anc_hi << s) | (anc_lo >> (64 - s)); }
+        else if (s == 64) { a_lo = 0ull; a_hi = anc_lo; }
+        else { a_lo = 0ull; a_hi = anc_lo << (s - 64); }
+        vis_lo |= a_lo; vis_hi |= a_hi;
+      } else {
+        const int t = -s;
+        if (t < 64) { vis_lo = (anc_lo >> t) | (anc_hi << (64 - t)); vis_hi = anc_hi >> t; }
+        else if (t < 128) { vis_lo = anc_hi >> (t - 64); vis_hi = 0ull; }
+      }
+    }
+    // pass 1: row maximum over the visible keys
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(tmem_base + lane_base + (uint32_t)(c * 32), r);
+      tmem_ld_wait();
+      const unsigned bits = (unsigned)(((c < 2) ? vis_lo : vis_hi) >> ((c & 1) * 32));
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if ((bits >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r[j]));
+    }
+    const float m_new = fmaxf(m_run, mx);
+    const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
+                                             : fast_exp2((m_run - m_new) * sl2);
+    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+    // pass 2: P = exp(S - max) as bf16 into the K buffer, row sum
+    float lsum = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(tmem_base + lane_base + (uint32_t)(c * 32), r);
+      tmem_ld_wait();
+      const unsigned bits = (unsigned)(((c < 2) ? vis_lo : vis_hi) >> ((c & 1) * 32));
+      uint32_t packed[16];
+#pragma unroll
+      for (int j = 0; j < 32; j += 2) {
+        const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(r[j]) - m_use) * sl2) : 0.f;
+        const float p1 = ((bits >> (j + 1)) & 1u)
+                             ? fast_exp2((__uint_as_float(r[j + 1]) - m_use) * sl2) : 0.f;
+        lsum += p0 + p1;
+        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+        packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const int ch = c * 4 + jj;               // 16-byte chunk of the 128-key row
+        const int kb = ch >> 3, cb = ch & 7;
+        *reinterpret_cast<uint4*>(skp + kb * 16384 + tid * 128 + ((cb ^ (tid & 7)) << 4)) =
+            make_uint4(packed[4 * jj], packed[4 * jj + 1], packed[4 * jj + 2], packed[4 * jj + 3]);
+      }
+    }
+    l_run = l_run * alpha + lsum;
+    m_run = m_new;
+    // rescale the running output when some row of this warp moved its maximum
+    if (tile > t0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+        tmem_st32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+      }
+      tmem_st_wait();
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      ok = mbar_wait(&T.bar_v, ph, abort_flag, status);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t pa = smem_u32(skp), va = smem_u32(sv);
+#pragma unroll
+        for (int j = 0; j < ATC_KEYS / 16; ++j)
+          tc_mma_bf16(tmem_base + O_COL, smem_desc_sw128(pa + (j >> 2) * 16384 + (j & 3) * 32),
+                      smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
+                      (tile > t0 || j > 0) ? 1u : 0u);
+        tc_commit(&T.bar_o);
+      }
+    }
+    ok = ok && mbar_wait(&T.bar_o, ph, abort_flag, status);
+    if (!__syncthreads_and(ok)) { ok = false; break; }
+    tc_fence_after();
+    if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
+  }
+  if (ok) {
+    float* po = part_o + ((size_t)split * n_out + orow) * D;
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+      tmem_ld_wait();
+      if (row_valid) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4)
+          *reinterpret_cast<float4*>(po + c * 32 + j) =
+              make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                          __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+      }
+    }
+    if (row_valid) {
+      part_ml[((size_t)split * n_out + orow) * 2] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
+      part_ml[((size_t)split * n_out + orow) * 2 + 1] = l_run;
+    }
+  } else if (tid == 0) {
+    // gave up, possibly with copies still in flight: give them a bounded time to land
+    const unsigned long long ts = global_ns();
+    while (global_ns() - ts < 2000000ull) { /* 2 ms: far longer than any TMA copy */ }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// jk_attn.cu
+int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_out, void* out);
+
+struct atc_map_entry {
+  const void* ptr;
+  int64_t sb, sh;
+  int rows;
+  CUtensorMap map;
+};
+struct atc_state {
+  atc_map_entry e[256];
+  int n, next;
+  int smem_set;
+};
+
+static const CUtensorMap* atc_map(jk_ctx* ctx, atc_state* s, const void* ptr, int64_t sb, int64_t sh,
+                                  int rows, int B) {
+  for (int i = 0; i < s->n; ++i)
+    if (s->e[i].ptr == ptr && s->e[i].sb == sb && s->e[i].sh == sh && s->e[i].rows == rows)
+      return &s->e[i].map;
+  const int slot = s->n < 256 ? s->n++ : (s->next++ & 255);
+  atc_map_entry& e = s->e[slot];
+  const jk_config& c = ctx->cfg;
+  const uint64_t dims[4] = {(uint64_t)c.head_dim, (uint64_t)rows, (uint64_t)c.n_kv_heads,
+                            (uint64_t)c.max_batch > (uint64_t)B ? (uint64_t)c.max_batch : (uint64_t)B};
+  const uint64_t strides[3] = {(uint64_t)c.head_dim * 2, (uint64_t)sh * 2, (uint64_t)sb * 2};
+  const uint32_t box[4] = {64, ATC_KEYS, 1, 1};
+  if (jk_tma_encode_bf16(ctx, &e.map, ptr, 4, dims, strides, box) != JK_OK) {
+    e.ptr = nullptr;
+    return nullptr;
+  }
+  e.ptr = ptr; e.sb = sb; e.sh = sh; e.rows = rows;
+  return &e.map;
+}
+
+void jk_attn_tc_destroy(jk_ctx* ctx) {
+  if (ctx && ctx->attn_tc_state) {
+    free(ctx->attn_tc_state);
+    ctx->attn_tc_state = nullptr;
+  }
+}
+
+int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
+               const void* vc, int64_t sb, int64_t sh, int cache_rows, const int32_t* kv_len,
+               const int32_t* parent, float scale, void* out) {
+  const jk_config& c = ctx->cfg;
+  const jk_ws_layout& L = ctx->lay;
+  if (!ctx->attn_tc_state) {
+    ctx->attn_tc_state = calloc(1, sizeof(atc_state));
+    if (!ctx->attn_tc_state) return JK_ERR_CUDA;
+  }
+  atc_state* s = (atc_state*)ctx->attn_tc_state;
+  // the map's batch extent must not reach past the caller's allocation: use B
+  const CUtensorMap* mk = atc_map(ctx, s, kc, sb, sh, cache_rows, B);
+  const CUtensorMap* mv = atc_map(ctx, s, vc, sb, sh, cache_rows, B);
+  if (!mk || !mv) return JK_ERR_CUDA;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int n_qblk = (G * M + ATC_ROWS - 1) / ATC_ROWS;
+  const int base = n_qblk * c.n_kv_heads * B;
+  const int tiles_max = (cache_rows + ATC_KEYS - 1) / ATC_KEYS;
+  int n_split = (2 * ctx->sm_count + base - 1) / base;
+  if (n_split > tiles_max) n_split = tiles_max;
+  if (n_split > L.attn_max_split) n_split = L.attn_max_split;
+  if (n_split < 1) n_split = 1;
+  const int D = c.head_dim;
+  const size_t smem = (size_t)ATC_ROWS * D * 2 + 2 * ATC_ROWS * 64 * 2 + (size_t)ATC_KEYS * D * 2 +
+                      sizeof(atc_tail) + 1024;
+  float* part_o = (float*)(ctx->ws + L.attn_o);
+  float* part_ml = (float*)(ctx->ws + L.attn_ml);
+  int32_t* status = (int32_t*)(ctx->ws + L.status);
+  const dim3 grid(n_split * n_qblk, c.n_kv_heads, B);
+  if (!s->smem_set) {
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_tc<128>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_tc<64>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+    s->smem_set = 1;
+  }
+  JK_PROF(ctx, st, JK_ST_ATTN);
+  if (D == 128)
+    k_tree_attn_tc<128><<<grid, 128, smem, st>>>(*mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+                                                 scale, M, c.n_q_heads, c.n_kv_heads, n_split,
+                                                 cache_rows, part_o, part_ml, status);
+  else
+    k_tree_attn_tc<64><<<grid, 128, smem, st>>>(*mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+                                                scale, M, c.n_q_heads, c.n_kv_heads, n_split,
+                                                cache_rows, part_o, part_ml, status);
+  JK_LAUNCH_CHECK(ctx);
+  return jk_attn_combine_launch(ctx, st, n_split, (size_t)B * M * c.n_q_heads, out);
+}

@@ -71,6 +71,7 @@ struct jk_ctx {
   int attn_smem_set;
   char cuda_err[256];
   void* tc_state;         // tensor-core path bookkeeping (tensor maps), host memory
+  void* attn_tc_state;    // tensor maps of the KV caches seen by the attention kernel
   jk_prof prof;
 };
 

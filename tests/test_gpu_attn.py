@@ -16,6 +16,7 @@ pytestmark = pytest.mark.gpu
 def _run(w, parent_np, ragged=False, layer=0):
     q, k, v, kv_len = synth.attn_inputs(w, layer, ragged)
     ctx = jk.Context.for_workload(w)
+    assert ctx.tensor_path_active == (w.dtype == "bf16")
     qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
     out = torch.empty_like(qd)
     ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, dev(kv_len), dev(parent_np),
@@ -54,6 +55,8 @@ def test_attn_tiny(name, kind):
     (37, 13, 8, 2, 128, 3),       # ragged tiles, GQA 4
     (300, 128, 4, 4, 64, 1),      # the largest tree
     (777, 60, 16, 2, 128, 2),     # GQA 8: several query blocks per kv head
+    (1500, 60, 32, 32, 128, 2),   # many heads: each CTA walks several key tiles (running max)
+    (900, 33, 16, 16, 64, 3),     # the same with head size 64
 ])
 def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype=dtype, prefix=P, tree_size=M,
