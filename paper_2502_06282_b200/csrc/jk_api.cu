@@ -25,6 +25,8 @@ static int validate_config(const jk_config& c) {
   if (c.n_kv_heads < 1 || c.n_q_heads < c.n_kv_heads || c.n_q_heads % c.n_kv_heads)
     return JK_ERR_SHAPE;
   if (!(c.rms_eps >= 0.f)) return JK_ERR_SHAPE;
+  // the top-k merge keeps chunks * k_e candidates in 16 registers per lane
+  if ((size_t)((c.vocab + JK_TOPK_CHUNK - 1) / JK_TOPK_CHUNK) * c.k_per_expert > 512) return JK_ERR_SHAPE;
   return JK_OK;
 }
 

@@ -9,51 +9,46 @@
 #include <math.h>
 
 #include "jk_common.cuh"
+#include "jk_topk.cuh"
 
 // tensor-core path (jk_gemm_tc.cu)
-int jk_tc_expert_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
-                     const int32_t* expert, int do_lm_head, float* logits, int RK,
-                     int rows_per_b, long long logits_stride_b);
+int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
+              const int32_t* expert, const float* gate, const void* u, void* out_feat);
+int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int RK, float* logits,
+                  int rows_per_b, long long logits_stride_b);
 int jk_tc_available(const jk_ctx* ctx);
 
 // ------------------------------------------------------------------------------------------
 // Router: RMSNorm, Eq. 2 softmax over the N centroids, Eq. 5 top-K gate.  One block per row.
 // ------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) k_router(
+__global__ void __launch_bounds__(512) k_router(
     const T* __restrict__ u, const T* __restrict__ router, const T* __restrict__ norm_w,
     int H, int N, int K, float eps, int use_norm, T* __restrict__ xn,
     float* __restrict__ out_probs, int32_t* __restrict__ out_expert, float* __restrict__ out_gate) {
+  // One pass over the row: the sum of squares and the N centroid dot products of u * gamma are
+  // accumulated together (the RMS factor is a scalar, applied to the dots afterwards).
   constexpr int VN = jk_vec<T>::N;
-  __shared__ float red[33];
-  __shared__ float zs[JK_MAX_EXPERTS];
+  __shared__ float part[16][JK_MAX_EXPERTS + 1];
+  __shared__ float tot[JK_MAX_EXPERTS + 1];
   const int row = blockIdx.x;
   const T* ur = u + (size_t)row * H;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   float ss = 0.f;
+  float z[JK_MAX_EXPERTS];
+#pragma unroll
+  for (int j = 0; j < JK_MAX_EXPERTS; ++j) z[j] = 0.f;
   for (int k = threadIdx.x * VN; k < H; k += blockDim.x * VN) {
     float v[VN];
     jk_vec<T>::load(ur + k, v);
 #pragma unroll
     for (int i = 0; i < VN; ++i) ss += v[i] * v[i];
-  }
-  ss = jk_block_sum(ss, red);
-  const float rinv = use_norm ? rsqrtf(ss / (float)H + eps) : 1.f;
-  float z[JK_MAX_EXPERTS];
-#pragma unroll
-  for (int j = 0; j < JK_MAX_EXPERTS; ++j) z[j] = 0.f;
-  for (int k = threadIdx.x * VN; k < H; k += blockDim.x * VN) {
-    float v[VN], g[VN];
-    jk_vec<T>::load(ur + k, v);
     if (use_norm && norm_w) {
+      float g[VN];
       jk_vec<T>::load(norm_w + k, g);
 #pragma unroll
-      for (int i = 0; i < VN; ++i) v[i] = v[i] * rinv * g[i];
-    } else {
-#pragma unroll
-      for (int i = 0; i < VN; ++i) v[i] = v[i] * rinv;
+      for (int i = 0; i < VN; ++i) v[i] *= g[i];
     }
-#pragma unroll
-    for (int i = 0; i < VN; ++i) xn[(size_t)row * H + k + i] = jk_from_float<T>(v[i]);
 #pragma unroll
     for (int j = 0; j < JK_MAX_EXPERTS; ++j) {
       if (j < N) {
@@ -64,21 +59,43 @@ __global__ void __launch_bounds__(256) k_router(
       }
     }
   }
+  ss = jk_warp_sum(ss);
 #pragma unroll
-  for (int j = 0; j < JK_MAX_EXPERTS; ++j) {
-    if (j < N) {
-      float t = jk_block_sum(z[j], red);
-      if (threadIdx.x == 0) zs[j] = t;
-    }
+  for (int j = 0; j < JK_MAX_EXPERTS; ++j) if (j < N) z[j] = jk_warp_sum(z[j]);
+  if (lane == 0) {
+    part[warp][JK_MAX_EXPERTS] = ss;
+#pragma unroll
+    for (int j = 0; j < JK_MAX_EXPERTS; ++j) if (j < N) part[warp][j] = z[j];
   }
   __syncthreads();
+  if (threadIdx.x <= JK_MAX_EXPERTS && (threadIdx.x < N || threadIdx.x == JK_MAX_EXPERTS)) {
+    float t = 0.f;
+    for (int w = 0; w < nw; ++w) t += part[w][threadIdx.x];
+    tot[threadIdx.x] = t;
+  }
+  __syncthreads();
+  const float rinv = use_norm ? rsqrtf(tot[JK_MAX_EXPERTS] / (float)H + eps) : 1.f;
+  // normalised hidden state for the expert GEMMs
+  for (int k = threadIdx.x * VN; k < H; k += blockDim.x * VN) {
+    float v[VN];
+    jk_vec<T>::load(ur + k, v);
+    if (use_norm && norm_w) {
+      float g[VN];
+      jk_vec<T>::load(norm_w + k, g);
+#pragma unroll
+      for (int i = 0; i < VN; ++i) v[i] *= g[i];
+    }
+#pragma unroll
+    for (int i = 0; i < VN; ++i) xn[(size_t)row * H + k + i] = jk_from_float<T>(v[i] * rinv);
+  }
   if (threadIdx.x == 0) {
+    float zs[JK_MAX_EXPERTS];
     float m = -INFINITY;
-    for (int j = 0; j < N; ++j) m = fmaxf(m, zs[j]);
-    float s[JK_MAX_EXPERTS], tot = 0.f;
-    for (int j = 0; j < N; ++j) { s[j] = expf(zs[j] - m); tot += s[j]; }
+    for (int j = 0; j < N; ++j) { zs[j] = tot[j] * rinv; m = fmaxf(m, zs[j]); }
+    float s[JK_MAX_EXPERTS], sum = 0.f;
+    for (int j = 0; j < N; ++j) { s[j] = expf(zs[j] - m); sum += s[j]; }
     for (int j = 0; j < N; ++j) {
-      s[j] = s[j] / tot;
+      s[j] = s[j] / sum;
       if (out_probs) out_probs[(size_t)row * N + j] = s[j];
     }
     unsigned taken = 0;
@@ -267,87 +284,46 @@ __global__ void __launch_bounds__(256) k_lmhead(
 __global__ void __launch_bounds__(256) k_topk_partial(
     const float* __restrict__ logits, int rows_per_b, long long stride_b, int V, int k_e,
     int chunks, float* __restrict__ tk_val, int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
-  constexpr int PER = JK_TOPK_CHUNK / 256;
-  __shared__ float red[33];
-  __shared__ float wv[8];
-  __shared__ int wi[8];
-  __shared__ int win_idx;
   const int chunk = blockIdx.x, row = blockIdx.y;
   const float* lr = logits + logit_row_off(row, rows_per_b, stride_b, V);
   const int base = chunk * JK_TOPK_CHUNK;
-  float vals[PER];
-  float lmax = -INFINITY;
+  float vals[JK_TOPK_PER];
 #pragma unroll
-  for (int j = 0; j < PER; ++j) {
+  for (int j = 0; j < JK_TOPK_PER; ++j) {
     const int idx = base + threadIdx.x + j * 256;
     vals[j] = idx < V ? lr[idx] : -INFINITY;
-    lmax = fmaxf(lmax, vals[j]);
   }
-  const float bmax = jk_block_max(lmax, red);
-  float s = 0.f;
-#pragma unroll
-  for (int j = 0; j < PER; ++j) {
-    const int idx = base + threadIdx.x + j * 256;
-    if (idx < V) s += expf(vals[j] - bmax);
-  }
-  const float bsum = jk_block_sum(s, red);
-  const size_t prow = (size_t)row * chunks + chunk;
-  if (threadIdx.x == 0) { tk_ms[prow * 2] = bmax; tk_ms[prow * 2 + 1] = bsum; }
-  unsigned taken = 0;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int it = 0; it < k_e; ++it) {
-    float bv = -INFINITY;
-    int bi = INT_MAX;
-#pragma unroll
-    for (int j = 0; j < PER; ++j) {
-      const int idx = base + threadIdx.x + j * 256;
-      if (!(taken & (1u << j)) && idx < V && jk_better(vals[j], idx, bv, bi)) { bv = vals[j]; bi = idx; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (jk_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
-    if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      float fv = wv[0];
-      int fi = wi[0];
-      for (int w = 1; w < 8; ++w)
-        if (jk_better(wv[w], wi[w], fv, fi)) { fv = wv[w]; fi = wi[w]; }
-      tk_val[prow * k_e + it] = fv;
-      tk_idx[prow * k_e + it] = fi;
-      win_idx = fi;
-    }
-    __syncthreads();
-    const int wsel = win_idx;
-    if (wsel != INT_MAX) {
-#pragma unroll
-      for (int j = 0; j < PER; ++j)
-        if (base + threadIdx.x + j * 256 == wsel) taken |= 1u << j;
-    }
-    __syncthreads();
-  }
+  jk_topk_chunk_select(vals, base, V, k_e, (size_t)row * chunks + chunk, tk_val, tk_idx, tk_ms);
 }
 
 // Merge the chunk partials of every logits row of one sequence, append the children to the
 // pool, then pick the next frontier.  One block per sequence.
-__global__ void __launch_bounds__(256) k_expand_finish(
+__global__ void __launch_bounds__(1024) k_expand_finish(
     int F, int K, int k_e, int chunks, int width,
     const float* __restrict__ tk_val, const int32_t* __restrict__ tk_idx,
     const float* __restrict__ tk_ms, const float* __restrict__ parent_score,
     const int32_t* __restrict__ parent_gidx, int gidx_base, int slot_base,
     jk_pool pool, float* __restrict__ out_lse, int32_t* __restrict__ next_frontier,
     float* __restrict__ next_parent_score, int32_t* __restrict__ next_parent_gidx) {
+  constexpr int PER_MAX = 16;                   // candidates per lane held in registers
   __shared__ float sc[JK_MAX_POOL];
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   const int rows = F * K;
   const size_t pb = (size_t)b * pool.stride_b;
+  const int nc = chunks * k_e;
   for (int lr = warp; lr < rows; lr += nw) {
     const int f = lr / K, r = lr % K;
     const size_t row = (size_t)b * rows + lr;
+    // candidates of this row: the chunks' partial winners (loaded once)
+    float cv[PER_MAX];
+    int ci[PER_MAX];
+#pragma unroll
+    for (int j = 0; j < PER_MAX; ++j) {
+      const int c = lane + j * 32;
+      cv[j] = c < nc ? tk_val[row * nc + c] : -INFINITY;
+      ci[j] = c < nc ? tk_idx[row * nc + c] : INT_MAX;
+    }
     // log-sum-exp over the chunk statistics
     float m = -INFINITY;
     for (int c = lane; c < chunks; c += 32) m = fmaxf(m, tk_ms[(row * chunks + c) * 2]);
@@ -358,23 +334,15 @@ __global__ void __launch_bounds__(256) k_expand_finish(
     s = jk_warp_sum(s);
     const float lse = m + logf(s);
     if (out_lse && lane == 0) out_lse[row] = lse;
-    // top-k_e of the chunks * k_e partial winners
-    const int nc = chunks * k_e;
-    const int per = (nc + 31) / 32;            // <= 16 with <= 32 chunks; more chunks loop below
-    unsigned long long taken = 0ull;
     const float ps = parent_score[(size_t)b * F + f];
     const int pg = parent_gidx[(size_t)b * F + f];
+    unsigned taken = 0u;
     for (int it = 0; it < k_e; ++it) {
       float bv = -INFINITY;
       int bi = INT_MAX, bj = -1;
-      for (int j = 0; j < per && j < 64; ++j) {
-        const int c = lane + j * 32;
-        if (c < nc && !(taken & (1ull << j))) {
-          const float v = tk_val[row * nc + c];
-          const int i = tk_idx[row * nc + c];
-          if (jk_better(v, i, bv, bi)) { bv = v; bi = i; bj = j; }
-        }
-      }
+#pragma unroll
+      for (int j = 0; j < PER_MAX; ++j)
+        if (!(taken & (1u << j)) && jk_better(cv[j], ci[j], bv, bi)) { bv = cv[j]; bi = ci[j]; bj = j; }
       float wv = bv;
       int wi = bi;
 #pragma unroll
@@ -383,7 +351,7 @@ __global__ void __launch_bounds__(256) k_expand_finish(
         const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
         if (jk_better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
       }
-      if (wi == bi && bj >= 0 && wi != INT_MAX) taken |= 1ull << bj;
+      if (wi == bi && bj >= 0 && wi != INT_MAX) taken |= 1u << bj;
       if (lane == 0) {
         const int flat = lr * k_e + it;
         const int g = gidx_base + flat;
@@ -518,13 +486,15 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
   const long long lsb = (out_logits && logits_stride_b) ? logits_stride_b : (long long)rows_per_b * V;
 
   JK_PROF(ctx, st, JK_ST_ROUTER);
-  k_router<T><<<R, 256, 0, st>>>((const T*)u, (const T*)w->router, (const T*)w->norm_weight, H,
+  k_router<T><<<R, 512, 0, st>>>((const T*)u, (const T*)w->router, (const T*)w->norm_weight, H,
                                  c.n_experts, K, c.rms_eps, c.use_pre_norm, xn, out_probs,
                                  out_expert, out_gate);
   JK_LAUNCH_CHECK(ctx);
   const bool tc = ctx->tensor_path && c.dtype == JK_BF16 && jk_tc_available(ctx);
   if (tc) {
-    int rc = jk_tc_expert_ffn(ctx, st, w, R, out_expert, 0, nullptr, RK, rows_per_b, lsb);
+    int rc = jk_tc_ffn(ctx, st, w, R, out_expert, out_gate, u, out_feat);
+    if (rc != JK_OK) return rc;
+    rc = jk_tc_lm_head(ctx, st, w, RK, out_logits, rows_per_b, lsb);
     if (rc != JK_OK) return rc;
   } else {
     JK_PROF(ctx, st, JK_ST_GATEUP);
@@ -535,27 +505,22 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
     k_down<T><<<dim3((H + 15) / 16, c.n_experts), 256, 0, st>>>(
         (const T*)w->w_down, hbuf, out_expert, R, K, H, I, Rp, ybuf);
     JK_LAUNCH_CHECK(ctx);
-  }
-  JK_PROF(ctx, st, JK_ST_BRANCH);
-  k_branch<T><<<R, 256, 0, st>>>((const T*)u, ybuf, out_expert, out_gate, K, H, Rp,
-                                 c.branch_residual, bbuf, (T*)out_feat);
-  JK_LAUNCH_CHECK(ctx);
-  if (tc) {
-    int rc = jk_tc_expert_ffn(ctx, st, w, R, out_expert, 1, logits, RK, rows_per_b, lsb);
-    if (rc != JK_OK) return rc;
-  } else {
+    JK_PROF(ctx, st, JK_ST_BRANCH);
+    k_branch<T><<<R, 256, 0, st>>>((const T*)u, ybuf, out_expert, out_gate, K, H, Rp,
+                                   c.branch_residual, bbuf, (T*)out_feat);
+    JK_LAUNCH_CHECK(ctx);
     JK_PROF(ctx, st, JK_ST_LMHEAD);
     k_lmhead<T><<<(V + 31) / 32, 256, 0, st>>>((const T*)w->lm_head, bbuf, RK, H, V, logits,
                                                rows_per_b, lsb);
     JK_LAUNCH_CHECK(ctx);
+    JK_PROF(ctx, st, JK_ST_TOPK);
+    k_topk_partial<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
+        logits, rows_per_b, lsb, V, c.k_per_expert, L.topk_chunks, (float*)(ws + L.tk_val),
+        (int32_t*)(ws + L.tk_idx), (float*)(ws + L.tk_ms));
+    JK_LAUNCH_CHECK(ctx);
   }
-  JK_PROF(ctx, st, JK_ST_TOPK);
-  k_topk_partial<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
-      logits, rows_per_b, lsb, V, c.k_per_expert, L.topk_chunks, (float*)(ws + L.tk_val),
-      (int32_t*)(ws + L.tk_idx), (float*)(ws + L.tk_ms));
-  JK_LAUNCH_CHECK(ctx);
   JK_PROF(ctx, st, JK_ST_FINISH);
-  k_expand_finish<<<B, 256, 0, st>>>(F, K, c.k_per_expert, L.topk_chunks, width,
+  k_expand_finish<<<B, 1024, 0, st>>>(F, K, c.k_per_expert, L.topk_chunks, width,
                                      (const float*)(ws + L.tk_val),
                                      (const int32_t*)(ws + L.tk_idx),
                                      (const float*)(ws + L.tk_ms), parent_score, parent_gidx,

@@ -12,7 +12,8 @@
 //   - a producer thread feeds a ring of shared-memory stages with TMA (128B swizzle), one thread
 //     issues the MMAs, four warps drain finished accumulators to fp32 partial tiles in global
 //     memory; a small second kernel adds the partials of each tile in a fixed order (no atomics,
-//     bitwise reproducible) and applies the epilogue (SiLU * up, or a plain store).
+//     bitwise reproducible) and applies the epilogue: SiLU * up; residual, gates and branch
+//     features; or the LM head's per-chunk top-k statistics.
 // Every wait on an mbarrier is bounded: after ~2 s it records JK_ERR_TIMEOUT in the status word,
 // and the CTA drains its copies, frees its tensor memory and returns.
 #include <cuda.h>
@@ -20,6 +21,7 @@
 
 #include "jk_common.cuh"
 #include "jk_tcgen05.cuh"
+#include "jk_topk.cuh"
 
 #define TC_TILE_M 128
 #define TC_TILE_K 64
@@ -65,12 +67,14 @@ struct tc_plan {
 
 __device__ __forceinline__ void tc_make_plan(const tc_params& p, const int32_t* expert,
                                              tc_plan* plan) {
-  // one thread
+  // called by one whole warp; lane 0 writes the plan
   unsigned active = 0;
-  for (int i = 0; i < p.R * p.K_top; ++i) {
+  for (int i = threadIdx.x & 31; i < p.R * p.K_top; i += 32) {
     const int e = expert[i];
     if (e >= 0 && e < p.n_experts) active |= 1u << e;
   }
+  active = __reduce_or_sync(0xffffffffu, active);
+  if ((threadIdx.x & 31) != 0) return;
   int n = 0;
   for (int g = 0; g < p.n_groups_max; ++g) {
     const int e = p.group_expert[g];
@@ -108,8 +112,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
     for (int s = 0; s < p.stages; ++s) { mbar_init(&T.full[s], 1); mbar_init(&T.empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&T.acc_full[a], 1); mbar_init(&T.acc_empty[a], 4); }
     T.abort_flag = 0;
-    tc_make_plan(p, expert, &T.plan);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tc_make_plan(p, expert, &T.plan);
   }
   if (warp == 1) {
     tmem_alloc(&T.tmem_base, (uint32_t)p.tmem_cols);
@@ -129,21 +136,38 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
     // ------------------------------------------------------------------ TMA producer
     int issued = 0;
     bool ok = true;
-    for (long long u = u0; u < u1 && ok; ++u, ++issued) {
-      const int s = issued % p.stages;
-      const uint32_t ph = (uint32_t)(issued / p.stages) & 1u;
+    // position of the span's first unit; advanced incrementally (no divisions in the loop)
+    int kt = (int)(u0 % units_per_tile);
+    int t = (int)(first_tile % p.tiles_per_group);
+    int gi = (int)(first_tile / p.tiles_per_group);
+    int g = (u0 < u1) ? T.plan.group_src[gi] : 0;
+    const CUtensorMap* ma = p.group_amap[g] ? &map_a1 : &map_a0;
+    int arow = p.group_arow0[g] + t * TC_TILE_M, brow = p.group_brow0[g];
+    int s = 0;
+    uint32_t ph = 0;
+    const int n_units = (int)(u1 - u0);
+    for (; issued < n_units; ++issued) {
       if (issued >= p.stages) ok = mbar_wait(&T.empty[s], ph ^ 1u, abort_flag, status);
       if (!ok) break;
-      const long long tile = u / units_per_tile;
-      const int kt = (int)(u - tile * units_per_tile);
-      const int g = T.plan.group_src[(int)(tile / p.tiles_per_group)];
-      const int t = (int)(tile % p.tiles_per_group);
       unsigned char* sa = smem + (size_t)s * stage_bytes;
       unsigned char* sb = sa + TC_TILE_M * TC_TILE_K * 2;
       mbar_expect_tx(&T.full[s], (uint32_t)stage_bytes);
-      tma_load_2d(sa, p.group_amap[g] ? &map_a1 : &map_a0, kt * TC_TILE_K,
-                  p.group_arow0[g] + t * TC_TILE_M, &T.full[s]);
-      tma_load_2d(sb, &map_b, kt * TC_TILE_K, p.group_brow0[g], &T.full[s]);
+      tma_load_2d(sa, ma, kt * TC_TILE_K, arow, &T.full[s]);
+      tma_load_2d(sb, &map_b, kt * TC_TILE_K, brow, &T.full[s]);
+      if (++s == p.stages) { s = 0; ph ^= 1u; }
+      if (++kt == units_per_tile) {
+        kt = 0;
+        if (++t == p.tiles_per_group) {
+          t = 0;
+          ++gi;
+          if (issued + 1 < n_units) {
+            g = T.plan.group_src[gi];
+            ma = p.group_amap[g] ? &map_a1 : &map_a0;
+            brow = p.group_brow0[g];
+          }
+        }
+        arow = p.group_arow0[g] + t * TC_TILE_M;
+      }
     }
     if (!ok) {
       // gave up: let the copies already in flight land before the CTA's memory goes away
@@ -157,11 +181,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
   } else if (warp == 1 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
     const uint32_t idesc = instr_desc_bf16(p.n_pad);
-    int consumed = 0, seg = 0;
+    int seg = 0, s = 0;
+    uint32_t fph = 0;
     bool ok = true;
-    for (long long u = u0; u < u1 && ok; ++seg) {
-      const long long tile = u / units_per_tile;
-      const long long tile_end = (tile + 1) * units_per_tile;
+    long long tile_end = (first_tile + 1) * units_per_tile;
+    for (long long u = u0; u < u1 && ok; ++seg, tile_end += units_per_tile) {
       const long long ue = tile_end < u1 ? tile_end : u1;
       const int acc = seg & 1;
       if (seg >= 2) ok = mbar_wait(&T.acc_empty[acc], ((uint32_t)(seg >> 1) & 1u) ^ 1u, abort_flag, status);
@@ -169,9 +193,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       tc_fence_after();
       const uint32_t d_addr = tmem_base + (uint32_t)(acc * p.n_pad);
       bool first = true;
-      for (; u < ue; ++u, ++consumed) {
-        const int s = consumed % p.stages;
-        ok = mbar_wait(&T.full[s], (uint32_t)(consumed / p.stages) & 1u, abort_flag, status);
+      for (; u < ue; ++u) {
+        ok = mbar_wait(&T.full[s], fph, abort_flag, status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
@@ -185,6 +208,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
         }
         first = false;
         tc_commit(&T.empty[s]);          // the stage is free once these MMAs have read it
+        if (++s == p.stages) { s = 0; fph ^= 1u; }
       }
       if (ok) tc_commit(&T.acc_full[acc]);
     }
@@ -227,24 +251,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
 }
 
 // ---------------------------------------------------------------------------------------------
-// Fix-up: out[n, m] = sum over the CTAs that touched the tile, in ascending CTA order.
-//   mode 0: out[(group_out0[g] + n) * ld + m]          (plain store, fp32)
-//   mode 1: groups come in (gate, up) pairs: h = SiLU(gate) * up as bf16
+// Fix-up kernels: every output element is the sum of the partial tiles of the CTAs whose spans
+// touched its tile, added in ascending CTA order (fixed order: bitwise reproducible), followed by
+// the epilogue of the contraction.
 // ---------------------------------------------------------------------------------------------
-struct tc_fix_params {
-  int mode;
-  int m_rows;                        // valid rows of a group (I, H or V)
-  int n_rows;                        // valid activation rows
-  long long ld;                      // output leading dimension (elements)
-  long long group_out0[TC_MAX_GROUPS];   // element offset of the group's output block (by source group)
-  int n_cta;                         // grid of the GEMM kernel
-  int rows_per_b;                    // mode 0 with a batch stride: n -> (n / rows_per_b, n % rows_per_b)
-  long long stride_b;
-};
+#define TC_MAX_CONTRIB 8
 
-__device__ __forceinline__ float tc_tile_sum(const float* __restrict__ partial, const tc_params& p,
-                                             long long total, int n_cta, long long tile, int n,
-                                             int m) {
+// Partial-tile slots that add up to `tile`, ascending CTA order.  Returns the count, or -1 if
+// there are more than TC_MAX_CONTRIB (then tc_tile_sum_slow is used).
+__device__ __forceinline__ int tc_tile_slots(const tc_params& p, long long total, int n_cta,
+                                             long long tile, int* slots) {
+  const long long a = tile * p.kt, b = a + p.kt;
+  int c = (int)(a * n_cta / total);
+  while (c + 1 < n_cta && tc_span_start(total, c + 1, n_cta) <= a) ++c;
+  while (c > 0 && tc_span_start(total, c, n_cta) > a) --c;
+  int n = 0;
+  for (; c < n_cta; ++c) {
+    const long long s0 = tc_span_start(total, c, n_cta);
+    if (s0 >= b) break;
+    const long long s1 = tc_span_start(total, c + 1, n_cta);
+    if (s1 <= a || s1 == s0) continue;                        // before the tile, or empty
+    if (n == TC_MAX_CONTRIB) return -1;
+    slots[n++] = c * p.max_seg + (int)(tile - s0 / p.kt);
+  }
+  return n;
+}
+
+__device__ __forceinline__ float tc_tile_sum_slow(const float* __restrict__ partial,
+                                                  const tc_params& p, long long total, int n_cta,
+                                                  long long tile, int n, int m) {
   const long long a = tile * p.kt, b = a + p.kt;
   int c = (int)(a * n_cta / total);
   while (c + 1 < n_cta && tc_span_start(total, c + 1, n_cta) <= a) ++c;
@@ -254,52 +289,127 @@ __device__ __forceinline__ float tc_tile_sum(const float* __restrict__ partial, 
     const long long s0 = tc_span_start(total, c, n_cta);
     if (s0 >= b) break;
     const long long s1 = tc_span_start(total, c + 1, n_cta);
-    if (s1 <= a || s1 == s0) continue;                        // before the tile, or empty
-    const long long first_tile = s0 / p.kt;
-    const int slot = c * p.max_seg + (int)(tile - first_tile);
+    if (s1 <= a || s1 == s0) continue;
+    const int slot = c * p.max_seg + (int)(tile - s0 / p.kt);
     acc += partial[((size_t)slot * p.n_pad + n) * TC_TILE_M + m];
   }
   return acc;
 }
 
-__global__ void __launch_bounds__(128) k_tc_fixup(const tc_params p, const tc_fix_params f,
-                                                  const int32_t* __restrict__ expert,
-                                                  const float* __restrict__ partial,
-                                                  void* __restrict__ out) {
+struct tc_slot_list {
+  int n;
+  int slot[TC_MAX_CONTRIB];
+};
+
+__device__ __forceinline__ float tc_sum_list(const float* __restrict__ partial, const tc_params& p,
+                                             const tc_slot_list& L, long long total, int n_cta,
+                                             long long tile, int n, int m) {
+  if (L.n < 0) return tc_tile_sum_slow(partial, p, total, n_cta, tile, n, m);
+  float acc = 0.f;
+  for (int i = 0; i < L.n; ++i) acc += partial[((size_t)L.slot[i] * p.n_pad + n) * TC_TILE_M + m];
+  return acc;
+}
+
+// h[e, n, i] = SiLU(gate) * up for every touched expert (Eq. 3's Expert_j, first half).
+// grid (tiles over I, experts, row slices); groups come in (gate, up) pairs.
+__global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int n_cta, int I, int n_rows,
+                                                     int Rp, const int32_t* __restrict__ expert,
+                                                     const float* __restrict__ partial,
+                                                     __nv_bfloat16* __restrict__ hbuf) {
   __shared__ tc_plan plan;
-  if (threadIdx.x == 0) tc_make_plan(p, expert, &plan);
+  __shared__ tc_slot_list lg, lu;
+  if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
   __syncthreads();
-  const int t = blockIdx.x;                       // tile within the group
-  const int go = blockIdx.y;                      // output group (a pair of groups in mode 1)
-  const int m = threadIdx.x;
-  const int mg = t * TC_TILE_M + m;
+  const int t = blockIdx.x, go = blockIdx.y, m = threadIdx.x;
+  if (2 * go + 1 >= plan.n_groups) return;
   const long long total = plan.total_units;
-  if (f.mode == 1) {
-    if (2 * go + 1 >= plan.n_groups || mg >= f.m_rows) return;
-    const int src = plan.group_src[2 * go];
-    const long long tile_g = (long long)(2 * go) * p.tiles_per_group + t;
-    const long long tile_u = (long long)(2 * go + 1) * p.tiles_per_group + t;
-    __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + f.group_out0[src];
-    for (int n = blockIdx.z; n < f.n_rows; n += gridDim.z) {
-      const float g = tc_tile_sum(partial, p, total, f.n_cta, tile_g, n, m);
-      const float u = tc_tile_sum(partial, p, total, f.n_cta, tile_u, n, m);
-      o[(size_t)n * f.ld + mg] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
-    }
-  } else {
-    if (go >= plan.n_groups || mg >= f.m_rows) return;
-    const int src = plan.group_src[go];
-    const long long tile = (long long)go * p.tiles_per_group + t;
-    float* o = reinterpret_cast<float*>(out) + f.group_out0[src];
-    for (int n = blockIdx.z; n < f.n_rows; n += gridDim.z) {
-      const float v = tc_tile_sum(partial, p, total, f.n_cta, tile, n, m);
-      size_t off;
-      if (f.rows_per_b > 0)
-        off = (size_t)(n / f.rows_per_b) * (size_t)f.stride_b + (size_t)(n % f.rows_per_b) * f.ld;
-      else
-        off = (size_t)n * f.ld;
-      o[off + mg] = v;
-    }
+  const long long tile_g = (long long)(2 * go) * p.tiles_per_group + t;
+  const long long tile_u = tile_g + p.tiles_per_group;
+  if (threadIdx.x == 0) lg.n = tc_tile_slots(p, total, n_cta, tile_g, lg.slot);
+  if (threadIdx.x == 32) lu.n = tc_tile_slots(p, total, n_cta, tile_u, lu.slot);
+  __syncthreads();
+  const int i = t * TC_TILE_M + m;
+  if (i >= I) return;
+  const int e = p.group_expert[plan.group_src[2 * go]];
+  __nv_bfloat16* o = hbuf + (size_t)e * Rp * I + i;
+#pragma unroll 4
+  for (int n = blockIdx.z; n < n_rows; n += gridDim.z) {
+    const float g = tc_sum_list(partial, p, lg, total, n_cta, tile_g, n, m);
+    const float u = tc_sum_list(partial, p, lu, total, n_cta, tile_u, n, m);
+    o[(size_t)n * I] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
   }
+}
+
+// y_r = W_down h for the K experts of row r, then Eq. 3 and the branch features:
+//   f = u + sum_r g_r y_r,  b_r = g_r y_r (+ u).   grid (tiles over H, rows).
+__global__ void __launch_bounds__(128) k_tc_fix_down_branch(
+    const tc_params p, int n_cta, int H, const int32_t* __restrict__ expert,
+    const float* __restrict__ gate, const __nv_bfloat16* __restrict__ u, int branch_residual,
+    const float* __restrict__ partial, __nv_bfloat16* __restrict__ bbuf,
+    __nv_bfloat16* __restrict__ out_feat) {
+  __shared__ tc_plan plan;
+  __shared__ tc_slot_list lists[JK_MAX_EXPERTS];
+  __shared__ long long tiles[JK_MAX_EXPERTS];
+  if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
+  __syncthreads();
+  const int t = blockIdx.x, r = blockIdx.y, m = threadIdx.x;
+  const int K = p.K_top;
+  const long long total = plan.total_units;
+  if (threadIdx.x < K) {
+    const int e = expert[r * K + threadIdx.x];
+    int ga = 0;                       // position of expert e among the active groups
+    for (int g = 0; g < plan.n_groups; ++g)
+      if (p.group_expert[plan.group_src[g]] == e) ga = g;
+    tiles[threadIdx.x] = (long long)ga * p.tiles_per_group + t;
+    lists[threadIdx.x].n = tc_tile_slots(p, total, n_cta, tiles[threadIdx.x], lists[threadIdx.x].slot);
+  }
+  __syncthreads();
+  const int h = t * TC_TILE_M + m;
+  if (h >= H) return;
+  const float uv = __bfloat162float(u[(size_t)r * H + h]);
+  float f = uv;
+  for (int k = 0; k < K; ++k) {
+    const float y = tc_sum_list(partial, p, lists[k], total, n_cta, tiles[k], r, m);
+    const float gy = gate[r * K + k] * y;
+    f += gy;
+    bbuf[((size_t)r * K + k) * H + h] = __float2bfloat16_rn(branch_residual ? gy + uv : gy);
+  }
+  out_feat[(size_t)r * H + h] = __float2bfloat16_rn(f);
+}
+
+// logits = b W_head^T (Eq. 4) assembled from the partial tiles, optionally stored, and the
+// per-chunk top-k statistics of jk_topk.cuh.   grid (chunks, logits rows), 256 threads.
+__global__ void __launch_bounds__(256) k_tc_fix_lmhead_topk(
+    const tc_params p, int n_cta, int V, int k_e, int chunks, const float* __restrict__ partial,
+    float* __restrict__ logits, int rows_per_b, long long stride_b, float* __restrict__ tk_val,
+    int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
+  constexpr int TILES = JK_TOPK_CHUNK / TC_TILE_M;     // 32 tiles per chunk
+  __shared__ tc_slot_list lists[TILES];
+  const int chunk = blockIdx.x, row = blockIdx.y;
+  const long long total = (long long)p.tiles_per_group * p.kt;     // one group, always active
+  if (threadIdx.x < TILES) {
+    const long long tile = (long long)chunk * TILES + threadIdx.x;
+    lists[threadIdx.x].n = tile < p.tiles_per_group
+                               ? tc_tile_slots(p, total, n_cta, tile, lists[threadIdx.x].slot) : 0;
+  }
+  __syncthreads();
+  const int base = chunk * JK_TOPK_CHUNK;
+  float vals[JK_TOPK_PER];
+  float* lrow = logits ? logits + (size_t)(row / rows_per_b) * (size_t)stride_b +
+                             (size_t)(row % rows_per_b) * V : nullptr;
+#pragma unroll
+  for (int j = 0; j < JK_TOPK_PER; ++j) {
+    const int off = threadIdx.x + j * 256;             // within the chunk
+    const int idx = base + off;
+    float v = -INFINITY;
+    if (idx < V) {
+      const int tl = off / TC_TILE_M, m = off % TC_TILE_M;
+      v = tc_sum_list(partial, p, lists[tl], total, n_cta, (long long)chunk * TILES + tl, row, m);
+      if (lrow) lrow[idx] = v;
+    }
+    vals[j] = v;
+  }
+  jk_topk_chunk_select(vals, base, V, k_e, (size_t)row * chunks + chunk, tk_val, tk_idx, tk_ms);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -325,9 +435,10 @@ struct tc_state {
   int failed;
 };
 
+#define TC_MAX_GRID 192
 static int tc_grid(const jk_ctx* ctx) {
   const int n = ctx->sm_count > 0 ? ctx->sm_count : 148;
-  return n > 192 ? 192 : n;
+  return n > TC_MAX_GRID ? TC_MAX_GRID : n;
 }
 
 static int tc_stage_bytes(int n_pad) { return TC_TILE_M * TC_TILE_K * 2 + n_pad * TC_TILE_K * 2; }
@@ -343,23 +454,21 @@ static int tc_max_seg(long long max_units, int n_cta, int kt) {
   return (int)((span + kt - 1) / kt) + 1;
 }
 
-// n_cta * max_seg <= tiles + 3 * n_cta for any grid size; grids are capped at TC_MAX_GRID.
-#define TC_MAX_GRID 192
-static size_t tc_partial_for(long long units, int, int kt, int n_pad) {
+// n_cta * max_seg <= tiles + 3 * n_cta for any grid size up to TC_MAX_GRID.
+static size_t tc_partial_for(long long units, int kt, int n_pad) {
   return (size_t)(units / kt + 3 * TC_MAX_GRID) * n_pad * TC_TILE_M * sizeof(float);
 }
 
 // Worst case over the three contractions.
 size_t jk_tc_partial_bytes(const jk_config& c) {
-  const int n_cta = TC_MAX_GRID;
   const int R = c.max_batch * c.max_frontier;
   const int np1 = (int)jk_align_up(R, 16), np2 = (int)jk_align_up((size_t)R * c.top_k, 16);
   const int kt_h = (c.hidden + TC_TILE_K - 1) / TC_TILE_K, kt_i = (c.inter + TC_TILE_K - 1) / TC_TILE_K;
   const long long t_i = (c.inter + TC_TILE_M - 1) / TC_TILE_M, t_h = (c.hidden + TC_TILE_M - 1) / TC_TILE_M,
                   t_v = (c.vocab + TC_TILE_M - 1) / TC_TILE_M;
-  size_t a = tc_partial_for(2ll * c.n_experts * t_i * kt_h, n_cta, kt_h, np1);
-  size_t b = tc_partial_for((long long)c.n_experts * t_h * kt_i, n_cta, kt_i, np1);
-  size_t d = tc_partial_for(t_v * kt_h, n_cta, kt_h, np2);
+  size_t a = tc_partial_for(2ll * c.n_experts * t_i * kt_h, kt_h, np1);
+  size_t b = tc_partial_for((long long)c.n_experts * t_h * kt_i, kt_i, np1);
+  size_t d = tc_partial_for(t_v * kt_h, kt_h, np2);
   size_t m = a > b ? a : b;
   return m > d ? m : d;
 }
@@ -426,10 +535,10 @@ static const CUtensorMap* tc_map(jk_ctx* ctx, tc_state* s, const void* ptr, uint
   return &e.map;
 }
 
-static int tc_launch(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUtensorMap* a0,
-                     const CUtensorMap* a1, const CUtensorMap* b, tc_params& p,
-                     const tc_fix_params& f, const int32_t* expert, void* out, int out_groups,
-                     int stage_id) {
+// Launch the streaming GEMM; fills the launch-dependent fields of p and returns the grid size.
+static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUtensorMap* a0,
+                          const CUtensorMap* a1, const CUtensorMap* b, tc_params& p,
+                          const int32_t* expert, int stage_id, int* n_cta_out) {
   const jk_ws_layout& L = ctx->lay;
   const int n_cta = tc_grid(ctx);
   p.stages = tc_stages(p.n_pad);
@@ -446,71 +555,88 @@ static int tc_launch(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUtensorMa
                                             TC_SMEM_BUDGET));
     s->smem_set = 1;
   }
-  float* partial = (float*)(ctx->ws + L.gemm_part);
-  int32_t* status = (int32_t*)(ctx->ws + L.status);
   JK_PROF(ctx, st, stage_id);
-  k_tc_gemm<<<n_cta, TC_THREADS, smem, st>>>(*a0, *a1, *b, p, expert, partial, status);
+  k_tc_gemm<<<n_cta, TC_THREADS, smem, st>>>(*a0, *a1, *b, p, expert,
+                                             (float*)(ctx->ws + L.gemm_part),
+                                             (int32_t*)(ctx->ws + L.status));
   JK_LAUNCH_CHECK(ctx);
-  tc_fix_params ff = f;
-  ff.n_cta = n_cta;
-  int zdim = 1;
-  const int base = p.tiles_per_group * out_groups;
-  while (zdim < ff.n_rows && base * zdim < 2 * n_cta) zdim <<= 1;
-  JK_PROF(ctx, st, JK_ST_GEMM_FIXUP);
-  k_tc_fixup<<<dim3(p.tiles_per_group, out_groups, zdim), 128, 0, st>>>(p, ff, expert, partial, out);
-  JK_LAUNCH_CHECK(ctx);
+  *n_cta_out = n_cta;
   return JK_OK;
 }
 
-// do_lm_head = 0: h = SiLU(W_gate x) * (W_up x) and y = W_down h for every touched expert
-//                 (hbuf, ybuf of the workspace);  do_lm_head = 1: logits = b W_head^T.
-int jk_tc_expert_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
-                     const int32_t* expert, int do_lm_head, float* logits, int RK, int rows_per_b,
-                     long long logits_stride_b) {
+static int tc_zdim(int base_blocks, int n_rows, int n_cta) {
+  int z = 1;
+  while (z < n_rows && base_blocks * z < 2 * n_cta) z <<= 1;
+  return z;
+}
+
+// Expert FFNs of the draft layer (Eq. 3) on the tensor core: gate/up GEMM, SiLU * up, down GEMM,
+// then the combined feature and the branch features (LM-head input).
+int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
+              const int32_t* expert, const float* gate, const void* u, void* out_feat) {
   tc_state* s = tc_get_state(ctx);
   if (!s || s->failed) return JK_ERR_CUDA;
   const jk_config& c = ctx->cfg;
   const jk_ws_layout& L = ctx->lay;
-  const int H = c.hidden, I = c.inter, V = c.vocab, N = c.n_experts, Rp = L.rows_pad;
+  const int H = c.hidden, I = c.inter, N = c.n_experts, Rp = L.rows_pad;
+  const float* partial = (const float*)(ctx->ws + L.gemm_part);
   tc_params p;
   memset(&p, 0, sizeof(p));
   p.R = R; p.K_top = c.top_k; p.n_experts = N;
-  tc_fix_params f;
-  memset(&f, 0, sizeof(f));
-  if (!do_lm_head) {
-    const int n_pad = (int)jk_align_up(R, 16);
-    // gate / up
-    const CUtensorMap* ag = tc_map(ctx, s, w->w_gate, (uint64_t)N * I, H, TC_TILE_M);
-    const CUtensorMap* au = tc_map(ctx, s, w->w_up, (uint64_t)N * I, H, TC_TILE_M);
-    const CUtensorMap* bx = tc_map(ctx, s, ctx->ws + L.xn, Rp, H, n_pad);
-    if (!ag || !au || !bx) return JK_ERR_CUDA;
-    p.n_groups_max = 2 * N;
-    for (int e = 0; e < N; ++e)
-      for (int h = 0; h < 2; ++h) {
-        const int g = 2 * e + h;
-        p.group_expert[g] = e; p.group_amap[g] = h; p.group_arow0[g] = e * I; p.group_brow0[g] = 0;
-        f.group_out0[g] = (long long)e * Rp * I;
-      }
-    p.tiles_per_group = (I + TC_TILE_M - 1) / TC_TILE_M;
-    p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
-    p.n_pad = n_pad;
-    f.mode = 1; f.m_rows = I; f.n_rows = R; f.ld = I;
-    int rc = tc_launch(ctx, st, s, ag, au, bx, p, f, expert, ctx->ws + L.hbuf, N, JK_ST_GATEUP);
-    if (rc != JK_OK) return rc;
-    // down
-    const CUtensorMap* ad = tc_map(ctx, s, w->w_down, (uint64_t)N * H, I, TC_TILE_M);
-    const CUtensorMap* bh = tc_map(ctx, s, ctx->ws + L.hbuf, (uint64_t)N * Rp, I, n_pad);
-    if (!ad || !bh) return JK_ERR_CUDA;
-    p.n_groups_max = N;
-    for (int e = 0; e < N; ++e) {
-      p.group_expert[e] = e; p.group_amap[e] = 0; p.group_arow0[e] = e * H; p.group_brow0[e] = e * Rp;
-      f.group_out0[e] = (long long)e * Rp * H;
+  const int n_pad = (int)jk_align_up(R, 16);
+  int n_cta = 0;
+  // gate / up
+  const CUtensorMap* ag = tc_map(ctx, s, w->w_gate, (uint64_t)N * I, H, TC_TILE_M);
+  const CUtensorMap* au = tc_map(ctx, s, w->w_up, (uint64_t)N * I, H, TC_TILE_M);
+  const CUtensorMap* bx = tc_map(ctx, s, ctx->ws + L.xn, Rp, H, n_pad);
+  if (!ag || !au || !bx) return JK_ERR_CUDA;
+  p.n_groups_max = 2 * N;
+  for (int e = 0; e < N; ++e)
+    for (int h = 0; h < 2; ++h) {
+      const int g = 2 * e + h;
+      p.group_expert[g] = e; p.group_amap[g] = h; p.group_arow0[g] = e * I; p.group_brow0[g] = 0;
     }
-    p.tiles_per_group = (H + TC_TILE_M - 1) / TC_TILE_M;
-    p.kt = (I + TC_TILE_K - 1) / TC_TILE_K;
-    f.mode = 0; f.m_rows = H; f.n_rows = R; f.ld = H; f.rows_per_b = 0;
-    return tc_launch(ctx, st, s, ad, ad, bh, p, f, expert, ctx->ws + L.ybuf, N, JK_ST_DOWN);
+  p.tiles_per_group = (I + TC_TILE_M - 1) / TC_TILE_M;
+  p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
+  p.n_pad = n_pad;
+  int rc = tc_launch_gemm(ctx, st, s, ag, au, bx, p, expert, JK_ST_GATEUP, &n_cta);
+  if (rc != JK_OK) return rc;
+  JK_PROF(ctx, st, JK_ST_GEMM_FIXUP);
+  k_tc_fix_silu<<<dim3(p.tiles_per_group, N, tc_zdim(p.tiles_per_group * N, R, n_cta)), 128, 0, st>>>(
+      p, n_cta, I, R, Rp, expert, partial, (__nv_bfloat16*)(ctx->ws + L.hbuf));
+  JK_LAUNCH_CHECK(ctx);
+  // down
+  const CUtensorMap* ad = tc_map(ctx, s, w->w_down, (uint64_t)N * H, I, TC_TILE_M);
+  const CUtensorMap* bh = tc_map(ctx, s, ctx->ws + L.hbuf, (uint64_t)N * Rp, I, n_pad);
+  if (!ad || !bh) return JK_ERR_CUDA;
+  p.n_groups_max = N;
+  for (int e = 0; e < N; ++e) {
+    p.group_expert[e] = e; p.group_amap[e] = 0; p.group_arow0[e] = e * H; p.group_brow0[e] = e * Rp;
   }
+  p.tiles_per_group = (H + TC_TILE_M - 1) / TC_TILE_M;
+  p.kt = (I + TC_TILE_K - 1) / TC_TILE_K;
+  rc = tc_launch_gemm(ctx, st, s, ad, ad, bh, p, expert, JK_ST_DOWN, &n_cta);
+  if (rc != JK_OK) return rc;
+  JK_PROF(ctx, st, JK_ST_BRANCH);
+  k_tc_fix_down_branch<<<dim3(p.tiles_per_group, R), 128, 0, st>>>(
+      p, n_cta, H, expert, gate, (const __nv_bfloat16*)u, c.branch_residual, partial,
+      (__nv_bfloat16*)(ctx->ws + L.bbuf), (__nv_bfloat16*)out_feat);
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
+
+// Shared LM head (Eq. 4) on the tensor core, with the per-chunk top-k statistics; `logits` may be
+// NULL when the caller does not keep the draft distributions.
+int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int RK, float* logits,
+                  int rows_per_b, long long logits_stride_b) {
+  tc_state* s = tc_get_state(ctx);
+  if (!s || s->failed) return JK_ERR_CUDA;
+  const jk_config& c = ctx->cfg;
+  const jk_ws_layout& L = ctx->lay;
+  const int H = c.hidden, V = c.vocab;
+  tc_params p;
+  memset(&p, 0, sizeof(p));
+  p.R = 0; p.K_top = c.top_k; p.n_experts = c.n_experts;
   const int n_pad = (int)jk_align_up(RK, 16);
   const CUtensorMap* ah = tc_map(ctx, s, w->lm_head, V, H, TC_TILE_M);
   const CUtensorMap* bb = tc_map(ctx, s, ctx->ws + L.bbuf, L.rk_pad, H, n_pad);
@@ -520,9 +646,16 @@ int jk_tc_expert_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, in
   p.tiles_per_group = (V + TC_TILE_M - 1) / TC_TILE_M;
   p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
   p.n_pad = n_pad;
-  f.mode = 0; f.m_rows = V; f.n_rows = RK; f.ld = V; f.group_out0[0] = 0;
-  f.rows_per_b = rows_per_b; f.stride_b = logits_stride_b;
-  return tc_launch(ctx, st, s, ah, ah, bb, p, f, expert, logits, 1, JK_ST_LMHEAD);
+  int n_cta = 0;
+  int rc = tc_launch_gemm(ctx, st, s, ah, ah, bb, p, nullptr, JK_ST_LMHEAD, &n_cta);
+  if (rc != JK_OK) return rc;
+  JK_PROF(ctx, st, JK_ST_TOPK);
+  k_tc_fix_lmhead_topk<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
+      p, n_cta, V, c.k_per_expert, L.topk_chunks, (const float*)(ctx->ws + L.gemm_part), logits,
+      rows_per_b, logits_stride_b, (float*)(ctx->ws + L.tk_val), (int32_t*)(ctx->ws + L.tk_idx),
+      (float*)(ctx->ws + L.tk_ms));
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
 }
 
 // General bf16 tensor map with the 128-byte swizzle (used by the attention kernel): `rank` dims,
