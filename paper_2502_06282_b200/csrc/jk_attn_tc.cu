@@ -12,7 +12,7 @@
 //   O (+)= P V on the tensor core, V taken MN-major straight from its row-major tile; when the
 //   running max moved, O is first rescaled in tensor memory.
 // The CTA writes an unnormalised partial (max, sum, O) per row; the merge kernel of jk_attn.cu
-// combines the slices.  96 KB of shared memory and 256 tensor-memory columns per CTA, so two CTAs
+// combines the slices.  96 KB of shared memory and 256 tensor-memory columns per CTA: two CTAs
 // share an SM and overlap each other's copy and math phases.  All mbarrier waits are bounded.
 #include <math.h>
 #include <stdlib.h>
@@ -27,6 +27,7 @@ struct atc_tail {
   uint64_t bar_k, bar_v, bar_s, bar_o;
   uint32_t tmem_base;
   int abort_flag;
+  int parent[JK_MAX_TREE];
 };
 
 template <int D>
@@ -34,7 +35,8 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
     const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ kv_len,
     const int32_t* __restrict__ parent, float scale, int M, int Hq, int Hkv, int n_split,
-    int cache_rows, float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status) {
+    int n_qblk, int cache_rows, float* __restrict__ part_o, float* __restrict__ part_ml,
+    int32_t* __restrict__ counters, __nv_bfloat16* __restrict__ out, int32_t* status) {
   constexpr int KB = D / 64;                       // 64-element blocks along d
   constexpr int Q_BYTES = ATC_ROWS * D * 2;
   constexpr int KP_BYTES = 2 * ATC_ROWS * 64 * 2;  // K tile (KB blocks) or P tile (2 blocks)
@@ -66,219 +68,219 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   const int node = row_valid ? (row0 + tid) % M : 0;
   const size_t n_out = (size_t)gridDim.z * M * Hq;
   const size_t orow = ((size_t)b * M + node) * Hq + kvh * G + g_idx;
+  int32_t* counter = counters + ((size_t)b * Hkv + kvh) * n_qblk + qblk;
   const int tiles_total = (Ltot + ATC_KEYS - 1) / ATC_KEYS;
   const int tiles_per = (tiles_total + n_split - 1) / n_split;
   const int t0 = split * tiles_per;
   const int t1 = min(tiles_total, t0 + tiles_per);
-  if (t0 >= t1) {                                  // no keys in this slice
-    if (row_valid) {
-      part_ml[((size_t)split * n_out + orow) * 2] = -INFINITY;
-      part_ml[((size_t)split * n_out + orow) * 2 + 1] = 0.f;
-    }
-    return;
-  }
-
-  auto issue_kv = [&](int tile) {
-    mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
-#pragma unroll
-    for (int kb = 0; kb < KB; ++kb)
-      tma_load_4d(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k);
-    mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
-#pragma unroll
-    for (int kb = 0; kb < KB; ++kb)
-      tma_load_4d(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v);
-  };
-
-  if (tid == 0) {
-    mbar_init(&T.bar_k, 1); mbar_init(&T.bar_v, 1); mbar_init(&T.bar_s, 1); mbar_init(&T.bar_o, 1);
-    T.abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    issue_kv(t0);
-  }
-  if (warp == 0) {
-    tmem_alloc(&T.tmem_base, TMEM_COLS);
-    tmem_relinquish();
-  }
-  // Q block -> shared memory in the K-major 128-byte-swizzled layout the MMA reads
-  for (int idx = tid; idx < ATC_ROWS * (D / 8); idx += 128) {
-    const int rr = idx / (D / 8), ch = idx % (D / 8);
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row0 + rr < n_rows) {
-      const int gg = (row0 + rr) / M, ii = (row0 + rr) % M;
-      v = *reinterpret_cast<const uint4*>(q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8);
-    }
-    const int kb = ch >> 3, cb = ch & 7;
-    *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = v;
-  }
-  // ancestor set of this thread's node (Fig. 4)
-  unsigned long long anc_lo = 0ull, anc_hi = 0ull;
-  if (row_valid) {
-    int c = node;
-    for (int guard = 0; c >= 0 && guard <= JK_MAX_TREE; ++guard) {
-      if (c < 64) anc_lo |= 1ull << c; else anc_hi |= 1ull << (c - 64);
-      const int pp = parent[(size_t)b * M + c];
-      c = (pp < c) ? pp : -1;
-    }
-  }
-  fence_proxy_async_smem();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = T.tmem_base;
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-  const uint32_t idesc_s = instr_desc_bf16_ex(ATC_KEYS, 0);
-  const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
-  const float sl2 = scale * 1.4426950408889634f;
-
-  float m_run = -INFINITY, l_run = 0.f;
+  const bool have_keys = t0 < t1;
   bool ok = true;
-  for (int tile = t0; tile < t1; ++tile) {
-    const uint32_t ph = (uint32_t)(tile - t0) & 1u;
-    if (tid == 0) {
-      ok = mbar_wait(&T.bar_k, ph, abort_flag, status);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t qa = smem_u32(sq), ka = smem_u32(skp);
-#pragma unroll
-        for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            tc_mma_bf16(tmem_base, smem_desc_sw128(qa + kb * 16384 + k * 32),
-                        smem_desc_sw128(ka + kb * 16384 + k * 32), idesc_s, (kb | k) ? 1u : 0u);
-        tc_commit(&T.bar_s);
-      }
-    }
-    ok = ok && mbar_wait(&T.bar_s, ph, abort_flag, status);
-    if (!__syncthreads_and(ok)) { ok = false; break; }
-    tc_fence_after();
+  uint32_t tmem_base = 0;
+  float m_run = -INFINITY, l_run = 0.f;
 
-    // visibility of keys key0 .. key0+127 for this row: prefix keys, then the ancestor set
-    unsigned long long vis_lo = 0ull, vis_hi = 0ull;
-    if (row_valid) {
-      const int s = P - tile * ATC_KEYS;
-      if (s >= 128) { vis_lo = ~0ull; vis_hi = ~0ull; }
-      else if (s >= 0) {
-        if (s >= 64) { vis_lo = ~0ull; vis_hi = (s == 64) ? 0ull : ((1ull << (s - 64)) - 1ull); }
-        else { vis_lo = (s == 0) ? 0ull : ((1ull << s) - 1ull); }
-        unsigned long long a_lo, a_hi;
-        if (s == 0) { a_lo = anc_lo; a_hi = anc_hi; }
-        else if (s < 64) { a_lo = anc_lo << s; a_hi = (anc_hi << s) | (anc_lo >> (64 - s)); }
-        else if (s == 64) { a_lo = 0ull; a_hi = anc_lo; }
-        else { a_lo = 0ull; a_hi = anc_lo << (s - 64); }
-        vis_lo |= a_lo; vis_hi |= a_hi;
-      } else {
-        const int t = -s;
-        if (t < 64) { vis_lo = (anc_lo >> t) | (anc_hi << (64 - t)); vis_hi = anc_hi >> t; }
-        else if (t < 128) { vis_lo = anc_hi >> (t - 64); vis_hi = 0ull; }
-      }
+  if (have_keys) {
+    auto issue_kv = [&](int tile) {
+      mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
+#pragma unroll
+      for (int kb = 0; kb < KB; ++kb)
+        tma_load_4d(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k);
+      mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
+#pragma unroll
+      for (int kb = 0; kb < KB; ++kb)
+        tma_load_4d(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v);
+    };
+
+    if (tid == 0) {
+      mbar_init(&T.bar_k, 1); mbar_init(&T.bar_v, 1); mbar_init(&T.bar_s, 1); mbar_init(&T.bar_o, 1);
+      T.abort_flag = 0;
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      issue_kv(t0);
     }
-    // pass 1: row maximum over the visible keys
-    float mx = -INFINITY;
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      uint32_t r[32];
-      tmem_ld32(tmem_base + lane_base + (uint32_t)(c * 32), r);
-      tmem_ld_wait();
-      const unsigned bits = (unsigned)(((c < 2) ? vis_lo : vis_hi) >> ((c & 1) * 32));
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if ((bits >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r[j]));
+    if (warp == 0) {
+      tmem_alloc(&T.tmem_base, TMEM_COLS);
+      tmem_relinquish();
     }
-    const float m_new = fmaxf(m_run, mx);
-    const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
-                                             : fast_exp2((m_run - m_new) * sl2);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    // pass 2: P = exp(S - max) as bf16 into the K buffer, row sum
-    float lsum = 0.f;
-#pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      uint32_t r[32];
-      tmem_ld32(tmem_base + lane_base + (uint32_t)(c * 32), r);
-      tmem_ld_wait();
-      const unsigned bits = (unsigned)(((c < 2) ? vis_lo : vis_hi) >> ((c & 1) * 32));
-      uint32_t packed[16];
-#pragma unroll
-      for (int j = 0; j < 32; j += 2) {
-        const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(r[j]) - m_use) * sl2) : 0.f;
-        const float p1 = ((bits >> (j + 1)) & 1u)
-                             ? fast_exp2((__uint_as_float(r[j + 1]) - m_use) * sl2) : 0.f;
-        lsum += p0 + p1;
-        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-        packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+    if (tid < M) T.parent[tid] = parent[(size_t)b * M + tid];
+    // Q block -> shared memory in the K-major 128-byte-swizzled layout the MMA reads
+    for (int idx = tid; idx < ATC_ROWS * (D / 8); idx += 128) {
+      const int rr = idx / (D / 8), ch = idx % (D / 8);
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (row0 + rr < n_rows) {
+        const int gg = (row0 + rr) / M, ii = (row0 + rr) % M;
+        v = *reinterpret_cast<const uint4*>(q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8);
       }
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        const int ch = c * 4 + jj;               // 16-byte chunk of the 128-key row
-        const int kb = ch >> 3, cb = ch & 7;
-        *reinterpret_cast<uint4*>(skp + kb * 16384 + tid * 128 + ((cb ^ (tid & 7)) << 4)) =
-            make_uint4(packed[4 * jj], packed[4 * jj + 1], packed[4 * jj + 2], packed[4 * jj + 3]);
-      }
-    }
-    l_run = l_run * alpha + lsum;
-    m_run = m_new;
-    // rescale the running output when some row of this warp moved its maximum
-    if (tile > t0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-        tmem_st32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
-      }
-      tmem_st_wait();
+      const int kb = ch >> 3, cb = ch & 7;
+      *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = v;
     }
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
-    if (tid == 0) {
-      ok = mbar_wait(&T.bar_v, ph, abort_flag, status);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t pa = smem_u32(skp), va = smem_u32(sv);
-#pragma unroll
-        for (int j = 0; j < ATC_KEYS / 16; ++j)
-          tc_mma_bf16(tmem_base + O_COL, smem_desc_sw128(pa + (j >> 2) * 16384 + (j & 3) * 32),
-                      smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
-                      (tile > t0 || j > 0) ? 1u : 0u);
-        tc_commit(&T.bar_o);
-      }
-    }
-    ok = ok && mbar_wait(&T.bar_o, ph, abort_flag, status);
-    if (!__syncthreads_and(ok)) { ok = false; break; }
     tc_fence_after();
-    if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
-  }
-  if (ok) {
-    float* po = part_o + ((size_t)split * n_out + orow) * D;
-#pragma unroll 1
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t r[32];
-      tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
-      tmem_ld_wait();
-      if (row_valid) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 4)
-          *reinterpret_cast<float4*>(po + c * 32 + j) =
-              make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                          __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-      }
-    }
+    tmem_base = T.tmem_base;
+    // ancestor set of this thread's node (Fig. 4), walked in shared memory
+    unsigned long long anc_lo = 0ull, anc_hi = 0ull;
     if (row_valid) {
-      part_ml[((size_t)split * n_out + orow) * 2] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
-      part_ml[((size_t)split * n_out + orow) * 2 + 1] = l_run;
+      int c = node;
+      for (int guard = 0; c >= 0 && guard <= JK_MAX_TREE; ++guard) {
+        if (c < 64) anc_lo |= 1ull << c; else anc_hi |= 1ull << (c - 64);
+        const int pp = T.parent[c];
+        c = (pp < c) ? pp : -1;
+      }
     }
-  } else if (tid == 0) {
-    // gave up, possibly with copies still in flight: give them a bounded time to land
-    const unsigned long long ts = global_ns();
-    while (global_ns() - ts < 2000000ull) { /* 2 ms: far longer than any TMA copy */ }
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const uint32_t idesc_s = instr_desc_bf16_ex(ATC_KEYS, 0);
+    const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
+    const float sl2 = scale * 1.4426950408889634f;
+
+    for (int tile = t0; tile < t1; ++tile) {
+      const uint32_t ph = (uint32_t)(tile - t0) & 1u;
+      if (tid == 0) {
+        ok = mbar_wait(&T.bar_k, ph, abort_flag, status);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t qa = smem_u32(sq), ka = smem_u32(skp);
+#pragma unroll
+          for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              tc_mma_bf16(tmem_base, smem_desc_sw128(qa + kb * 16384 + k * 32),
+                          smem_desc_sw128(ka + kb * 16384 + k * 32), idesc_s, (kb | k) ? 1u : 0u);
+          tc_commit(&T.bar_s);
+        }
+      }
+      // visibility of keys key0 .. key0+127 for this row: prefix keys, then the ancestor set
+      unsigned long long vis_lo = 0ull, vis_hi = 0ull;
+      if (row_valid) {
+        const int s = P - tile * ATC_KEYS;
+        if (s >= 128) { vis_lo = ~0ull; vis_hi = ~0ull; }
+        else if (s >= 0) {
+          if (s >= 64) { vis_lo = ~0ull; vis_hi = (s == 64) ? 0ull : ((1ull << (s - 64)) - 1ull); }
+          else { vis_lo = (s == 0) ? 0ull : ((1ull << s) - 1ull); }
+          unsigned long long a_lo, a_hi;
+          if (s == 0) { a_lo = anc_lo; a_hi = anc_hi; }
+          else if (s < 64) { a_lo = anc_lo << s; a_hi = (anc_hi << s) | (anc_lo >> (64 - s)); }
+          else if (s == 64) { a_lo = 0ull; a_hi = anc_lo; }
+          else { a_lo = 0ull; a_hi = anc_lo << (s - 64); }
+          vis_lo |= a_lo; vis_hi |= a_hi;
+        } else {
+          const int t = -s;
+          if (t < 64) { vis_lo = (anc_lo >> t) | (anc_hi << (64 - t)); vis_hi = anc_hi >> t; }
+          else if (t < 128) { vis_lo = anc_hi >> (t - 64); vis_hi = 0ull; }
+        }
+      }
+      ok = ok && mbar_wait(&T.bar_s, ph, abort_flag, status);
+      if (!__syncthreads_and(ok)) { ok = false; break; }
+      tc_fence_after();
+
+      // the whole row of S in registers: one round of tensor-memory loads
+      uint32_t s0[32], s1[32], s2[32], s3[32];
+      tmem_ld32(tmem_base + lane_base + 0u, s0);
+      tmem_ld32(tmem_base + lane_base + 32u, s1);
+      tmem_ld32(tmem_base + lane_base + 64u, s2);
+      tmem_ld32(tmem_base + lane_base + 96u, s3);
+      tmem_ld_wait();
+      const unsigned b0 = (unsigned)vis_lo, b1 = (unsigned)(vis_lo >> 32);
+      const unsigned b2 = (unsigned)vis_hi, b3 = (unsigned)(vis_hi >> 32);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s0[j]));
+        if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s1[j]));
+        if ((b2 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s2[j]));
+        if ((b3 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s3[j]));
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
+                                               : fast_exp2((m_run - m_new) * sl2);
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+      float lsum = 0.f;
+      auto emit = [&](const uint32_t (&sr)[32], unsigned bits, int c) {
+        uint32_t packed[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(sr[j]) - m_use) * sl2) : 0.f;
+          const float p1 = ((bits >> (j + 1)) & 1u)
+                               ? fast_exp2((__uint_as_float(sr[j + 1]) - m_use) * sl2) : 0.f;
+          lsum += p0 + p1;
+          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+          packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const int ch = c * 4 + jj;             // 16-byte chunk of the 128-key row
+          const int kb = ch >> 3, cb = ch & 7;
+          *reinterpret_cast<uint4*>(skp + kb * 16384 + tid * 128 + ((cb ^ (tid & 7)) << 4)) =
+              make_uint4(packed[4 * jj], packed[4 * jj + 1], packed[4 * jj + 2], packed[4 * jj + 3]);
+        }
+      };
+      emit(s0, b0, 0); emit(s1, b1, 1); emit(s2, b2, 2); emit(s3, b3, 3);
+      l_run = l_run * alpha + lsum;
+      m_run = m_new;
+      // rescale the running output when some row of this warp moved its maximum
+      if (tile > t0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+          tmem_st32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+        }
+        tmem_st_wait();
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      __syncthreads();
+      if (tid == 0) {
+        ok = mbar_wait(&T.bar_v, ph, abort_flag, status);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t pa = smem_u32(skp), va = smem_u32(sv);
+#pragma unroll
+          for (int j = 0; j < ATC_KEYS / 16; ++j)
+            tc_mma_bf16(tmem_base + O_COL, smem_desc_sw128(pa + (j >> 2) * 16384 + (j & 3) * 32),
+                        smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
+                        (tile > t0 || j > 0) ? 1u : 0u);
+          tc_commit(&T.bar_o);
+        }
+      }
+      ok = ok && mbar_wait(&T.bar_o, ph, abort_flag, status);
+      if (!__syncthreads_and(ok)) { ok = false; break; }
+      tc_fence_after();
+      if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
+    }
+    if (ok) {
+      float* po = part_o + ((size_t)split * n_out + orow) * D;
+      const uint32_t lane_base2 = (uint32_t)(warp * 32) << 16;
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + lane_base2 + O_COL + (uint32_t)(c * 32), r);
+        tmem_ld_wait();
+        if (row_valid) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<float4*>(po + c * 32 + j) =
+                make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                            __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+        }
+      }
+    } else if (tid == 0) {
+      // gave up, possibly with copies still in flight: give them a bounded time to land
+      const unsigned long long ts = global_ns();
+      while (global_ns() - ts < 2000000ull) { /* 2 ms: far longer than any TMA copy */ }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+      tc_fence_after();
+      tmem_dealloc(tmem_base, TMEM_COLS);
+    }
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+  if (row_valid && ok) {
+    part_ml[((size_t)split * n_out + orow) * 2] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
+    part_ml[((size_t)split * n_out + orow) * 2 + 1] = l_run;
   }
 }
 
@@ -298,7 +300,7 @@ struct atc_state {
 };
 
 static const CUtensorMap* atc_map(jk_ctx* ctx, atc_state* s, const void* ptr, int64_t sb, int64_t sh,
-                                  int rows, int B) {
+                                  int rows) {
   for (int i = 0; i < s->n; ++i)
     if (s->e[i].ptr == ptr && s->e[i].sb == sb && s->e[i].sh == sh && s->e[i].rows == rows)
       return &s->e[i].map;
@@ -306,7 +308,7 @@ static const CUtensorMap* atc_map(jk_ctx* ctx, atc_state* s, const void* ptr, in
   atc_map_entry& e = s->e[slot];
   const jk_config& c = ctx->cfg;
   const uint64_t dims[4] = {(uint64_t)c.head_dim, (uint64_t)rows, (uint64_t)c.n_kv_heads,
-                            (uint64_t)c.max_batch > (uint64_t)B ? (uint64_t)c.max_batch : (uint64_t)B};
+                            (uint64_t)c.max_batch};
   const uint64_t strides[3] = {(uint64_t)c.head_dim * 2, (uint64_t)sh * 2, (uint64_t)sb * 2};
   const uint32_t box[4] = {64, ATC_KEYS, 1, 1};
   if (jk_tma_encode_bf16(ctx, &e.map, ptr, 4, dims, strides, box) != JK_OK) {
@@ -334,9 +336,8 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
     if (!ctx->attn_tc_state) return JK_ERR_CUDA;
   }
   atc_state* s = (atc_state*)ctx->attn_tc_state;
-  // the map's batch extent must not reach past the caller's allocation: use B
-  const CUtensorMap* mk = atc_map(ctx, s, kc, sb, sh, cache_rows, B);
-  const CUtensorMap* mv = atc_map(ctx, s, vc, sb, sh, cache_rows, B);
+  const CUtensorMap* mk = atc_map(ctx, s, kc, sb, sh, cache_rows);
+  const CUtensorMap* mv = atc_map(ctx, s, vc, sb, sh, cache_rows);
   if (!mk || !mv) return JK_ERR_CUDA;
   const int G = c.n_q_heads / c.n_kv_heads;
   const int n_qblk = (G * M + ATC_ROWS - 1) / ATC_ROWS;
@@ -351,6 +352,7 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                       sizeof(atc_tail) + 1024;
   float* part_o = (float*)(ctx->ws + L.attn_o);
   float* part_ml = (float*)(ctx->ws + L.attn_ml);
+  int32_t* counters = (int32_t*)(ctx->ws + L.attn_cnt);
   int32_t* status = (int32_t*)(ctx->ws + L.status);
   const dim3 grid(n_split * n_qblk, c.n_kv_heads, B);
   if (!s->smem_set) {
@@ -364,11 +366,13 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   if (D == 128)
     k_tree_attn_tc<128><<<grid, 128, smem, st>>>(*mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                  scale, M, c.n_q_heads, c.n_kv_heads, n_split,
-                                                 cache_rows, part_o, part_ml, status);
+                                                 n_qblk, cache_rows, part_o, part_ml, counters,
+                                                 (__nv_bfloat16*)out, status);
   else
     k_tree_attn_tc<64><<<grid, 128, smem, st>>>(*mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                 scale, M, c.n_q_heads, c.n_kv_heads, n_split,
-                                                cache_rows, part_o, part_ml, status);
+                                                n_qblk, cache_rows, part_o, part_ml, counters,
+                                                (__nv_bfloat16*)out, status);
   JK_LAUNCH_CHECK(ctx);
   return jk_attn_combine_launch(ctx, st, n_split, (size_t)B * M * c.n_q_heads, out);
 }

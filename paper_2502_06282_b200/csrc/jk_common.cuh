@@ -34,6 +34,7 @@ struct jk_ws_layout {
   size_t gemm_part;     // f32 partial tiles of the tensor-core GEMMs
   size_t attn_o;        // f32 [split, B*M*Hq, d]
   size_t attn_ml;       // f32 [split, B*M*Hq, 2]
+  size_t attn_cnt;      // i32 [B, Hkv, query blocks] arrival counters (zero between calls)
   size_t rs_arg;        // i32 [B, M]        per tree node: top-1 token of the target row
   size_t rs_max;        // f32 [B, M]
   size_t rs_sum;        // f32 [B, M]
