@@ -64,6 +64,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   const int n_rows = G * M;
   const int row0 = qblk * ATC_ROWS;
   const bool row_valid = row0 + tid < n_rows;
+  const bool warp_has_rows = row0 + (tid & ~31) < n_rows;
   const int g_idx = row_valid ? (row0 + tid) / M : 0;
   const int node = row_valid ? (row0 + tid) % M : 0;
   const size_t n_out = (size_t)gridDim.z * M * Hq;
@@ -102,15 +103,26 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
     }
     if (tid < M) T.parent[tid] = parent[(size_t)b * M + tid];
     // Q block -> shared memory in the K-major 128-byte-swizzled layout the MMA reads
-    for (int idx = tid; idx < ATC_ROWS * (D / 8); idx += 128) {
+    // (all loads are issued before the first store, so that they overlap)
+    constexpr int QV = ATC_ROWS * (D / 8) / 128;   // 16-byte vectors per thread
+    uint4 qv[QV];
+#pragma unroll
+    for (int it = 0; it < QV; ++it) {
+      const int idx = tid + it * 128;
       const int rr = idx / (D / 8), ch = idx % (D / 8);
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      qv[it] = make_uint4(0u, 0u, 0u, 0u);
       if (row0 + rr < n_rows) {
         const int gg = (row0 + rr) / M, ii = (row0 + rr) % M;
-        v = *reinterpret_cast<const uint4*>(q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8);
+        qv[it] = __ldg(reinterpret_cast<const uint4*>(
+            q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8));
       }
+    }
+#pragma unroll
+    for (int it = 0; it < QV; ++it) {
+      const int idx = tid + it * 128;
+      const int rr = idx / (D / 8), ch = idx % (D / 8);
       const int kb = ch >> 3, cb = ch & 7;
-      *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = v;
+      *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = qv[it];
     }
     fence_proxy_async_smem();
     tc_fence_before();
@@ -172,6 +184,9 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
       if (!__syncthreads_and(ok)) { ok = false; break; }
       tc_fence_after();
 
+      // (warps whose 32 rows all lie past the last query row skip the row work: their rows of P
+      // and O are never stored)
+      if (warp_has_rows) {
       // the whole row of S in registers: one round of tensor-memory loads
       uint32_t s0[32], s1[32], s2[32], s3[32];
       tmem_ld32(tmem_base + lane_base + 0u, s0);
@@ -229,6 +244,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
         }
         tmem_st_wait();
       }
+      }
       fence_proxy_async_smem();
       tc_fence_before();
       __syncthreads();
@@ -256,6 +272,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
 #pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {
         uint32_t r[32];
+        if (!warp_has_rows) break;
         tmem_ld32(tmem_base + lane_base2 + O_COL + (uint32_t)(c * 32), r);
         tmem_ld_wait();
         if (row_valid) {
