@@ -118,8 +118,12 @@ __global__ void __launch_bounds__(128) k_walk_greedy(
                 status);
 }
 
-// Sampling walk.  p and the q_r start "lazy" (read from the logits with the row's max and sum)
-// and are written out to pbuf/qbuf the first time a rejection changes them.
+// Sampling walk.  One block of 1024 threads per sequence.  p and the q_r start "lazy" (read from
+// the logits with the row's precomputed max and sum) and are written out to pbuf/qbuf the first
+// time a rejection changes them.  Every pass over the vocabulary works on 4 entries per thread
+// per step (16-byte loads; the host checks V % 4 == 0 for this mode).
+struct walk_vec4 { float v[4]; };
+
 __global__ void __launch_bounds__(1024) k_walk_sample(
     int M, int max_depth, int V, int K, int n_slots, float inv_t,
     const void* __restrict__ tl_raw, int tl_bf16, const int32_t* __restrict__ tok,
@@ -127,9 +131,11 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     const int32_t* __restrict__ branch, const int32_t* __restrict__ qslot,
     const float* __restrict__ draft_logits, const float* __restrict__ u_accept,
     const float* __restrict__ u_bonus, const float* __restrict__ rs_max,
-    const float* __restrict__ rs_sum, float* __restrict__ pbuf_all, float* __restrict__ qbuf_all,
+    const float* __restrict__ rs_sum, const float* __restrict__ qs_max,
+    const float* __restrict__ qs_sum, float* __restrict__ pbuf_all, float* __restrict__ qbuf_all,
     walk_out o, int cache_rows, int32_t* status) {
-  __shared__ float red[33];
+  __shared__ float red[66];
+  __shared__ int s_parent[JK_MAX_TREE], s_tok[JK_MAX_TREE], s_branch[JK_MAX_TREE];
   __shared__ int kids[JK_MAX_TREE];
   __shared__ int n_kids;
   __shared__ int path[16], path_tok[16];
@@ -137,18 +143,61 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
   __shared__ float scan_s[1024];
   __shared__ int s_found;
   const int b = blockIdx.x, t = threadIdx.x, nt = blockDim.x;
+  const int lane = t & 31, warp = t >> 5, nw = nt >> 5;
   float* pbuf = pbuf_all + (size_t)b * V;
   const float* tlf = (const float*)tl_raw;
   const __nv_bfloat16* tlh = (const __nv_bfloat16*)tl_raw;
+  if (t < M) {
+    s_parent[t] = parent[(size_t)b * M + t];
+    s_tok[t] = tok[(size_t)b * M + t];
+    s_branch[t] = branch[(size_t)b * M + t];
+  }
+  __syncthreads();
   int cur = 0, n = 0;
   bool p_mat = false;                 // p lives in pbuf (scaled by p_scale) instead of the logits
   float p_scale = 1.f, p_max = 0.f, p_isum = 1.f;
   size_t tl_row = 0;
-  auto tl_at = [&](size_t row, int v) -> float {
-    return tl_bf16 ? __bfloat162float(tlh[row * V + v]) : tlf[row * V + v];
-  };
   auto p_at = [&](int v) -> float {
-    return p_mat ? pbuf[v] * p_scale : expf((tl_at(tl_row, v) - p_max) * inv_t) * p_isum;
+    if (p_mat) return pbuf[v] * p_scale;
+    const float x = tl_bf16 ? __bfloat162float(tlh[tl_row * V + v]) : tlf[tl_row * V + v];
+    return expf((x - p_max) * inv_t) * p_isum;
+  };
+  auto p_at4 = [&](int v) -> walk_vec4 {           // v % 4 == 0
+    walk_vec4 r;
+    if (p_mat) {
+      const float4 x = *reinterpret_cast<const float4*>(pbuf + v);
+      r.v[0] = x.x * p_scale; r.v[1] = x.y * p_scale; r.v[2] = x.z * p_scale; r.v[3] = x.w * p_scale;
+    } else {
+      float x[4];
+      if (tl_bf16) {
+        const uint2 h = *reinterpret_cast<const uint2*>(tlh + tl_row * V + v);
+        x[0] = __uint_as_float(h.x << 16); x[1] = __uint_as_float(h.x & 0xffff0000u);
+        x[2] = __uint_as_float(h.y << 16); x[3] = __uint_as_float(h.y & 0xffff0000u);
+      } else {
+        const float4 f = *reinterpret_cast<const float4*>(tlf + tl_row * V + v);
+        x[0] = f.x; x[1] = f.y; x[2] = f.z; x[3] = f.w;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) r.v[i] = expf((x[i] - p_max) * inv_t) * p_isum;
+    }
+    return r;
+  };
+  // sum of two values over the block in one round
+  auto block_sum2 = [&](float& a, float& c) {
+    a = jk_warp_sum(a);
+    c = jk_warp_sum(c);
+    __syncthreads();
+    if (lane == 0) { red[warp] = a; red[33 + warp] = c; }
+    __syncthreads();
+    if (warp == 0) {
+      float x = lane < nw ? red[lane] : 0.f, y = lane < nw ? red[33 + lane] : 0.f;
+      x = jk_warp_sum(x);
+      y = jk_warp_sum(y);
+      if (lane == 0) { red[32] = x; red[65] = y; }
+    }
+    __syncthreads();
+    a = red[32];
+    c = red[65];
   };
   while (true) {
     tl_row = (size_t)b * M + cur;
@@ -159,7 +208,7 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     if (t == 0) {
       int c = 0;
       for (int i = 1; i < M; ++i)
-        if (parent[(size_t)b * M + i] == cur) kids[c++] = i;
+        if (s_parent[i] == cur) kids[c++] = i;
       n_kids = c;
     }
     __syncthreads();
@@ -167,33 +216,28 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     const int slot = qslot[(size_t)b * M + cur];
     int accepted = -1;
     if (nk > 0 && n < max_depth && slot >= 0 && slot < n_slots) {
-      // per-branch draft distributions: lazy (max, 1/sum) until a rejection touches them
+      // per-branch draft distributions: lazy (row max, 1/sum) until a rejection touches them
       float q_max[JK_MAX_EXPERTS], q_isum[JK_MAX_EXPERTS], q_scale[JK_MAX_EXPERTS];
       bool q_mat[JK_MAX_EXPERTS];
       for (int r = 0; r < K; ++r) {
-        const float* dl = draft_logits + (((size_t)b * n_slots + slot) * K + r) * V;
-        float mx = -INFINITY;
-        for (int v = t; v < V; v += nt) mx = fmaxf(mx, dl[v]);
-        mx = jk_block_max(mx, red);
-        float s = 0.f;
-        for (int v = t; v < V; v += nt) s += expf((dl[v] - mx) * inv_t);
-        s = jk_block_sum(s, red);
-        q_max[r] = mx; q_isum[r] = 1.f / s; q_scale[r] = 1.f; q_mat[r] = false;
+        const size_t qrow = ((size_t)b * n_slots + slot) * K + r;
+        q_max[r] = qs_max[qrow]; q_isum[r] = 1.f / qs_sum[qrow]; q_scale[r] = 1.f; q_mat[r] = false;
       }
       for (int ci = 0; ci < nk; ++ci) {
         const int c = kids[ci];
-        const int x = tok[(size_t)b * M + c];
-        int r = branch[(size_t)b * M + c];
+        const int x = s_tok[c];
+        const int r = s_branch[c];
         if (x < 0 || x >= V || r < 0 || r >= K) {
           if (t == 0) jk_set_status(status, JK_ERR_BOUNDS);
           break;
         }
         const float* dl = draft_logits + (((size_t)b * n_slots + slot) * K + r) * V;
         float* qbuf = qbuf_all + ((size_t)b * K + r) * V;
+        const bool qm = q_mat[r];
+        const float qmx = q_max[r], qis = q_isum[r], qsc = q_scale[r];
         if (t == 0) {
           const float px = p_at(x);
-          const float qx = q_mat[r] ? qbuf[x] * q_scale[r]
-                                    : expf((dl[x] - q_max[r]) * inv_t) * q_isum[r];
+          const float qx = qm ? qbuf[x] * qsc : expf((dl[x] - qmx) * inv_t) * qis;
           bool acc;
           if (qx > 0.f) acc = u_accept[(size_t)b * M + c] < fminf(1.f, px / qx);
           else acc = px > 0.f;
@@ -205,19 +249,29 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
         if (dec) { accepted = c; break; }
         // rejection: p <- max(0, p - q_r) (normalised through p_scale); q_r[x] <- 0, renormalised
         float sp = 0.f, sq = 0.f;
-        for (int v = t; v < V; v += nt) {
-          const float pv = p_at(v);
-          const float qv = q_mat[r] ? qbuf[v] * q_scale[r]
-                                    : expf((dl[v] - q_max[r]) * inv_t) * q_isum[r];
-          const float res = fmaxf(0.f, pv - qv);
-          const float qn = (v == x) ? 0.f : qv;
-          pbuf[v] = res;
-          qbuf[v] = qn;
-          sp += res;
-          sq += qn;
+#pragma unroll 2
+        for (int v = t * 4; v < V; v += nt * 4) {
+          const walk_vec4 pv = p_at4(v);
+          float qv[4];
+          const float4 qr = *reinterpret_cast<const float4*>((qm ? qbuf : dl) + v);
+          if (qm) {
+            qv[0] = qr.x * qsc; qv[1] = qr.y * qsc; qv[2] = qr.z * qsc; qv[3] = qr.w * qsc;
+          } else {
+            qv[0] = expf((qr.x - qmx) * inv_t) * qis; qv[1] = expf((qr.y - qmx) * inv_t) * qis;
+            qv[2] = expf((qr.z - qmx) * inv_t) * qis; qv[3] = expf((qr.w - qmx) * inv_t) * qis;
+          }
+          float res[4], qn[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            res[i] = fmaxf(0.f, pv.v[i] - qv[i]);
+            qn[i] = (v + i == x) ? 0.f : qv[i];
+            sp += res[i];
+            sq += qn[i];
+          }
+          *reinterpret_cast<float4*>(pbuf + v) = make_float4(res[0], res[1], res[2], res[3]);
+          *reinterpret_cast<float4*>(qbuf + v) = make_float4(qn[0], qn[1], qn[2], qn[3]);
         }
-        sp = jk_block_sum(sp, red);
-        sq = jk_block_sum(sq, red);
+        block_sum2(sp, sq);
         q_mat[r] = true;
         q_scale[r] = sq > 0.f ? 1.f / sq : 1.f;
         if (!(sp > 0.f)) {            // residual vanished: keep the node's own p for the bonus
@@ -229,19 +283,23 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
       }
     }
     if (accepted >= 0) {
-      if (t == 0) { path[n] = accepted; path_tok[n] = tok[(size_t)b * M + accepted]; }
+      if (t == 0) { path[n] = accepted; path_tok[n] = s_tok[accepted]; }
       ++n;
       cur = accepted;
       __syncthreads();
       continue;
     }
-    // bonus token: inverse CDF of the current p at u_bonus[depth]
+    // bonus token: inverse CDF of the current p at u_bonus[depth]; every thread owns a contiguous
+    // run of `per` entries (a multiple of 4)
     const int dcur = depth[(size_t)b * M + cur];
     const float ub = u_bonus[(size_t)b * (max_depth + 1) + min(max(dcur, 0), max_depth)];
-    const int per = (V + nt - 1) / nt;
-    const int v0 = t * per, v1 = min(V, v0 + per);
+    const int per = ((V + nt - 1) / nt + 3) / 4 * 4;
+    const int v0 = min(V, t * per), v1 = min(V, v0 + per);
     float loc = 0.f;
-    for (int v = v0; v < v1; ++v) loc += p_at(v);
+    for (int v = v0; v < v1; v += 4) {
+      const walk_vec4 pv = p_at4(v);
+      loc += (pv.v[0] + pv.v[1]) + (pv.v[2] + pv.v[3]);
+    }
     scan_s[t] = loc;
     if (t == 0) s_found = INT_MAX;
     __syncthreads();
@@ -253,10 +311,13 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     }
     const float total = scan_s[nt - 1];
     const float thr = ub * total;
-    float run = scan_s[t] - loc;
-    for (int v = v0; v < v1; ++v) {
-      run += p_at(v);
-      if (run > thr) { atomicMin(&s_found, v); break; }
+    const float before = scan_s[t] - loc;
+    if (before <= thr && scan_s[t] > thr) {          // the crossing lies in this thread's run
+      float run = before;
+      for (int v = v0; v < v1; ++v) {
+        run += p_at(v);
+        if (run > thr) { atomicMin(&s_found, v); break; }
+      }
     }
     __syncthreads();
     if (s_found == INT_MAX) {            // rounding left no bin: last token with p > 0
@@ -320,6 +381,8 @@ extern "C" int jk_accept_and_compact(
   if (mode != 0 && mode != 1) return JK_ERR_SHAPE;
   if (mode == 1 && (!draft_logits || !u_accept || !u_bonus)) return JK_ERR_NULL;
   if (mode == 1 && (!(temperature > 0.f) || n_slots < 1)) return JK_ERR_SHAPE;
+  if (mode == 1 && n_slots > ctx->cfg.max_depth * ctx->cfg.max_frontier) return JK_ERR_CAPACITY;
+  if (mode == 1 && ctx->cfg.vocab % 4) return JK_ERR_ALIGN;      // 16-byte rows of draft logits
   if (n_layers < 0 || (n_layers > 0 && (!k_caches || !v_caches))) return JK_ERR_NULL;
   if (tl_dtype != JK_F32 && tl_dtype != JK_BF16) return JK_ERR_DTYPE;
   const jk_config& c = ctx->cfg;
@@ -351,6 +414,14 @@ extern "C" int jk_accept_and_compact(
     k_row_stats<float><<<rows, 512, 0, st>>>((const float*)target_logits, c.vocab, inv_t, rs_arg,
                                              rs_max, rs_sum);
   JK_LAUNCH_CHECK(ctx);
+  if (mode == 1) {
+    // max and sum of exp of every stored draft row, in parallel, before the serial walk
+    JK_PROF(ctx, st, JK_ST_ROWSTATS);
+    k_row_stats<float><<<batch * n_slots * c.top_k, 512, 0, st>>>(
+        draft_logits, c.vocab, inv_t, (int32_t*)(ws + L.qs_arg), (float*)(ws + L.qs_max),
+        (float*)(ws + L.qs_sum));
+    JK_LAUNCH_CHECK(ctx);
+  }
   walk_out o{kv_len, (int32_t*)(ws + L.p_old), n_acc, acc_idx, acc_tok, bonus_tok};
   JK_PROF(ctx, st, JK_ST_WALK);
   if (mode == 0) {
@@ -360,7 +431,8 @@ extern "C" int jk_accept_and_compact(
     k_walk_sample<<<batch, 1024, 0, st>>>(
         tree_size, c.max_depth, c.vocab, c.top_k, n_slots, inv_t, target_logits,
         tl_dtype == JK_BF16, tok, parent, depth, branch, qslot, draft_logits, u_accept, u_bonus,
-        rs_max, rs_sum, (float*)(ws + L.pbuf), (float*)(ws + L.qbuf), o, cache_rows, status);
+        rs_max, rs_sum, (const float*)(ws + L.qs_max), (const float*)(ws + L.qs_sum),
+        (float*)(ws + L.pbuf), (float*)(ws + L.qbuf), o, cache_rows, status);
   }
   JK_LAUNCH_CHECK(ctx);
   if (n_layers > 0) {

@@ -71,6 +71,10 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->pbuf = take((size_t)c.max_batch * c.vocab * 4);
   L->qbuf = take((size_t)c.max_batch * c.top_k * c.vocab * 4);
   L->p_old = take((size_t)c.max_batch * 4);
+  const size_t qrows = (size_t)c.max_batch * c.max_depth * c.max_frontier * c.top_k;
+  L->qs_arg = take(qrows * 4);
+  L->qs_max = take(qrows * 4);
+  L->qs_sum = take(qrows * 4);
   L->total = off;
 }
 

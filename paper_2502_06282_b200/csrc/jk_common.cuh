@@ -41,6 +41,9 @@ struct jk_ws_layout {
   size_t pbuf;          // f32 [B, V]
   size_t qbuf;          // f32 [B, K, V]
   size_t p_old;         // i32 [B]
+  size_t qs_arg;        // i32 [B, S, K]     (unused top-1 of the draft rows)
+  size_t qs_max;        // f32 [B, S, K]     max of every stored draft logits row
+  size_t qs_sum;        // f32 [B, S, K]     its sum of exp((x - max)/T)
   size_t total;
   int attn_max_split;
   int topk_chunks;
