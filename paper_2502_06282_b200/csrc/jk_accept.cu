@@ -15,6 +15,8 @@ __global__ void __launch_bounds__(512) k_row_stats(const TL* __restrict__ tl, in
                                                    int32_t* __restrict__ rs_arg,
                                                    float* __restrict__ rs_max,
                                                    float* __restrict__ rs_sum) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   constexpr int VN = jk_vec<TL>::N;
   __shared__ float red[33];
   __shared__ float wv[16];
@@ -93,6 +95,8 @@ __global__ void __launch_bounds__(128) k_walk_greedy(
     int M, int max_depth, int V, const int32_t* __restrict__ tok,
     const int32_t* __restrict__ parent, const int32_t* __restrict__ rs_arg, walk_out o,
     int cache_rows, int32_t* status) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   __shared__ int s_next;
   __shared__ int path[16], path_tok[16];
   const int b = blockIdx.x;
@@ -134,6 +138,8 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     const float* __restrict__ rs_sum, const float* __restrict__ qs_max,
     const float* __restrict__ qs_sum, float* __restrict__ pbuf_all, float* __restrict__ qbuf_all,
     walk_out o, int cache_rows, int32_t* status) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   __shared__ float red[66];
   __shared__ int s_parent[JK_MAX_TREE], s_tok[JK_MAX_TREE], s_branch[JK_MAX_TREE];
   __shared__ int kids[JK_MAX_TREE];
@@ -343,6 +349,8 @@ __global__ void __launch_bounds__(256) k_compact(
     long long stride_b, long long stride_h, int row_bytes, int cache_rows, int max_depth, int M,
     const int32_t* __restrict__ p_old, const int32_t* __restrict__ n_acc,
     const int32_t* __restrict__ acc_idx, int elem_size) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   const int which = blockIdx.z;                  // layer*2 + (0 = K, 1 = V)
   const int b = blockIdx.y, kvh = blockIdx.x;
   const int n = n_acc[b];
@@ -408,16 +416,16 @@ extern "C" int jk_accept_and_compact(
   const int rows = batch * tree_size;
   JK_PROF(ctx, st, JK_ST_ROWSTATS);
   if (tl_dtype == JK_BF16)
-    k_row_stats<__nv_bfloat16><<<rows, 512, 0, st>>>((const __nv_bfloat16*)target_logits, c.vocab,
+    jk_launch_pdl(k_row_stats<__nv_bfloat16>, dim3(rows), dim3(512), 0, st, (const __nv_bfloat16*)target_logits, c.vocab,
                                                      inv_t, rs_arg, rs_max, rs_sum);
   else
-    k_row_stats<float><<<rows, 512, 0, st>>>((const float*)target_logits, c.vocab, inv_t, rs_arg,
+    jk_launch_pdl(k_row_stats<float>, dim3(rows), dim3(512), 0, st, (const float*)target_logits, c.vocab, inv_t, rs_arg,
                                              rs_max, rs_sum);
   JK_LAUNCH_CHECK(ctx);
   if (mode == 1) {
     // max and sum of exp of every stored draft row, in parallel, before the serial walk
     JK_PROF(ctx, st, JK_ST_ROWSTATS);
-    k_row_stats<float><<<batch * n_slots * c.top_k, 512, 0, st>>>(
+    jk_launch_pdl(k_row_stats<float>, dim3(batch * n_slots * c.top_k), dim3(512), 0, st, 
         draft_logits, c.vocab, inv_t, (int32_t*)(ws + L.qs_arg), (float*)(ws + L.qs_max),
         (float*)(ws + L.qs_sum));
     JK_LAUNCH_CHECK(ctx);
@@ -425,10 +433,10 @@ extern "C" int jk_accept_and_compact(
   walk_out o{kv_len, (int32_t*)(ws + L.p_old), n_acc, acc_idx, acc_tok, bonus_tok};
   JK_PROF(ctx, st, JK_ST_WALK);
   if (mode == 0) {
-    k_walk_greedy<<<batch, 128, 0, st>>>(tree_size, c.max_depth, c.vocab, tok, parent, rs_arg, o,
+    jk_launch_pdl(k_walk_greedy, dim3(batch), dim3(128), 0, st, tree_size, c.max_depth, c.vocab, tok, parent, rs_arg, o,
                                          cache_rows, status);
   } else {
-    k_walk_sample<<<batch, 1024, 0, st>>>(
+    jk_launch_pdl(k_walk_sample, dim3(batch), dim3(1024), 0, st, 
         tree_size, c.max_depth, c.vocab, c.top_k, n_slots, inv_t, target_logits,
         tl_dtype == JK_BF16, tok, parent, depth, branch, qslot, draft_logits, u_accept, u_bonus,
         rs_max, rs_sum, (const float*)(ws + L.qs_max), (const float*)(ws + L.qs_sum),
@@ -437,7 +445,7 @@ extern "C" int jk_accept_and_compact(
   JK_LAUNCH_CHECK(ctx);
   if (n_layers > 0) {
     JK_PROF(ctx, st, JK_ST_COMPACT);
-    k_compact<<<dim3(c.n_kv_heads, batch, 2 * n_layers), 256, 0, st>>>(
+    jk_launch_pdl(k_compact, dim3(c.n_kv_heads, batch, 2 * n_layers), dim3(256), 0, st, 
         k_caches, v_caches, n_layers, cache_stride_b, cache_stride_h, row_bytes, cache_rows,
         c.max_depth, tree_size, (const int32_t*)(ws + L.p_old), n_acc, acc_idx, es);
     JK_LAUNCH_CHECK(ctx);

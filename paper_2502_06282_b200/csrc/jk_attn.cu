@@ -149,6 +149,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256) k_attn_combine(
     const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_split,
     size_t n_out, T* __restrict__ out) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   constexpr int DPL = D / 32;
   const int lane = threadIdx.x & 31;
   const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);

@@ -55,6 +55,8 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   const int kvh = blockIdx.y, b = blockIdx.z;
   const int G = Hq / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5;
+  jk_pdl_wait();
+  jk_pdl_trigger();
   const int P = kv_len[b];
   const int Ltot = P + M;
   if (P < 0 || Ltot > cache_rows) {
@@ -381,12 +383,12 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   }
   JK_PROF(ctx, st, JK_ST_ATTN);
   if (D == 128)
-    k_tree_attn_tc<128><<<grid, 128, smem, st>>>(*mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+    jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(128), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                  scale, M, c.n_q_heads, c.n_kv_heads, n_split,
                                                  n_qblk, cache_rows, part_o, part_ml, counters,
                                                  (__nv_bfloat16*)out, status);
   else
-    k_tree_attn_tc<64><<<grid, 128, smem, st>>>(*mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+    jk_launch_pdl(k_tree_attn_tc<64>, dim3(grid), dim3(128), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                 scale, M, c.n_q_heads, c.n_kv_heads, n_split,
                                                 n_qblk, cache_rows, part_o, part_ml, counters,
                                                 (__nv_bfloat16*)out, status);

@@ -115,6 +115,33 @@ static inline bool jk_aligned16(const void* p) { return (reinterpret_cast<uintpt
 int jk_ensure_device_info(jk_ctx* ctx);
 
 #ifdef __CUDACC__
+// ---------------------------------------------------------------- programmatic dependent launch
+// The kernels of one call form a chain on one stream.  Launched with the programmatic-
+// serialization attribute, a kernel may start while its predecessor is still running; it must
+// call jk_pdl_wait() before it reads or writes global memory that an earlier kernel of the
+// stream touches, and it calls jk_pdl_trigger() only after that wait, so that at most two
+// consecutive kernels overlap and everything older is complete when a kernel starts.
+__device__ __forceinline__ void jk_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void jk_pdl_trigger() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t jk_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                                        size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------- device helpers
 __device__ __forceinline__ float jk_warp_sum(float v) {
 #pragma unroll

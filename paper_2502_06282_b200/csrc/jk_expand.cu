@@ -26,6 +26,8 @@ __global__ void __launch_bounds__(512) k_router(
     const T* __restrict__ u, const T* __restrict__ router, const T* __restrict__ norm_w,
     int H, int N, int K, float eps, int use_norm, T* __restrict__ xn,
     float* __restrict__ out_probs, int32_t* __restrict__ out_expert, float* __restrict__ out_gate) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   // One pass over the row: the sum of squares and the N centroid dot products of u * gamma are
   // accumulated together (the RMS factor is a scalar, applied to the dots afterwards).
   constexpr int VN = jk_vec<T>::N;
@@ -305,6 +307,8 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
     const int32_t* __restrict__ parent_gidx, int gidx_base, int slot_base,
     jk_pool pool, float* __restrict__ out_lse, int32_t* __restrict__ next_frontier,
     float* __restrict__ next_parent_score, int32_t* __restrict__ next_parent_gidx) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   constexpr int PER_MAX = 16;                   // candidates per lane held in registers
   __shared__ float sc[JK_MAX_POOL];
   const int b = blockIdx.x;
@@ -390,6 +394,8 @@ __global__ void __launch_bounds__(1024) k_tree_finalize(
     int32_t* __restrict__ tok, int32_t* __restrict__ parent, int32_t* __restrict__ depth,
     int32_t* __restrict__ branch, int32_t* __restrict__ qslot, unsigned long long* __restrict__ anc,
     int32_t* status) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   __shared__ float sc[JK_MAX_POOL];
   __shared__ short newid[JK_MAX_POOL];      // 0 = dropped, else node index
   __shared__ int par_s[JK_MAX_TREE];
@@ -486,7 +492,7 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
   const long long lsb = (out_logits && logits_stride_b) ? logits_stride_b : (long long)rows_per_b * V;
 
   JK_PROF(ctx, st, JK_ST_ROUTER);
-  k_router<T><<<R, 512, 0, st>>>((const T*)u, (const T*)w->router, (const T*)w->norm_weight, H,
+  jk_launch_pdl(k_router<T>, dim3(R), dim3(512), 0, st, (const T*)u, (const T*)w->router, (const T*)w->norm_weight, H,
                                  c.n_experts, K, c.rms_eps, c.use_pre_norm, xn, out_probs,
                                  out_expert, out_gate);
   JK_LAUNCH_CHECK(ctx);
@@ -520,7 +526,7 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
     JK_LAUNCH_CHECK(ctx);
   }
   JK_PROF(ctx, st, JK_ST_FINISH);
-  k_expand_finish<<<B, 1024, 0, st>>>(F, K, c.k_per_expert, L.topk_chunks, width,
+  jk_launch_pdl(k_expand_finish, dim3(B), dim3(1024), 0, st, F, K, c.k_per_expert, L.topk_chunks, width,
                                      (const float*)(ws + L.tk_val),
                                      (const int32_t*)(ws + L.tk_idx),
                                      (const float*)(ws + L.tk_ms), parent_score, parent_gidx,
@@ -590,7 +596,7 @@ extern "C" int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const 
   if (!ctx->ws) return JK_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   JK_PROF(ctx, st, JK_ST_FINALIZE);
-  k_tree_finalize<<<batch, 1024, 0, st>>>(
+  jk_launch_pdl(k_tree_finalize, dim3(batch), dim3(1024), 0, st, 
       *pool, pool_n, root_tok, tree_size, tok, parent, depth, branch, qslot,
       (unsigned long long*)anc, (int32_t*)(ctx->ws + ctx->lay.status));
   JK_LAUNCH_CHECK(ctx);

@@ -43,6 +43,7 @@ struct tc_params {
   int max_seg;                       // partial slots per CTA
   int R, K_top, n_experts;           // to derive the active experts from `expert`
   int tmem_cols;
+  int prefetch;                      // 1: the producer streams weight tiles before the grid-dependency wait
 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
@@ -114,6 +115,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
     T.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // The plan reads the router's output.  Without prefetch the preceding kernel may be the
+  // router itself, so wait for it first; with prefetch the router is at least two kernels back
+  // and therefore complete (a kernel releases its successor only after its own wait).
+  if (!p.prefetch) jk_pdl_wait();
   if (warp == 0) {
     __syncwarp();
     tc_make_plan(p, expert, &T.plan);
@@ -131,43 +136,76 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
   const long long u1 = tc_span_start(total, blockIdx.x + 1, gridDim.x);
   const int units_per_tile = p.kt;
   const long long first_tile = u0 / units_per_tile;
+  if (!(p.prefetch && warp == 0 && lane == 0)) {
+    jk_pdl_wait();                      // (the prefetching producer waits after its first ring)
+    jk_pdl_trigger();
+  }
 
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
     int issued = 0;
     bool ok = true;
-    // position of the span's first unit; advanced incrementally (no divisions in the loop)
-    int kt = (int)(u0 % units_per_tile);
-    int t = (int)(first_tile % p.tiles_per_group);
-    int gi = (int)(first_tile / p.tiles_per_group);
-    int g = (u0 < u1) ? T.plan.group_src[gi] : 0;
-    const CUtensorMap* ma = p.group_amap[g] ? &map_a1 : &map_a0;
-    int arow = p.group_arow0[g] + t * TC_TILE_M, brow = p.group_brow0[g];
+    const int n_units = (int)(u1 - u0);
+    // position of a unit of the span, advanced incrementally (no divisions in the loop)
+    struct cursor {
+      int kt, t, gi, g, arow, brow;
+      const CUtensorMap* ma;
+    };
+    auto cur_load = [&](cursor& c) {
+      c.g = T.plan.group_src[c.gi];
+      c.ma = p.group_amap[c.g] ? &map_a1 : &map_a0;
+      c.brow = p.group_brow0[c.g];
+      c.arow = p.group_arow0[c.g] + c.t * TC_TILE_M;
+    };
+    auto cur_next = [&](cursor& c, bool more) {
+      if (++c.kt == units_per_tile) {
+        c.kt = 0;
+        if (++c.t == p.tiles_per_group) {
+          c.t = 0;
+          ++c.gi;
+          if (more) cur_load(c);
+        }
+        c.arow = p.group_arow0[c.g] + c.t * TC_TILE_M;
+      }
+    };
+    cursor ca;
+    ca.kt = (int)(u0 % units_per_tile);
+    ca.t = (int)(first_tile % p.tiles_per_group);
+    ca.gi = (int)(first_tile / p.tiles_per_group);
+    ca.g = 0; ca.arow = 0; ca.brow = 0; ca.ma = &map_a0;
+    if (n_units > 0) cur_load(ca);
     int s = 0;
     uint32_t ph = 0;
-    const int n_units = (int)(u1 - u0);
+    if (p.prefetch) {
+      // The weights do not depend on the kernel that runs before this one: start streaming the
+      // first ring of weight tiles now, and add the activation tiles once that kernel is done.
+      const int npre = n_units < p.stages ? n_units : p.stages;
+      cursor cb = ca;
+      for (int i = 0; i < npre; ++i) {
+        mbar_expect_tx(&T.full[i], (uint32_t)stage_bytes);
+        tma_load_2d(smem + (size_t)i * stage_bytes, ca.ma, ca.kt * TC_TILE_K, ca.arow, &T.full[i]);
+        cur_next(ca, i + 1 < n_units);
+      }
+      jk_pdl_wait();
+      jk_pdl_trigger();
+      for (int i = 0; i < npre; ++i) {
+        tma_load_2d(smem + (size_t)i * stage_bytes + TC_TILE_M * TC_TILE_K * 2, &map_b,
+                    cb.kt * TC_TILE_K, cb.brow, &T.full[i]);
+        cur_next(cb, i + 1 < n_units);
+      }
+      issued = npre;
+      if (npre == p.stages) { s = 0; ph = 1u; } else { s = npre; }
+    }
     for (; issued < n_units; ++issued) {
       if (issued >= p.stages) ok = mbar_wait(&T.empty[s], ph ^ 1u, abort_flag, status);
       if (!ok) break;
       unsigned char* sa = smem + (size_t)s * stage_bytes;
       unsigned char* sb = sa + TC_TILE_M * TC_TILE_K * 2;
       mbar_expect_tx(&T.full[s], (uint32_t)stage_bytes);
-      tma_load_2d(sa, ma, kt * TC_TILE_K, arow, &T.full[s]);
-      tma_load_2d(sb, &map_b, kt * TC_TILE_K, brow, &T.full[s]);
+      tma_load_2d(sa, ca.ma, ca.kt * TC_TILE_K, ca.arow, &T.full[s]);
+      tma_load_2d(sb, &map_b, ca.kt * TC_TILE_K, ca.brow, &T.full[s]);
       if (++s == p.stages) { s = 0; ph ^= 1u; }
-      if (++kt == units_per_tile) {
-        kt = 0;
-        if (++t == p.tiles_per_group) {
-          t = 0;
-          ++gi;
-          if (issued + 1 < n_units) {
-            g = T.plan.group_src[gi];
-            ma = p.group_amap[g] ? &map_a1 : &map_a0;
-            brow = p.group_brow0[g];
-          }
-        }
-        arow = p.group_arow0[g] + t * TC_TILE_M;
-      }
+      cur_next(ca, issued + 1 < n_units);
     }
     if (!ok) {
       // gave up: let the copies already in flight land before the CTA's memory goes away
@@ -259,22 +297,34 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
 
 // Partial-tile slots that add up to `tile`, ascending CTA order.  Returns the count, or -1 if
 // there are more than TC_MAX_CONTRIB (then tc_tile_sum_slow is used).
-__device__ __forceinline__ int tc_tile_slots(const tc_params& p, long long total, int n_cta,
+__device__ __forceinline__ int tc_tile_slots(const tc_params& p, long long total64, int n_cta,
                                              long long tile, int* slots) {
-  const long long a = tile * p.kt, b = a + p.kt;
-  int c = (int)(a * n_cta / total);
-  while (c + 1 < n_cta && tc_span_start(total, c + 1, n_cta) <= a) ++c;
-  while (c > 0 && tc_span_start(total, c, n_cta) > a) --c;
-  int n = 0;
-  for (; c < n_cta; ++c) {
-    const long long s0 = tc_span_start(total, c, n_cta);
-    if (s0 >= b) break;
-    const long long s1 = tc_span_start(total, c + 1, n_cta);
-    if (s1 <= a || s1 == s0) continue;                        // before the tile, or empty
-    if (n == TC_MAX_CONTRIB) return -1;
-    slots[n++] = c * p.max_seg + (int)(tile - s0 / p.kt);
+  // 32-bit arithmetic (the host checks total * n_cta < 2^31); span starts are stepped from one
+  // CTA to the next with a quotient/remainder pair instead of one division each.
+  const unsigned total = (unsigned)total64, n = (unsigned)n_cta, kt = (unsigned)p.kt;
+  const unsigned a = (unsigned)tile * kt, b = a + kt;
+  const unsigned q = total / n, r = total - q * n;          // start(c + 1) - start(c) = q or q + 1
+  unsigned c = a * n / total;
+  if (c >= n) c = n - 1;
+  unsigned s0 = total * c / n, rem = total * c - s0 * n;     // start(c) and its remainder
+  // step back while this CTA starts after a
+  while (c > 0 && s0 > a) {
+    --c;
+    if (rem >= r) { rem -= r; s0 -= q; } else { rem = rem + n - r; s0 -= q + 1; }
   }
-  return n;
+  int cnt = 0;
+  for (; c < n; ++c) {
+    if (s0 >= b) break;
+    unsigned s1 = s0 + q, rem1 = rem + r;
+    if (rem1 >= n) { rem1 -= n; ++s1; }
+    if (s1 > a && s1 != s0) {                                 // overlaps the tile and is not empty
+      if (cnt == TC_MAX_CONTRIB) return -1;
+      slots[cnt++] = (int)(c * (unsigned)p.max_seg + ((unsigned)tile - s0 / kt));
+    }
+    s0 = s1;
+    rem = rem1;
+  }
+  return cnt;
 }
 
 __device__ __forceinline__ float tc_tile_sum_slow(const float* __restrict__ partial,
@@ -316,6 +366,8 @@ __global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int n_ct
                                                      int Rp, const int32_t* __restrict__ expert,
                                                      const float* __restrict__ partial,
                                                      __nv_bfloat16* __restrict__ hbuf) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   __shared__ tc_plan plan;
   __shared__ tc_slot_list lg, lu;
   if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
@@ -347,6 +399,8 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
     const float* __restrict__ gate, const __nv_bfloat16* __restrict__ u, int branch_residual,
     const float* __restrict__ partial, __nv_bfloat16* __restrict__ bbuf,
     __nv_bfloat16* __restrict__ out_feat) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   __shared__ tc_plan plan;
   __shared__ tc_slot_list lists[JK_MAX_EXPERTS];
   __shared__ long long tiles[JK_MAX_EXPERTS];
@@ -383,6 +437,8 @@ __global__ void __launch_bounds__(256) k_tc_fix_lmhead_topk(
     const tc_params p, int n_cta, int V, int k_e, int chunks, const float* __restrict__ partial,
     float* __restrict__ logits, int rows_per_b, long long stride_b, float* __restrict__ tk_val,
     int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
   constexpr int TILES = JK_TOPK_CHUNK / TC_TILE_M;     // 32 tiles per chunk
   __shared__ tc_slot_list lists[TILES];
   const int chunk = blockIdx.x, row = blockIdx.y;
@@ -544,6 +600,7 @@ static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUten
   p.stages = tc_stages(p.n_pad);
   const long long max_units = (long long)p.n_groups_max * p.tiles_per_group * p.kt;
   p.max_seg = tc_max_seg(max_units, n_cta, p.kt);
+  if (max_units * TC_MAX_GRID >= (1ll << 31)) return JK_ERR_SHAPE;   // 32-bit span arithmetic
   int cols = 32;
   while (cols < 2 * p.n_pad) cols <<= 1;
   p.tmem_cols = cols;
@@ -556,7 +613,7 @@ static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUten
     s->smem_set = 1;
   }
   JK_PROF(ctx, st, stage_id);
-  k_tc_gemm<<<n_cta, TC_THREADS, smem, st>>>(*a0, *a1, *b, p, expert,
+  jk_launch_pdl(k_tc_gemm, dim3(n_cta), dim3(TC_THREADS), smem, st, *a0, *a1, *b, p, expert,
                                              (float*)(ctx->ws + L.gemm_part),
                                              (int32_t*)(ctx->ws + L.status));
   JK_LAUNCH_CHECK(ctx);
@@ -602,7 +659,7 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   int rc = tc_launch_gemm(ctx, st, s, ag, au, bx, p, expert, JK_ST_GATEUP, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_GEMM_FIXUP);
-  k_tc_fix_silu<<<dim3(p.tiles_per_group, N, tc_zdim(p.tiles_per_group * N, R, n_cta)), 128, 0, st>>>(
+  jk_launch_pdl(k_tc_fix_silu, dim3(p.tiles_per_group, N, tc_zdim(p.tiles_per_group * N, R, n_cta)), dim3(128), 0, st, 
       p, n_cta, I, R, Rp, expert, partial, (__nv_bfloat16*)(ctx->ws + L.hbuf));
   JK_LAUNCH_CHECK(ctx);
   // down
@@ -615,10 +672,11 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   }
   p.tiles_per_group = (H + TC_TILE_M - 1) / TC_TILE_M;
   p.kt = (I + TC_TILE_K - 1) / TC_TILE_K;
+  p.prefetch = 1;
   rc = tc_launch_gemm(ctx, st, s, ad, ad, bh, p, expert, JK_ST_DOWN, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_BRANCH);
-  k_tc_fix_down_branch<<<dim3(p.tiles_per_group, R), 128, 0, st>>>(
+  jk_launch_pdl(k_tc_fix_down_branch, dim3(p.tiles_per_group, R), dim3(128), 0, st, 
       p, n_cta, H, expert, gate, (const __nv_bfloat16*)u, c.branch_residual, partial,
       (__nv_bfloat16*)(ctx->ws + L.bbuf), (__nv_bfloat16*)out_feat);
   JK_LAUNCH_CHECK(ctx);
@@ -647,10 +705,11 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
   p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
   p.n_pad = n_pad;
   int n_cta = 0;
+  p.prefetch = 1;
   int rc = tc_launch_gemm(ctx, st, s, ah, ah, bb, p, nullptr, JK_ST_LMHEAD, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_TOPK);
-  k_tc_fix_lmhead_topk<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
+  jk_launch_pdl(k_tc_fix_lmhead_topk, dim3(L.topk_chunks, RK), dim3(256), 0, st, 
       p, n_cta, V, c.k_per_expert, L.topk_chunks, (const float*)(ctx->ws + L.gemm_part), logits,
       rows_per_b, logits_stride_b, (float*)(ctx->ws + L.tk_val), (int32_t*)(ctx->ws + L.tk_idx),
       (float*)(ctx->ws + L.tk_ms));

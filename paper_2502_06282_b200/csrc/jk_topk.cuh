@@ -2,6 +2,9 @@
 // chunk maximum, sum of exp(x - max) and the k_e best (value descending, token id ascending).
 // Shared by the CUDA-core path (logits read from global memory) and the tensor-core path (logits
 // assembled from the GEMM's partial tiles).
+//
+// Every warp first picks the k_e best of its own 512 entries with shuffles only; warp 0 then
+// merges the 8 * k_e warp winners.  Two block barriers in total.
 #pragma once
 
 #include <limits.h>
@@ -11,62 +14,92 @@
 
 #define JK_TOPK_PER (JK_TOPK_CHUNK / 256)
 
+__device__ __forceinline__ void jk_warp_argbest(float& v, int& i) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+    if (jk_better(ov, oi, v, i)) { v = ov; i = oi; }
+  }
+}
+
 // 256 threads; thread t holds entries base + t + j*256 in vals[j] (-inf past the vocabulary).
 __device__ __forceinline__ void jk_topk_chunk_select(const float (&vals)[JK_TOPK_PER], int base,
                                                      int V, int k_e, size_t prow,
                                                      float* __restrict__ tk_val,
                                                      int32_t* __restrict__ tk_idx,
                                                      float* __restrict__ tk_ms) {
-  __shared__ float red[33];
-  __shared__ float wv[8];
-  __shared__ int wi[8];
-  __shared__ int win_idx;
+  __shared__ float s_wmax[8], s_wsum[8];
+  __shared__ float s_cv[8 * JK_MAX_KE];
+  __shared__ int s_ci[8 * JK_MAX_KE];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // warp maximum and the warp's own k_e best
   float lmax = -INFINITY;
 #pragma unroll
   for (int j = 0; j < JK_TOPK_PER; ++j) lmax = fmaxf(lmax, vals[j]);
-  const float bmax = jk_block_max(lmax, red);
+  lmax = jk_warp_max(lmax);
+  unsigned taken = 0;
+  for (int it = 0; it < k_e; ++it) {
+    float bv = -INFINITY;
+    int bi = INT_MAX, bj = -1;
+#pragma unroll
+    for (int j = 0; j < JK_TOPK_PER; ++j) {
+      const int idx = base + threadIdx.x + j * 256;
+      if (!(taken & (1u << j)) && idx < V && jk_better(vals[j], idx, bv, bi)) {
+        bv = vals[j]; bi = idx; bj = j;
+      }
+    }
+    float wv = bv;
+    int wi = bi;
+    jk_warp_argbest(wv, wi);
+    if (wi == bi && bj >= 0) taken |= 1u << bj;       // token ids are unique: one lane matches
+    if (lane == 0) { s_cv[warp * JK_MAX_KE + it] = wv; s_ci[warp * JK_MAX_KE + it] = wi; }
+  }
+  if (lane == 0) s_wmax[warp] = lmax;
+  __syncthreads();
+  float bmax = s_wmax[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) bmax = fmaxf(bmax, s_wmax[w]);
   float s = 0.f;
 #pragma unroll
   for (int j = 0; j < JK_TOPK_PER; ++j) {
     const int idx = base + threadIdx.x + j * 256;
     if (idx < V) s += expf(vals[j] - bmax);
   }
-  const float bsum = jk_block_sum(s, red);
-  if (threadIdx.x == 0) { tk_ms[prow * 2] = bmax; tk_ms[prow * 2 + 1] = bsum; }
-  unsigned taken = 0;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  s = jk_warp_sum(s);
+  if (lane == 0) s_wsum[warp] = s;
+  __syncthreads();
+  if (warp != 0) return;
+  if (lane == 0) {
+    float bsum = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) bsum += s_wsum[w];
+    tk_ms[prow * 2] = bmax;
+    tk_ms[prow * 2 + 1] = bsum;
+  }
+  // merge: lane holds warp winners lane, lane + 32, ... (8 * k_e <= 128 of them)
+  float cv[4];
+  int ci[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = lane + j * 32;                      // candidate (warp = c / k_e, rank = c % k_e)
+    const bool in = c < 8 * k_e;
+    cv[j] = in ? s_cv[(c / k_e) * JK_MAX_KE + c % k_e] : -INFINITY;
+    ci[j] = in ? s_ci[(c / k_e) * JK_MAX_KE + c % k_e] : INT_MAX;
+  }
+  unsigned mtaken = 0;
   for (int it = 0; it < k_e; ++it) {
     float bv = -INFINITY;
-    int bi = INT_MAX;
+    int bi = INT_MAX, bj = -1;
 #pragma unroll
-    for (int j = 0; j < JK_TOPK_PER; ++j) {
-      const int idx = base + threadIdx.x + j * 256;
-      if (!(taken & (1u << j)) && idx < V && jk_better(vals[j], idx, bv, bi)) { bv = vals[j]; bi = idx; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (jk_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
-    if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      float fv = wv[0];
-      int fi = wi[0];
-      for (int w = 1; w < 8; ++w)
-        if (jk_better(wv[w], wi[w], fv, fi)) { fv = wv[w]; fi = wi[w]; }
-      tk_val[prow * k_e + it] = fv;
-      tk_idx[prow * k_e + it] = fi;
-      win_idx = fi;
-    }
-    __syncthreads();
-    const int wsel = win_idx;
-    if (wsel != INT_MAX) {
-#pragma unroll
-      for (int j = 0; j < JK_TOPK_PER; ++j)
-        if (base + threadIdx.x + j * 256 == wsel) taken |= 1u << j;
-    }
-    __syncthreads();
+    for (int j = 0; j < 4; ++j)
+      if (!(mtaken & (1u << j)) && ci[j] != INT_MAX && jk_better(cv[j], ci[j], bv, bi)) {
+        bv = cv[j]; bi = ci[j]; bj = j;
+      }
+    float wv = bv;
+    int wi = bi;
+    jk_warp_argbest(wv, wi);
+    if (wi == bi && bj >= 0) mtaken |= 1u << bj;
+    if (lane == 0) { tk_val[prow * k_e + it] = wv; tk_idx[prow * k_e + it] = wi; }
   }
 }
