@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(256) k_lmhead(
 // ------------------------------------------------------------------------------------------
 // Per-expert top-k over the vocabulary: partial pass per 4096-entry chunk, then a merge.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_topk_partial(
+__global__ void __launch_bounds__(JK_TOPK_THREADS) k_topk_partial(
     const float* __restrict__ logits, int rows_per_b, long long stride_b, int V, int k_e,
     int chunks, float* __restrict__ tk_val, int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
   const int chunk = blockIdx.x, row = blockIdx.y;
@@ -292,7 +292,7 @@ __global__ void __launch_bounds__(256) k_topk_partial(
   float vals[JK_TOPK_PER];
 #pragma unroll
   for (int j = 0; j < JK_TOPK_PER; ++j) {
-    const int idx = base + threadIdx.x + j * 256;
+    const int idx = base + threadIdx.x + j * JK_TOPK_THREADS;
     vals[j] = idx < V ? lr[idx] : -INFINITY;
   }
   jk_topk_chunk_select(vals, base, V, k_e, (size_t)row * chunks + chunk, tk_val, tk_idx, tk_ms);
@@ -520,7 +520,7 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
                                                rows_per_b, lsb);
     JK_LAUNCH_CHECK(ctx);
     JK_PROF(ctx, st, JK_ST_TOPK);
-    k_topk_partial<<<dim3(L.topk_chunks, RK), 256, 0, st>>>(
+    k_topk_partial<<<dim3(L.topk_chunks, RK), JK_TOPK_THREADS, 0, st>>>(
         logits, rows_per_b, lsb, V, c.k_per_expert, L.topk_chunks, (float*)(ws + L.tk_val),
         (int32_t*)(ws + L.tk_idx), (float*)(ws + L.tk_ms));
     JK_LAUNCH_CHECK(ctx);

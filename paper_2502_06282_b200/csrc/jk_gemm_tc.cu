@@ -432,8 +432,8 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
 }
 
 // logits = b W_head^T (Eq. 4) assembled from the partial tiles, optionally stored, and the
-// per-chunk top-k statistics of jk_topk.cuh.   grid (chunks, logits rows), 256 threads.
-__global__ void __launch_bounds__(256) k_tc_fix_lmhead_topk(
+// per-chunk top-k statistics of jk_topk.cuh.   grid (chunks, logits rows), JK_TOPK_THREADS threads.
+__global__ void __launch_bounds__(JK_TOPK_THREADS) k_tc_fix_lmhead_topk(
     const tc_params p, int n_cta, int V, int k_e, int chunks, const float* __restrict__ partial,
     float* __restrict__ logits, int rows_per_b, long long stride_b, float* __restrict__ tk_val,
     int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(256) k_tc_fix_lmhead_topk(
                              (size_t)(row % rows_per_b) * V : nullptr;
 #pragma unroll
   for (int j = 0; j < JK_TOPK_PER; ++j) {
-    const int off = threadIdx.x + j * 256;             // within the chunk
+    const int off = threadIdx.x + j * JK_TOPK_THREADS; // within the chunk
     const int idx = base + off;
     float v = -INFINITY;
     if (idx < V) {
@@ -659,7 +659,7 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   int rc = tc_launch_gemm(ctx, st, s, ag, au, bx, p, expert, JK_ST_GATEUP, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_GEMM_FIXUP);
-  jk_launch_pdl(k_tc_fix_silu, dim3(p.tiles_per_group, N, tc_zdim(p.tiles_per_group * N, R, n_cta)), dim3(128), 0, st, 
+  jk_launch_pdl(k_tc_fix_silu, dim3(p.tiles_per_group, N, R), dim3(128), 0, st, 
       p, n_cta, I, R, Rp, expert, partial, (__nv_bfloat16*)(ctx->ws + L.hbuf));
   JK_LAUNCH_CHECK(ctx);
   // down
@@ -709,7 +709,7 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
   int rc = tc_launch_gemm(ctx, st, s, ah, ah, bb, p, nullptr, JK_ST_LMHEAD, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_TOPK);
-  jk_launch_pdl(k_tc_fix_lmhead_topk, dim3(L.topk_chunks, RK), dim3(256), 0, st, 
+  jk_launch_pdl(k_tc_fix_lmhead_topk, dim3(L.topk_chunks, RK), dim3(JK_TOPK_THREADS), 0, st, 
       p, n_cta, V, c.k_per_expert, L.topk_chunks, (const float*)(ctx->ws + L.gemm_part), logits,
       rows_per_b, logits_stride_b, (float*)(ctx->ws + L.tk_val), (int32_t*)(ctx->ws + L.tk_idx),
       (float*)(ctx->ws + L.tk_ms));

@@ -3,8 +3,8 @@
 // Shared by the CUDA-core path (logits read from global memory) and the tensor-core path (logits
 // assembled from the GEMM's partial tiles).
 //
-// Every warp first picks the k_e best of its own 512 entries with shuffles only; warp 0 then
-// merges the 8 * k_e warp winners.  Two block barriers in total.
+// 1024 threads, 4 entries each.  Every warp first picks the k_e best of its own 128 entries with
+// shuffles only; warp 0 then merges the 32 * k_e warp winners.  Two block barriers in total.
 #pragma once
 
 #include <limits.h>
@@ -12,7 +12,9 @@
 
 #include "jk_common.cuh"
 
-#define JK_TOPK_PER (JK_TOPK_CHUNK / 256)
+#define JK_TOPK_THREADS 1024
+#define JK_TOPK_WARPS (JK_TOPK_THREADS / 32)
+#define JK_TOPK_PER (JK_TOPK_CHUNK / JK_TOPK_THREADS)
 
 __device__ __forceinline__ void jk_warp_argbest(float& v, int& i) {
 #pragma unroll
@@ -23,15 +25,18 @@ __device__ __forceinline__ void jk_warp_argbest(float& v, int& i) {
   }
 }
 
-// 256 threads; thread t holds entries base + t + j*256 in vals[j] (-inf past the vocabulary).
+// JK_TOPK_THREADS threads; thread t holds entries base + t + j*JK_TOPK_THREADS in vals[j]
+// (-inf past the vocabulary).
 __device__ __forceinline__ void jk_topk_chunk_select(const float (&vals)[JK_TOPK_PER], int base,
                                                      int V, int k_e, size_t prow,
                                                      float* __restrict__ tk_val,
                                                      int32_t* __restrict__ tk_idx,
                                                      float* __restrict__ tk_ms) {
-  __shared__ float s_wmax[8], s_wsum[8];
-  __shared__ float s_cv[8 * JK_MAX_KE];
-  __shared__ int s_ci[8 * JK_MAX_KE];
+  constexpr int NW = JK_TOPK_WARPS;
+  constexpr int MC = NW * JK_MAX_KE / 32;          // merge candidates per lane
+  __shared__ float s_wmax[NW], s_wsum[NW];
+  __shared__ float s_cv[NW * JK_MAX_KE];
+  __shared__ int s_ci[NW * JK_MAX_KE];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // warp maximum and the warp's own k_e best
   float lmax = -INFINITY;
@@ -44,7 +49,7 @@ __device__ __forceinline__ void jk_topk_chunk_select(const float (&vals)[JK_TOPK
     int bi = INT_MAX, bj = -1;
 #pragma unroll
     for (int j = 0; j < JK_TOPK_PER; ++j) {
-      const int idx = base + threadIdx.x + j * 256;
+      const int idx = base + threadIdx.x + j * JK_TOPK_THREADS;
       if (!(taken & (1u << j)) && idx < V && jk_better(vals[j], idx, bv, bi)) {
         bv = vals[j]; bi = idx; bj = j;
       }
@@ -59,11 +64,11 @@ __device__ __forceinline__ void jk_topk_chunk_select(const float (&vals)[JK_TOPK
   __syncthreads();
   float bmax = s_wmax[0];
 #pragma unroll
-  for (int w = 1; w < 8; ++w) bmax = fmaxf(bmax, s_wmax[w]);
+  for (int w = 1; w < NW; ++w) bmax = fmaxf(bmax, s_wmax[w]);
   float s = 0.f;
 #pragma unroll
   for (int j = 0; j < JK_TOPK_PER; ++j) {
-    const int idx = base + threadIdx.x + j * 256;
+    const int idx = base + threadIdx.x + j * JK_TOPK_THREADS;
     if (idx < V) s += expf(vals[j] - bmax);
   }
   s = jk_warp_sum(s);
@@ -73,17 +78,17 @@ __device__ __forceinline__ void jk_topk_chunk_select(const float (&vals)[JK_TOPK
   if (lane == 0) {
     float bsum = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) bsum += s_wsum[w];
+    for (int w = 0; w < NW; ++w) bsum += s_wsum[w];
     tk_ms[prow * 2] = bmax;
     tk_ms[prow * 2 + 1] = bsum;
   }
-  // merge: lane holds warp winners lane, lane + 32, ... (8 * k_e <= 128 of them)
-  float cv[4];
-  int ci[4];
+  // merge: lane holds warp winners lane, lane + 32, ... (NW * k_e of them)
+  float cv[MC];
+  int ci[MC];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
+  for (int j = 0; j < MC; ++j) {
     const int c = lane + j * 32;                      // candidate (warp = c / k_e, rank = c % k_e)
-    const bool in = c < 8 * k_e;
+    const bool in = c < NW * k_e;
     cv[j] = in ? s_cv[(c / k_e) * JK_MAX_KE + c % k_e] : -INFINITY;
     ci[j] = in ? s_ci[(c / k_e) * JK_MAX_KE + c % k_e] : INT_MAX;
   }
@@ -92,7 +97,7 @@ __device__ __forceinline__ void jk_topk_chunk_select(const float (&vals)[JK_TOPK
     float bv = -INFINITY;
     int bi = INT_MAX, bj = -1;
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+    for (int j = 0; j < MC; ++j)
       if (!(mtaken & (1u << j)) && ci[j] != INT_MAX && jk_better(cv[j], ci[j], bv, bi)) {
         bv = cv[j]; bi = ci[j]; bj = j;
       }
