@@ -203,3 +203,34 @@ def test_accept_llama2_7b_shape():
                                          tree["depth"][0], tree["branch"][0], tree["qslot"][0],
                                          dl[0], ua[0], ub[0], 1.0, trace=trace)
     assert (acc_idx[0, :n_acc[0]].tolist() == path and bonus[0] == bo) or _near_tie(trace, ua[0])
+
+
+def test_accept_llama2_13b_batch4_sampling():
+    """Batch 4 at the 13B shape: four independent walks, ragged prefix lengths, 2 layers."""
+    w = synth.scaled(synth.WORKLOADS["llama2_13b_b4"], n_layers=2)
+    tree, n_slots = _tree_arrays(w, "random", 41)
+    tl = synth.target_logits(w, tree["tok"], tree["parent"], 0.8, boost=6.0)
+    rng = np.random.default_rng(8)
+    dl = rng.standard_normal((w.batch, n_slots, 2, w.vocab)).astype(np.float32)
+    for b in range(w.batch):
+        for i in range(w.tree_size):
+            s = tree["qslot"][b, i]
+            if s >= 0:
+                dl[b, s] = 0.5 * dl[b, s] + 0.5 * tl[b, i][None]
+    ua, ub = synth.uniforms(w)
+    caches = _caches(w, 2, "bf16", 800)
+    kv_len = np.array([w.prefix, 1500, 7, w.prefix - 1], dtype=np.int32)
+    n_acc, acc_idx, acc_tok, bonus, kvl, gk, gv = _call(w, tree, 1, 1.0, tl, dl, n_slots, ua, ub,
+                                                        caches, kv_len, "bf16")
+    paths = []
+    for b in range(w.batch):
+        trace = []
+        path, toks, bo = orc.accept_sampling(tl[b], tree["tok"][b], tree["parent"][b],
+                                             tree["depth"][b], tree["branch"][b],
+                                             tree["qslot"][b], dl[b], ua[b], ub[b], 1.0,
+                                             trace=trace)
+        got = acc_idx[b, :n_acc[b]].tolist()
+        assert (got == path and bonus[b] == bo) or _near_tie(trace, ua[b]), (b, got, path)
+        paths.append(got)
+        assert kvl[b] == kv_len[b] + 1 + len(got)
+    _check_compaction(w, caches, kv_len, paths, gk, gv)

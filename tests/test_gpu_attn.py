@@ -66,22 +66,31 @@ def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     assert rel_err(got, ref) <= TOL[dtype]
 
 
-def test_attn_llama2_7b_shape_sampled_heads():
-    """Benchmark shape (32 heads x 128, P = 1024, M = 60); the oracle checks three heads."""
-    w = synth.WORKLOADS["llama2_7b"]
+@pytest.mark.parametrize("name,heads,ragged", [
+    ("llama2_7b", (0, 13, 31), False),          # benchmark shape: MHA 32 x 128, P = 1024
+    ("llama2_13b_b4", (5, 39), True),           # batch 4 with ragged prefix lengths, P <= 2048
+    ("llama3_8b", (0, 17), False),              # GQA 32/8, P = 4096: two query blocks per kv head
+    ("llama2_70b_layer", (9, 63), False),       # GQA 64/8, P = 4096: four query blocks per kv head
+])
+def test_attn_full_shapes_sampled_heads(name, heads, ragged):
+    """Full-size shapes, launch configuration as benchmarked; the oracle checks a few q heads."""
+    w = synth.WORKLOADS[name]
     par = _trees(w, "random")
-    q, k, v, kv_len = synth.attn_inputs(w, 0)
+    q, k, v, kv_len = synth.attn_inputs(w, 0, ragged)
     ctx = jk.Context.for_workload(w)
+    assert ctx.tensor_path_active
     qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
     out = torch.empty_like(qd)
-    ctx.tree_verify_attn(1, w.tree_size, qd, kd, vd, dev(kv_len), dev(par),
+    ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, dev(kv_len), dev(par),
                          1.0 / math.sqrt(w.head_dim), out)
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
     got = host(out)
-    for h in (0, 13, 31):
-        ref = orc.tree_verify_attn(q[:, :, h:h + 1], k[:, h:h + 1], v[:, h:h + 1], kv_len, par,
-                                   1.0 / math.sqrt(w.head_dim))
+    G = w.n_q_heads // w.n_kv_heads
+    for h in heads:
+        kh = h // G
+        ref = orc.tree_verify_attn(q[:, :, h:h + 1], k[:, kh:kh + 1], v[:, kh:kh + 1], kv_len,
+                                   par, 1.0 / math.sqrt(w.head_dim))
         assert rel_err(got[:, :, h:h + 1], ref) <= TOL[w.dtype]
 
 

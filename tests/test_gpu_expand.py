@@ -159,37 +159,58 @@ def test_expand_is_deterministic():
         assert torch.equal(a.pool[k], b.pool[k])
 
 
-def test_expand_llama2_7b_shape_sampled_rows():
-    """Full-size shapes of the benchmark configuration, launch configuration as benchmarked;
-    the oracle recomputes two frontier rows of layer 2 and the root row of layer 1."""
-    w = synth.WORKLOADS["llama2_7b"]
+def _sampled_rows(w, samples):
+    """Two draft layers at full-size shapes, launch configuration as benchmarked; the oracle
+    recomputes the (batch, frontier row) pairs in `samples[layer]`."""
     wts = synth.draft_weights(w)
     fs = w.frontier_sizes[:2]
     us = [synth.layer_hidden(w, l, F) for l, F in enumerate(fs)]
-    w2 = synth.scaled(w, depth=2, tree_size=30)
+    w2 = synth.scaled(w, depth=2, tree_size=min(w.tree_size, 12))
     ctx, bufs = _run_gpu(w2, wts, us)
     tol = TOL[w.dtype]
     head64 = wts["lm_head"].astype(np.float64)
+    K, ke = w.top_k, w.k_per_expert
     slot_base = 0
     for l, F in enumerate(fs):
-        rows = [0] if F == 1 else [3, 8]
         u = us[l].astype(np.float64)
         probs_g = host(bufs.probs[l])
-        for f in rows:
-            x = orc.rmsnorm(u[0, f], wts["norm_weight"], 1e-5)
+        for b, f in samples[l]:
+            x = orc.rmsnorm(u[b, f], wts["norm_weight"], 1e-5)
             probs_o = orc.router_scores(x, wts["router"])
-            assert rel_err(probs_g[0, f], probs_o) <= tol
-            ids, _ = orc.topk_gate(probs_g[0, f], w.top_k)
-            assert host(bufs.expert[l])[0, f].tolist() == ids.tolist()
-            _, br, ff = orc.moe_features(u[0, f], x, ids, probs_o[ids], wts)
-            assert rel_err(host(bufs.feat[l])[0, f], ff) <= tol
+            assert rel_err(probs_g[b, f], probs_o) <= tol
+            ids, _ = orc.topk_gate(probs_g[b, f], K)
+            assert host(bufs.expert[l])[b, f].tolist() == ids.tolist()
+            _, br, ff = orc.moe_features(u[b, f], x, ids, probs_o[ids], wts)
+            assert rel_err(host(bufs.feat[l])[b, f], ff) <= tol
             lg_o = br @ head64.T
-            lg_g = host(bufs.logits)[0, slot_base + f]
+            lg_g = host(bufs.logits[b, slot_base + f])
             assert rel_err(lg_g, lg_o) <= tol
-            for r in range(w.top_k):
-                ids_t, sc_t, _ = orc.branch_topk(lg_g[r], w.k_per_expert,
-                                                 float(host(bufs.parent_score[l])[0, f]))
-                g0 = (0 if l == 0 else fs[0] * w.top_k * w.k_per_expert) + \
-                    (f * w.top_k + r) * w.k_per_expert
-                assert host(bufs.pool["tok"])[0, g0:g0 + w.k_per_expert].tolist() == ids_t.tolist()
+            for r in range(K):
+                ids_t, sc_t, _ = orc.branch_topk(lg_g[r], ke,
+                                                 float(host(bufs.parent_score[l])[b, f]))
+                g0 = (0 if l == 0 else fs[0] * K * ke) + (f * K + r) * ke
+                assert host(bufs.pool["tok"])[b, g0:g0 + ke].tolist() == ids_t.tolist()
+                assert np.allclose(host(bufs.pool["score"])[b, g0:g0 + ke], sc_t, rtol=1e-5,
+                                   atol=2e-5)
         slot_base += F
+
+
+def test_expand_llama2_7b_shape_sampled_rows():
+    _sampled_rows(synth.WORKLOADS["llama2_7b"], [[(0, 0)], [(0, 3), (0, 8)]])
+
+
+def test_expand_llama2_13b_batch4_sampled_rows():
+    # 4 sequences x 10 frontier rows = 40 activation rows (48 after padding), 80 logits rows
+    _sampled_rows(synth.WORKLOADS["llama2_13b_b4"], [[(2, 0)], [(0, 9), (3, 4)]])
+
+
+def test_expand_llama3_8b_vocab_sampled_rows():
+    # vocabulary 128256: 32 top-k chunks per row, LM head dominates the bytes
+    _sampled_rows(synth.WORKLOADS["llama3_8b"], [[(0, 0)], [(0, 6)]])
+
+
+def test_expand_llama2_70b_shape_two_experts():
+    # hidden 8192, inner 28672; N = K = 2 (the setting with the best speedup in Table 3) keeps
+    # the host-side weight generation of this test affordable
+    w = synth.scaled(synth.WORKLOADS["llama2_70b_layer"], n_experts=2, name="llama2_70b_n2")
+    _sampled_rows(w, [[(0, 0)], [(0, 5)]])
