@@ -136,8 +136,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
   const long long u1 = tc_span_start(total, blockIdx.x + 1, gridDim.x);
   const int units_per_tile = p.kt;
   const long long first_tile = u0 / units_per_tile;
-  if (!(p.prefetch && warp == 0 && lane == 0)) {
-    jk_pdl_wait();                      // (the prefetching producer waits after its first ring)
+  // (the whole producer warp skips this wait when it prefetches: lanes of that warp waiting here
+  // would hold back the lane that issues the copies; its other lanes touch no global memory)
+  if (!(p.prefetch && warp == 0)) {
+    jk_pdl_wait();
     jk_pdl_trigger();
   }
 
