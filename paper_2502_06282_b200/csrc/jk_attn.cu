@@ -155,19 +155,36 @@ __global__ void __launch_bounds__(256) k_attn_combine(
   const int lane = threadIdx.x & 31;
   const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= n_out) return;
-  float m = -INFINITY;
-  for (int s = 0; s < n_split; ++s) m = fmaxf(m, part_ml[((size_t)s * n_out + row) * 2]);
-  float l = 0.f, acc[DPL];
+  // lane s holds (max, sum) of slice s (n_split <= 32); one load round for all slices
+  float ms = -INFINITY, ls = 0.f;
+  if (lane < n_split) {
+    const float2 v = *reinterpret_cast<const float2*>(part_ml + ((size_t)lane * n_out + row) * 2);
+    ms = v.x;
+    ls = v.y;
+  }
+  const float m = jk_warp_max(ms);
+  const float w_lane = (ms == -INFINITY) ? 0.f : __expf(ms - m);
+  const float l = jk_warp_sum(w_lane * ls);
+  float acc[DPL];
 #pragma unroll
   for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
-  for (int s = 0; s < n_split; ++s) {
-    const float ms = part_ml[((size_t)s * n_out + row) * 2];
-    if (ms == -INFINITY) continue;
-    const float w = __expf(ms - m);
-    l += w * part_ml[((size_t)s * n_out + row) * 2 + 1];
+  for (int s0 = 0; s0 < n_split; s0 += 8) {
+    float v[8][DPL];
 #pragma unroll
-    for (int t = 0; t < DPL; ++t)
-      acc[t] += w * part_o[((size_t)s * n_out + row) * D + lane * DPL + t];
+    for (int j = 0; j < 8; ++j) {                 // eight independent loads in flight
+      const int s = s0 + j;
+#pragma unroll
+      for (int t = 0; t < DPL; ++t)
+        v[j][t] = s < n_split ? part_o[((size_t)s * n_out + row) * D + lane * DPL + t] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float w = __shfl_sync(0xffffffffu, w_lane, (s0 + j) & 31);
+      if (s0 + j < n_split && w != 0.f) {
+#pragma unroll
+        for (int t = 0; t < DPL; ++t) acc[t] += w * v[j][t];
+      }
+    }
   }
   const float inv = 1.f / l;
 #pragma unroll
