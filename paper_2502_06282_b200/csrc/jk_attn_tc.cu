@@ -83,14 +83,15 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
 
   if (have_keys) {
     auto issue_kv = [&](int tile) {
+      const uint64_t pol = l2_policy_evict_first();   // the cache is read once per call
       mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
 #pragma unroll
       for (int kb = 0; kb < KB; ++kb)
-        tma_load_4d(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k);
+        tma_load_4d_hint(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k, pol);
       mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
 #pragma unroll
       for (int kb = 0; kb < KB; ++kb)
-        tma_load_4d(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v);
+        tma_load_4d_hint(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v, pol);
     };
 
     if (tid == 0) {

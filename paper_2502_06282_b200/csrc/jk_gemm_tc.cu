@@ -148,6 +148,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
     int issued = 0;
     bool ok = true;
     const int n_units = (int)(u1 - u0);
+    const uint64_t pol = l2_policy_evict_first();   // weight tiles are read once per call
     // position of a unit of the span, advanced incrementally (no divisions in the loop)
     struct cursor {
       int kt, t, gi, g, arow, brow;
@@ -185,7 +186,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       cursor cb = ca;
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&T.full[i], (uint32_t)stage_bytes);
-        tma_load_2d(smem + (size_t)i * stage_bytes, ca.ma, ca.kt * TC_TILE_K, ca.arow, &T.full[i]);
+        tma_load_2d_hint(smem + (size_t)i * stage_bytes, ca.ma, ca.kt * TC_TILE_K, ca.arow,
+                         &T.full[i], pol);
         cur_next(ca, i + 1 < n_units);
       }
       jk_pdl_wait();
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       unsigned char* sa = smem + (size_t)s * stage_bytes;
       unsigned char* sb = sa + TC_TILE_M * TC_TILE_K * 2;
       mbar_expect_tx(&T.full[s], (uint32_t)stage_bytes);
-      tma_load_2d(sa, ca.ma, ca.kt * TC_TILE_K, ca.arow, &T.full[s]);
+      tma_load_2d_hint(sa, ca.ma, ca.kt * TC_TILE_K, ca.arow, &T.full[s], pol);
       tma_load_2d(sb, &map_b, ca.kt * TC_TILE_K, ca.brow, &T.full[s]);
       if (++s == p.stages) { s = 0; ph ^= 1u; }
       cur_next(ca, issued + 1 < n_units);
