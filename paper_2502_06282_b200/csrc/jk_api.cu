@@ -56,11 +56,11 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->tk_ms = take(RK * L->topk_chunks * 2 * 4);
   L->gemm_part_bytes = c.dtype == JK_BF16 ? jk_tc_partial_bytes(c) : 0;
   L->gemm_part = take(L->gemm_part_bytes);
-  // split-KV partials, capped at 64 MiB
+  // split-KV partials, capped at 256 MiB
   const size_t rows = BM * c.n_q_heads;
   const size_t per_split = rows * (c.head_dim + 2) * 4;
   int ms = JK_ATTN_MAX_SPLIT;
-  while (ms > 1 && per_split * ms > ((size_t)64 << 20)) --ms;
+  while (ms > 1 && per_split * ms > ((size_t)256 << 20)) --ms;
   L->attn_max_split = ms;
   L->attn_o = take(rows * c.head_dim * 4 * ms);
   L->attn_ml = take(rows * 2 * 4 * ms);

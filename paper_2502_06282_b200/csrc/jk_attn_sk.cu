@@ -1,0 +1,632 @@
+// Persistent, pipelined tensor-core kernel of jk_tree_verify_attn for bf16 (arXiv 2502.06282,
+// Sec. 2.1 step 2, mask of Fig. 4).
+//
+// Work is counted in units of one (sequence, kv head, block of 128 query rows, tile of 128 keys).
+// The U units of a call, ordered by sequence, kv head, query block and key tile, are dealt evenly
+// to one CTA per SM: CTA j takes units [floor(j U / n), floor((j + 1) U / n)).  A CTA's range is a
+// list of segments, each a run of key tiles of one query block; a query block whose tiles are
+// spread over several CTAs gets one unnormalised partial (max, sum, O) per CTA, numbered from the
+// first CTA that touches it, and the merge kernel below combines them.
+//
+// Inside the CTA the roles are split across warps and every stage is double-buffered, so that the
+// copy of tile i+1, the S product of tile i+1 and the softmax of tile i run at the same time:
+//   warp 0      TMA producer (K and V tiles, two buffers each)
+//   warp 1      MMA issuer (S = Q K^T into one of two tensor-memory buffers, then O += P V with V
+//               taken MN-major straight from its row-major tile)
+//   warps 2-9   softmax: two threads per query row, each owning 64 of the tile's 128 keys; they
+//               apply the tree mask (a visibility word built from the node's ancestor set and the
+//               prefix length), keep a running max and sum, rescale O in tensor memory when the
+//               max moved and write P = exp(S - max) as bf16 for the second product.
+// 192 KB of shared memory and 512 tensor-memory columns per CTA.  All waits are bounded mbarrier
+// waits (no named barriers), so a role that gives up cannot leave another one waiting for ever.
+#include <math.h>
+#include <stdlib.h>
+
+#include "jk_common.cuh"
+#include "jk_tcgen05.cuh"
+
+#define ASK_ROWS 128
+#define ASK_KEYS 128
+#define ASK_THREADS 320
+#define ASK_SM_THREADS 256
+#define ASK_MAX_UNITS_X_CTAS 0x7fffffffu   // unit index * CTA count stays in 32 bits
+
+struct ask_tail {
+  uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2], s_empty[2];
+  uint64_t p_full, pv_done, q_full, par_full;
+  uint64_t pair[4];                  // the two threads of a row meet here (64 arrivals)
+  uint32_t tmem_base;
+  int abort_flag;
+  int bad;
+  int parent[JK_MAX_TREE];
+  int tiles[JK_MAX_ROWS];            // key tiles of every sequence
+  int plen[JK_MAX_ROWS];             // prefix length of every sequence
+  float xmax[2][2][ASK_ROWS];        // [tile parity][key half][row]: tile maximum of that half
+  float xsum[2][ASK_ROWS];
+};
+
+struct ask_plan {
+  uint32_t U;       // units of the call
+  uint32_t n;       // CTAs that take part
+};
+struct ask_seg {
+  int b, kvh, qblk, tile_lo, tile_hi, slice;
+};
+
+// CTA that owns unit x when U units are dealt to n CTAs as [floor(j U / n), floor((j+1) U / n))
+__device__ __forceinline__ uint32_t ask_owner(uint32_t x, const ask_plan& pl) {
+  return ((x + 1u) * pl.n - 1u) / pl.U;
+}
+__device__ __forceinline__ uint32_t ask_range_start(uint32_t cta, const ask_plan& pl) {
+  return (uint32_t)(((unsigned long long)cta * pl.U) / pl.n);
+}
+
+// U and the number of participating CTAs.  Every range is at least
+// max(min_units, ceil(Tmax / (max_split - 2))) units long, so that no query block is spread over
+// more than max_split - 1 CTAs.
+__device__ __forceinline__ ask_plan ask_make_plan(const int* tiles, int B, int items_per_b,
+                                                  int n_cta, int max_split, int min_units) {
+  uint32_t U = 0;
+  int tmax = 1;
+  for (int b = 0; b < B; ++b) {
+    U += (uint32_t)tiles[b] * (uint32_t)items_per_b;
+    tmax = max(tmax, tiles[b]);
+  }
+  int cmin = (tmax + max_split - 3) / (max_split - 2);
+  if (cmin < min_units) cmin = min_units;
+  uint32_t n = U / (uint32_t)cmin;
+  if (n > (uint32_t)n_cta) n = (uint32_t)n_cta;
+  if (n < 1u) n = 1u;
+  ask_plan p;
+  p.U = U;
+  p.n = n;
+  return p;
+}
+
+// The segment that starts at unit x of a range that ends at x1.
+__device__ __forceinline__ ask_seg ask_segment(const int* tiles, int B, int items_per_b, int n_qblk,
+                                               uint32_t x, uint32_t x1, const ask_plan& pl,
+                                               int cta) {
+  uint32_t base = 0;
+  int b = 0;
+  for (; b < B - 1; ++b) {
+    const uint32_t span = (uint32_t)tiles[b] * (uint32_t)items_per_b;
+    if (x < base + span) break;
+    base += span;
+  }
+  const uint32_t Tb = (uint32_t)tiles[b];
+  const uint32_t rem = x - base;
+  const uint32_t item = rem / Tb;
+  ask_seg s;
+  s.b = b;
+  s.kvh = (int)(item / (uint32_t)n_qblk);
+  s.qblk = (int)(item % (uint32_t)n_qblk);
+  s.tile_lo = (int)(rem - item * Tb);
+  const uint32_t left = x1 - x;
+  s.tile_hi = (int)min(Tb, (uint32_t)s.tile_lo + left);
+  s.slice = cta - (int)ask_owner(base + item * Tb, pl);
+  return s;
+}
+
+template <int D>
+__global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
+    const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+    const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ kv_len,
+    const int32_t* __restrict__ parent, float scale, int B, int M, int Hq, int Hkv, int max_split,
+    int min_units, int cache_rows, float* __restrict__ part_o, float* __restrict__ part_ml,
+    int32_t* status) {
+  constexpr int KB = D / 64;
+  constexpr int Q_BYTES = ASK_ROWS * D * 2;
+  constexpr int KV_BYTES = ASK_KEYS * D * 2;
+  constexpr int P_BYTES = ASK_ROWS * ASK_KEYS * 2;
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t O_COL = 256;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* sq = smem;
+  unsigned char* sk = sq + Q_BYTES;
+  unsigned char* sv = sk + 2 * KV_BYTES;
+  unsigned char* sp = sv + 2 * KV_BYTES;
+  ask_tail& T = *reinterpret_cast<ask_tail*>(sp + P_BYTES);
+  volatile int* abort_flag = &T.abort_flag;
+
+  const int G = Hq / Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_rows = G * M;
+  const int n_qblk = (n_rows + ASK_ROWS - 1) / ASK_ROWS;
+  const int items_per_b = Hkv * n_qblk;
+  const size_t n_out = (size_t)B * M * Hq;
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&T.k_full[i], 1); mbar_init(&T.v_full[i], 1);
+      mbar_init(&T.k_empty[i], 1); mbar_init(&T.v_empty[i], 1);
+      mbar_init(&T.s_full[i], 1); mbar_init(&T.s_empty[i], ASK_SM_THREADS);
+    }
+    mbar_init(&T.p_full, ASK_SM_THREADS);
+    mbar_init(&T.pv_done, 1);
+    mbar_init(&T.q_full, ASK_SM_THREADS);
+    mbar_init(&T.par_full, ASK_SM_THREADS);
+    for (int i = 0; i < 4; ++i) mbar_init(&T.pair[i], 64);
+    T.abort_flag = 0;
+    T.bad = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(&T.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  __syncthreads();
+  // everything above touches no global memory; kv_len may be the product of the kernel before
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  for (int i = tid; i < B; i += ASK_THREADS) {
+    const int P = kv_len[i];
+    const bool bad = P < 0 || P + M > cache_rows;
+    T.plen[i] = P;
+    T.tiles[i] = bad ? 1 : (P + M + ASK_KEYS - 1) / ASK_KEYS;
+    if (bad) T.bad = 1;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = T.tmem_base;
+  const bool bad = T.bad != 0;
+  if (bad && blockIdx.x == 0 && tid == 0) jk_set_status(status, JK_ERR_BOUNDS);
+  const ask_plan pl = ask_make_plan(T.tiles, B, items_per_b, (int)gridDim.x, max_split, min_units);
+  const int cta = (int)blockIdx.x;
+  uint32_t x0 = 0, x1 = 0;
+  if (!bad && (uint32_t)cta < pl.n) {
+    x0 = ask_range_start((uint32_t)cta, pl);
+    x1 = ask_range_start((uint32_t)cta + 1u, pl);
+  }
+  bool ok = true;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    // K runs one tile ahead of V: the K buffer of tile g is free as soon as S of tile g-2 has
+    // completed, the V buffer only after the second product of tile g-2.
+    if (lane == 0) {
+      const uint64_t pol = l2_policy_evict_first();   // the cache is read once per call
+      int g = 0;
+      int pt = 0, pkvh = 0, pb = 0;                 // coordinates of tile g-1 (its V is still due)
+      auto load_v = [&](int gv, int t, int kvh, int b) -> bool {
+        const int bf = gv & 1;
+        if (gv >= 2 &&
+            !mbar_wait(&T.v_empty[bf], (uint32_t)((gv >> 1) - 1) & 1u, abort_flag, status))
+          return false;
+        mbar_expect_tx(&T.v_full[bf], KV_BYTES);
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_4d_hint(sv + bf * KV_BYTES + kb * 16384, &map_v, kb * 64, t * ASK_KEYS, kvh, b,
+                           &T.v_full[bf], pol);
+        return true;
+      };
+      for (uint32_t x = x0; x < x1 && ok;) {
+        const ask_seg s = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
+        for (int t = s.tile_lo; t < s.tile_hi; ++t, ++g) {
+          const int bf = g & 1;
+          if (g >= 2)
+            ok = mbar_wait(&T.k_empty[bf], (uint32_t)((g >> 1) - 1) & 1u, abort_flag, status);
+          if (!ok) break;
+          mbar_expect_tx(&T.k_full[bf], KV_BYTES);
+#pragma unroll
+          for (int kb = 0; kb < KB; ++kb)
+            tma_load_4d_hint(sk + bf * KV_BYTES + kb * 16384, &map_k, kb * 64, t * ASK_KEYS, s.kvh,
+                             s.b, &T.k_full[bf], pol);
+          if (g >= 1) ok = load_v(g - 1, pt, pkvh, pb);
+          if (!ok) break;
+          pt = t; pkvh = s.kvh; pb = s.b;
+        }
+        x += (uint32_t)(s.tile_hi - s.tile_lo);
+      }
+      if (ok && g >= 1) ok = load_v(g - 1, pt, pkvh, pb);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = instr_desc_bf16_ex(ASK_KEYS, 0);
+      const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
+      const uint32_t qa = smem_u32(sq), pa = smem_u32(sp);
+      auto s_ready = [&](int g) -> bool {
+        const int bf = g & 1;
+        const uint32_t ph = (uint32_t)(g >> 1) & 1u;
+        return mbar_try_wait(&T.k_full[bf], ph) && (g < 2 || mbar_try_wait(&T.s_empty[bf], ph ^ 1u));
+      };
+      auto issue_s = [&](int g) -> bool {
+        const int bf = g & 1;
+        const uint32_t ph = (uint32_t)(g >> 1) & 1u;
+        if (!mbar_wait(&T.k_full[bf], ph, abort_flag, status)) return false;
+        if (g >= 2 && !mbar_wait(&T.s_empty[bf], ph ^ 1u, abort_flag, status)) return false;
+        tc_fence_after();
+        const uint32_t ka = smem_u32(sk + bf * KV_BYTES);
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            tc_mma_bf16(tmem_base + (uint32_t)bf * 128u, smem_desc_sw128(qa + kb * 16384 + k * 32),
+                        smem_desc_sw128(ka + kb * 16384 + k * 32), idesc_s, (kb | k) ? 1u : 0u);
+        tc_commit(&T.s_full[bf]);
+        tc_commit(&T.k_empty[bf]);
+        return true;
+      };
+      int g = 0, seg = 0;
+      for (uint32_t x = x0; x < x1 && ok; ++seg) {
+        const ask_seg s = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
+        ok = mbar_wait(&T.q_full, (uint32_t)seg & 1u, abort_flag, status);
+        ok = ok && issue_s(g);
+        for (int t = s.tile_lo; t < s.tile_hi && ok; ++t, ++g) {
+          const int bf = g & 1;
+          // S of the next tile goes first if its K tile is already there, else after P V
+          bool ahead = false;
+          if (t + 1 < s.tile_hi && s_ready(g + 1)) { ok = issue_s(g + 1); ahead = true; }
+          ok = ok && mbar_wait(&T.p_full, (uint32_t)g & 1u, abort_flag, status);
+          ok = ok && mbar_wait(&T.v_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t va = smem_u32(sv + bf * KV_BYTES);
+#pragma unroll
+          for (int j = 0; j < ASK_KEYS / 16; ++j)
+            tc_mma_bf16(tmem_base + O_COL, smem_desc_sw128(pa + (j >> 2) * 16384 + (j & 3) * 32),
+                        smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
+                        (t > s.tile_lo || j > 0) ? 1u : 0u);
+          tc_commit(&T.v_empty[bf]);
+          tc_commit(&T.pv_done);
+          if (t + 1 < s.tile_hi && !ahead) ok = issue_s(g + 1);
+        }
+        x += (uint32_t)(s.tile_hi - s.tile_lo);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax (2 threads / row)
+    // tensor-memory lane quarter = warp % 4, key half = (warp - 2) / 4
+    const int quarter = warp & 3, half = (warp - 2) >> 2;
+    const int row = quarter * 32 + lane;
+    const int sm_tid = tid - 64;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const float sl2 = scale * 1.4426950408889634f;
+    unsigned char* prow = sp + half * 16384 + row * 128;
+    constexpr int QV = D / 16;                       // 16-byte vectors of half a query row
+    int g = 0, seg = 0;
+    uint32_t pair_uses = 0;
+    auto pair_sync = [&]() -> bool {
+      mbar_arrive(&T.pair[quarter]);
+      const bool o = mbar_wait(&T.pair[quarter], pair_uses & 1u, abort_flag, status);
+      ++pair_uses;
+      return __all_sync(0xffffffffu, o);
+    };
+    for (uint32_t x = x0; x < x1; ++seg) {
+      const ask_seg s = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
+      x += (uint32_t)(s.tile_hi - s.tile_lo);
+      const int P = T.plen[s.b];
+      const int row0 = s.qblk * ASK_ROWS;
+      const bool row_valid = row0 + row < n_rows;
+      const bool warp_active = row0 + quarter * 32 < n_rows;
+      const int g_idx = row_valid ? (row0 + row) / M : 0;
+      const int node = row_valid ? (row0 + row) % M : 0;
+      const size_t orow = ((size_t)s.b * M + node) * Hq + s.kvh * G + g_idx;
+      // this segment's tree and query rows (every MMA of the previous segment has completed)
+      uint4 qv[QV];
+#pragma unroll
+      for (int c = 0; c < QV; ++c) {
+        qv[c] = make_uint4(0u, 0u, 0u, 0u);
+        if (row_valid)
+          qv[c] = __ldg(reinterpret_cast<const uint4*>(q + orow * D + half * (D / 2) + c * 8));
+      }
+      if (sm_tid < M) T.parent[sm_tid] = __ldg(parent + (size_t)s.b * M + sm_tid);
+      mbar_arrive(&T.par_full);
+#pragma unroll
+      for (int c = 0; c < QV; ++c) {
+        const int ch = half * QV + c;
+        *reinterpret_cast<uint4*>(sq + (ch >> 3) * 16384 + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
+            qv[c];
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&T.q_full);
+      {
+        const bool okp = mbar_wait(&T.par_full, (uint32_t)seg & 1u, abort_flag, status);
+        ok = __all_sync(0xffffffffu, okp);
+      }
+      if (!ok) break;
+      unsigned long long anc_lo = 0ull, anc_hi = 0ull;
+      if (row_valid) {
+        int c = node;
+        for (int guard = 0; c >= 0 && guard <= JK_MAX_TREE; ++guard) {
+          if (c < 64) anc_lo |= 1ull << c; else anc_hi |= 1ull << (c - 64);
+          const int pp = T.parent[c];
+          c = (pp < c) ? pp : -1;
+        }
+      }
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int tile = s.tile_lo; tile < s.tile_hi; ++tile, ++g) {
+        const int bf = g & 1;
+        // visibility of this thread's 64 keys (Fig. 4): prefix keys, then the ancestor set
+        unsigned long long vis_lo = 0ull, vis_hi = 0ull;
+        if (row_valid) {
+          const int sft = P - tile * ASK_KEYS;
+          if (sft >= 128) { vis_lo = ~0ull; vis_hi = ~0ull; }
+          else if (sft >= 0) {
+            if (sft >= 64) { vis_lo = ~0ull; vis_hi = (sft == 64) ? 0ull : ((1ull << (sft - 64)) - 1ull); }
+            else { vis_lo = (sft == 0) ? 0ull : ((1ull << sft) - 1ull); }
+            unsigned long long a_lo, a_hi;
+            if (sft == 0) { a_lo = anc_lo; a_hi = anc_hi; }
+            else if (sft < 64) { a_lo = anc_lo << sft; a_hi = (anc_hi << sft) | (anc_lo >> (64 - sft)); }
+            else if (sft == 64) { a_lo = 0ull; a_hi = anc_lo; }
+            else { a_lo = 0ull; a_hi = anc_lo << (sft - 64); }
+            vis_lo |= a_lo; vis_hi |= a_hi;
+          } else {
+            const int t = -sft;
+            if (t < 64) { vis_lo = (anc_lo >> t) | (anc_hi << (64 - t)); vis_hi = anc_hi >> t; }
+            else if (t < 128) { vis_lo = anc_hi >> (t - 64); vis_hi = 0ull; }
+          }
+        }
+        const unsigned long long vis = half ? vis_hi : vis_lo;
+        const unsigned b0 = (unsigned)vis, b1 = (unsigned)(vis >> 32);
+        {
+          const bool okw = mbar_wait(&T.s_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
+          ok = __all_sync(0xffffffffu, okw);
+        }
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = tmem_base + lane_base + (uint32_t)bf * 128u + (uint32_t)half * 64u;
+        // pass 1: maximum of the visible scores of this half; the row maximum via the partner
+        float mx = -INFINITY;
+        if (warp_active) {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(sa, r0);
+          tmem_ld32(sa + 32u, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
+            if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r1[j]));
+          }
+        }
+        T.xmax[bf][half][row] = mx;
+        ok = pair_sync();
+        if (!ok) break;
+        const float m_new = fmaxf(m_run, fmaxf(mx, T.xmax[bf][half ^ 1][row]));
+        const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
+                                                 : fast_exp2((m_run - m_new) * sl2);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        if (tile > s.tile_lo) {
+          // P and O are free once the previous tile's P V product has completed
+          const bool okp = mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
+          ok = __all_sync(0xffffffffu, okp);
+          if (!ok) break;
+          tc_fence_after();
+          if (warp_active && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+            for (int c = 0; c < D / 64; ++c) {
+              uint32_t r[32];
+              const uint32_t oa = tmem_base + lane_base + O_COL + (uint32_t)(half * (D / 2) + c * 32);
+              tmem_ld32(oa, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+              tmem_st32(oa, r);
+            }
+            tmem_st_wait();
+          }
+        }
+        // pass 2: P = exp(S - max) as bf16, 32 keys at a time, read again from tensor memory
+        float lsum = 0.f;
+        if (warp_active) {
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t r[32];
+            tmem_ld32(sa + (uint32_t)(hh * 32), r);
+            tmem_ld_wait();
+            const unsigned bits = hh ? b1 : b0;
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(r[j]) - m_use) * sl2) : 0.f;
+              const float p1 = ((bits >> (j + 1)) & 1u)
+                                   ? fast_exp2((__uint_as_float(r[j + 1]) - m_use) * sl2) : 0.f;
+              lsum += p0 + p1;
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+              pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              const int cb = hh * 4 + cc;
+              *reinterpret_cast<uint4*>(prow + ((cb ^ (row & 7)) << 4)) =
+                  make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+            }
+          }
+        }
+        l_run = l_run * alpha + lsum;
+        m_run = m_new;
+        fence_proxy_async_smem();
+        tc_fence_before();
+        mbar_arrive(&T.s_empty[bf]);
+        mbar_arrive(&T.p_full);
+      }
+      if (!ok) break;
+      // ---- the segment's partial (max, sum, O) of every row
+      {
+        const bool okd = mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
+        ok = __all_sync(0xffffffffu, okd);
+      }
+      if (!ok) break;
+      tc_fence_after();
+      T.xsum[half][row] = l_run;
+      ok = pair_sync();
+      if (!ok) break;
+      if (warp_active) {
+        float* po = part_o + ((size_t)s.slice * n_out + orow) * D + half * (D / 2);
+#pragma unroll 1
+        for (int c = 0; c < D / 64; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(half * (D / 2) + c * 32), r);
+          tmem_ld_wait();
+          if (row_valid) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(po + c * 32 + j) =
+                  make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                              __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+          }
+        }
+        if (row_valid && half == 0) {
+          part_ml[((size_t)s.slice * n_out + orow) * 2] =
+              (m_run == -INFINITY) ? -INFINITY : m_run * scale;
+          part_ml[((size_t)s.slice * n_out + orow) * 2 + 1] = l_run + T.xsum[1][row];
+        }
+      }
+      tc_fence_before();
+    }
+  }
+  if (tid == 0 && *abort_flag) {
+    // some role gave up, possibly with copies still in flight: give them a bounded time to land
+    const unsigned long long ts = global_ns();
+    while (global_ns() - ts < 2000000ull) { /* 2 ms: far longer than any TMA copy */ }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// Merge of the partials of one output row (one warp per row): the number of partials of the
+// row's query block follows from the same dealing of units to CTAs as in the kernel above.
+template <int D>
+__global__ void __launch_bounds__(256) k_attn_combine_sk(
+    const float* __restrict__ part_o, const float* __restrict__ part_ml,
+    const int32_t* __restrict__ kv_len, int B, int M, int Hq, int Hkv, int n_cta, int max_split,
+    int min_units, int cache_rows, __nv_bfloat16* __restrict__ out) {
+  __shared__ int s_tiles[JK_MAX_ROWS];
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  for (int i = threadIdx.x; i < B; i += blockDim.x) {
+    const int P = kv_len[i];         // not written by the attention kernel: read before the wait
+    const bool bad = P < 0 || P + M > cache_rows;
+    s_tiles[i] = bad ? 1 : (P + M + ASK_KEYS - 1) / ASK_KEYS;
+    if (bad) s_bad = 1;
+  }
+  __syncthreads();
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  if (s_bad) return;
+  constexpr int DPL = D / 32;
+  const int lane = threadIdx.x & 31;
+  const size_t n_out = (size_t)B * M * Hq;
+  const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= n_out) return;
+  const int G = Hq / Hkv;
+  const int n_qblk = (G * M + ASK_ROWS - 1) / ASK_ROWS;
+  const int items_per_b = Hkv * n_qblk;
+  const ask_plan pl = ask_make_plan(s_tiles, B, items_per_b, n_cta, max_split, min_units);
+  const int head = (int)(row % Hq);
+  const int node = (int)((row / Hq) % M);
+  const int b = (int)(row / ((size_t)Hq * M));
+  uint32_t base = 0;
+  for (int i = 0; i < b; ++i) base += (uint32_t)s_tiles[i] * (uint32_t)items_per_b;
+  const uint32_t Tb = (uint32_t)s_tiles[b];
+  const uint32_t item = (uint32_t)((head / G) * n_qblk + ((head % G) * M + node) / ASK_ROWS);
+  const uint32_t start = base + item * Tb;
+  const int n_split = (int)(ask_owner(start + Tb - 1u, pl) - ask_owner(start, pl)) + 1;
+  // lane s holds (max, sum) of partial s (n_split < 32); one load round for all partials
+  float ms = -INFINITY, ls = 0.f;
+  if (lane < n_split) {
+    const float2 v = *reinterpret_cast<const float2*>(part_ml + ((size_t)lane * n_out + row) * 2);
+    ms = v.x;
+    ls = v.y;
+  }
+  const float m = jk_warp_max(ms);
+  const float w_lane = (ms == -INFINITY) ? 0.f : __expf(ms - m);
+  const float l = jk_warp_sum(w_lane * ls);
+  float acc[DPL];
+#pragma unroll
+  for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
+  for (int s0 = 0; s0 < n_split; s0 += 4) {
+    float v[4][DPL];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {                 // four independent loads in flight
+      const int s = s0 + j;
+#pragma unroll
+      for (int t = 0; t < DPL; ++t)
+        v[j][t] = s < n_split ? part_o[((size_t)s * n_out + row) * D + lane * DPL + t] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float w = __shfl_sync(0xffffffffu, w_lane, (s0 + j) & 31);
+      if (s0 + j < n_split && w != 0.f) {
+#pragma unroll
+        for (int t = 0; t < DPL; ++t) acc[t] += w * v[j][t];
+      }
+    }
+  }
+  const float inv = 1.f / l;
+#pragma unroll
+  for (int t = 0; t < DPL; ++t)
+    out[row * D + lane * DPL + t] = __float2bfloat16_rn(acc[t] * inv);
+}
+
+// jk_attn_tc.cu: tensor maps of the two caches
+int jk_attn_tc_maps(jk_ctx* ctx, const void* kc, const void* vc, int64_t sb, int64_t sh,
+                    int cache_rows, const CUtensorMap** mk, const CUtensorMap** mv);
+
+// The kernel needs room for at least three partials per query block, sequence counts that fit
+// its shared arrays, and unit indices that stay in 32 bits.
+int jk_attn_sk_usable(const jk_ctx* ctx, int B, int M, int cache_rows) {
+  const jk_config& c = ctx->cfg;
+  if (ctx->lay.attn_max_split < 4 || B > JK_MAX_ROWS || ctx->sm_count < 1) return 0;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const unsigned long long units = (unsigned long long)B * c.n_kv_heads *
+                                   ((G * M + ASK_ROWS - 1) / ASK_ROWS) *
+                                   ((cache_rows + ASK_KEYS - 1) / ASK_KEYS);
+  return units * (unsigned long long)ctx->sm_count <= ASK_MAX_UNITS_X_CTAS;
+}
+
+int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
+               const void* vc, int64_t sb, int64_t sh, int cache_rows, const int32_t* kv_len,
+               const int32_t* parent, float scale, void* out) {
+  const jk_config& c = ctx->cfg;
+  const jk_ws_layout& L = ctx->lay;
+  const CUtensorMap *mk = nullptr, *mv = nullptr;
+  int rc = jk_attn_tc_maps(ctx, kc, vc, sb, sh, cache_rows, &mk, &mv);
+  if (rc != JK_OK) return rc;
+  const int D = c.head_dim;
+  float* part_o = (float*)(ctx->ws + L.attn_o);
+  float* part_ml = (float*)(ctx->ws + L.attn_ml);
+  int32_t* status = (int32_t*)(ctx->ws + L.status);
+  if (!ctx->attn_sk_smem_set) {
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<128>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024));
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<64>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024));
+    ctx->attn_sk_smem_set = 1;
+  }
+  const size_t smem = (size_t)ASK_ROWS * D * 2 + 4 * (size_t)ASK_KEYS * D * 2 +
+                      (size_t)ASK_ROWS * ASK_KEYS * 2 + sizeof(ask_tail) + 1024;
+  const int n_cta = ctx->sm_count;
+  const int ms = L.attn_max_split;
+  const char* mu_env = getenv("JK_ATTN_MINU");
+  const int min_units = mu_env ? atoi(mu_env) : 1;
+  JK_PROF(ctx, st, JK_ST_ATTN);
+  if (D == 128)
+    jk_launch_pdl(k_tree_attn_sk<128>, dim3(n_cta), dim3(ASK_THREADS), smem, st, *mk, *mv,
+                  (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
+                  ms, min_units, cache_rows, part_o, part_ml, status);
+  else
+    jk_launch_pdl(k_tree_attn_sk<64>, dim3(n_cta), dim3(ASK_THREADS), smem, st, *mk, *mv,
+                  (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
+                  ms, min_units, cache_rows, part_o, part_ml, status);
+  JK_LAUNCH_CHECK(ctx);
+  const size_t n_out = (size_t)B * M * c.n_q_heads;
+  JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
+  if (D == 128)
+    jk_launch_pdl(k_attn_combine_sk<128>, dim3((unsigned)((n_out + 7) / 8)), dim3(256), 0, st,
+                  (const float*)part_o, (const float*)part_ml, kv_len, B, M, c.n_q_heads,
+                  c.n_kv_heads, n_cta, ms, min_units, cache_rows, (__nv_bfloat16*)out);
+  else
+    jk_launch_pdl(k_attn_combine_sk<64>, dim3((unsigned)((n_out + 7) / 8)), dim3(256), 0, st,
+                  (const float*)part_o, (const float*)part_ml, kv_len, B, M, c.n_q_heads,
+                  c.n_kv_heads, n_cta, ms, min_units, cache_rows, (__nv_bfloat16*)out);
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}

@@ -346,19 +346,36 @@ void jk_attn_tc_destroy(jk_ctx* ctx) {
   }
 }
 
-int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
-               const void* vc, int64_t sb, int64_t sh, int cache_rows, const int32_t* kv_len,
-               const int32_t* parent, float scale, void* out) {
-  const jk_config& c = ctx->cfg;
-  const jk_ws_layout& L = ctx->lay;
+// Tensor maps of a K and a V cache (cached per pointer and strides).
+int jk_attn_tc_maps(jk_ctx* ctx, const void* kc, const void* vc, int64_t sb, int64_t sh,
+                    int cache_rows, const CUtensorMap** mk, const CUtensorMap** mv) {
   if (!ctx->attn_tc_state) {
     ctx->attn_tc_state = calloc(1, sizeof(atc_state));
     if (!ctx->attn_tc_state) return JK_ERR_CUDA;
   }
   atc_state* s = (atc_state*)ctx->attn_tc_state;
-  const CUtensorMap* mk = atc_map(ctx, s, kc, sb, sh, cache_rows);
-  const CUtensorMap* mv = atc_map(ctx, s, vc, sb, sh, cache_rows);
-  if (!mk || !mv) return JK_ERR_CUDA;
+  *mk = atc_map(ctx, s, kc, sb, sh, cache_rows);
+  *mv = atc_map(ctx, s, vc, sb, sh, cache_rows);
+  return (*mk && *mv) ? JK_OK : JK_ERR_CUDA;
+}
+
+// jk_attn_sk.cu: the persistent pipelined kernel
+int jk_attn_sk_usable(const jk_ctx* ctx, int B, int M, int cache_rows);
+int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
+               const void* vc, int64_t sb, int64_t sh, int cache_rows, const int32_t* kv_len,
+               const int32_t* parent, float scale, void* out);
+
+int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
+               const void* vc, int64_t sb, int64_t sh, int cache_rows, const int32_t* kv_len,
+               const int32_t* parent, float scale, void* out) {
+  const jk_config& c = ctx->cfg;
+  const jk_ws_layout& L = ctx->lay;
+  const char* sk_env = getenv("JK_ATTN_SK");
+  if (sk_env && sk_env[0] == '1' && jk_attn_sk_usable(ctx, B, M, cache_rows))
+    return jk_attn_sk(ctx, st, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale, out);
+  const CUtensorMap *mk = nullptr, *mv = nullptr;
+  if (jk_attn_tc_maps(ctx, kc, vc, sb, sh, cache_rows, &mk, &mv) != JK_OK) return JK_ERR_CUDA;
+  atc_state* s = (atc_state*)ctx->attn_tc_state;
   const int G = c.n_q_heads / c.n_kv_heads;
   const int n_qblk = (G * M + ATC_ROWS - 1) / ATC_ROWS;
   const int base = n_qblk * c.n_kv_heads * B;

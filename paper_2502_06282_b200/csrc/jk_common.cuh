@@ -73,6 +73,7 @@ struct jk_ctx {
   int tensor_path;
   int sm_count;           // filled at the first launch
   int attn_smem_set;
+  int attn_sk_smem_set;
   char cuda_err[256];
   void* tc_state;         // tensor-core path bookkeeping (tensor maps), host memory
   void* attn_tc_state;    // tensor maps of the KV caches seen by the attention kernel
