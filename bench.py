@@ -229,17 +229,32 @@ def main():
     ua, ub = dev(ua_np), dev(ub_np)
     mode = 1 if args.mode == "sampling" else 0
 
-    def step():
+    inA = {"us": us, "q_all": q_all, "tl": tl, "ua": ua, "ub": ub, "root": root}
+
+    def step(inp=inA):
         kv_len.copy_(kv_len0)
-        jk.run_draft(ctx, bufs, wstruct, us, root)
+        jk.run_draft(ctx, bufs, wstruct, inp["us"], inp["root"])
         for l in range(L):
-            ctx.tree_verify_attn(w.batch, w.tree_size, q_all[l], ks[l], vs[l], kv_len,
+            ctx.tree_verify_attn(w.batch, w.tree_size, inp["q_all"][l], ks[l], vs[l], kv_len,
                                  bufs.tree["parent"], scale, outs[l])
-        ctx.accept_and_compact(w.batch, w.tree_size, mode, 1.0, tl, bufs.tree,
-                               bufs.logits if mode else None, w.n_slots, ua if mode else None,
-                               ub if mode else None, L, kp, vp, ks[0].stride(0), ks[0].stride(1),
-                               ks[0].shape[2], kv_len, bufs.n_acc, bufs.acc_idx, bufs.acc_tok,
-                               bufs.bonus)
+        ctx.accept_and_compact(w.batch, w.tree_size, mode, 1.0, inp["tl"], bufs.tree,
+                               bufs.logits if mode else None, w.n_slots,
+                               inp["ua"] if mode else None, inp["ub"] if mode else None, L, kp, vp,
+                               ks[0].stride(0), ks[0].stride(1), ks[0].shape[2], kv_len,
+                               bufs.n_acc, bufs.acc_idx, bufs.acc_tok, bufs.bonus)
+
+    def capture(inp):
+        cs = torch.cuda.Stream()
+        cs.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cs):
+            step(inp)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cs):
+            step(inp)
+        g.replay()
+        torch.cuda.synchronize()
+        return g
 
     def barrier():
         if world > 1:
@@ -254,16 +269,7 @@ def main():
     graph = None
     if not args.no_graph:
         try:
-            cs = torch.cuda.Stream()
-            cs.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(cs):
-                step()
-            torch.cuda.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=cs):
-                step()
-            graph.replay()
-            torch.cuda.synchronize()
+            graph = capture(inA)
         except Exception as exc:          # fall back to launching every call
             sys.stderr.write(f"graph capture failed, timing eager launches: {exc}\n")
             graph = None
@@ -333,31 +339,57 @@ def main():
     # ---------------------------------------------------------------- end to end from host
     e2e = None
     if not args.no_e2e:
+        # Every step copies its own inputs from pinned host memory and reads its results back.
+        # Inputs are double-buffered on the device: the copies of step s+1 run on a copy stream
+        # while step s computes, and the results of step s are read while step s+1 runs.
         pin = lambda t: t.cpu().pin_memory()
-        h_us, h_q, h_tl, h_ua, h_ub, h_root = ([pin(u) for u in us], pin(q_all), pin(tl), pin(ua),
-                                               pin(ub), pin(root))
-        h2d = sum(t.numel() * t.element_size() for t in h_us + [h_q, h_tl, h_ua, h_ub, h_root])
-        d2h = sum(t.numel() * t.element_size() for t in (bufs.n_acc, bufs.acc_idx, bufs.acc_tok,
-                                                          bufs.bonus, kv_len))
+        hostA = {"us": [pin(u) for u in us], "q_all": pin(q_all), "tl": pin(tl), "ua": pin(ua),
+                 "ub": pin(ub), "root": pin(root)}
+        inB = {"us": [u.clone() for u in us], "q_all": q_all.clone(), "tl": tl.clone(),
+               "ua": ua.clone(), "ub": ub.clone(), "root": root.clone()}
+        sets = [inA, inB]
+        runs = [run_step, (capture(inB).replay if graph is not None else (lambda: step(inB)))]
+        flat = lambda d: d["us"] + [d["q_all"], d["tl"], d["ua"], d["ub"], d["root"]]
+        h2d = sum(t.numel() * t.element_size() for t in flat(hostA))
+        results = (bufs.n_acc, bufs.acc_idx, bufs.acc_tok, bufs.bonus, kv_len)
+        d2h = sum(t.numel() * t.element_size() for t in results)
+        host_out = [[torch.empty_like(t, device="cpu").pin_memory() for t in results] for _ in range(2)]
+        copy_stream, comp_stream = torch.cuda.Stream(), torch.cuda.Stream()
+        h2d_done = [torch.cuda.Event() for _ in range(2)]
+        comp_done = [torch.cuda.Event() for _ in range(2)]
+        out_done = [torch.cuda.Event() for _ in range(2)]
 
-        def step_e2e():
-            for d, h in zip(us, h_us):
-                d.copy_(h, non_blocking=True)
-            q_all.copy_(h_q, non_blocking=True)
-            tl.copy_(h_tl, non_blocking=True)
-            ua.copy_(h_ua, non_blocking=True)
-            ub.copy_(h_ub, non_blocking=True)
-            root.copy_(h_root, non_blocking=True)
-            run_step()
-            return (bufs.n_acc.cpu(), bufs.acc_idx.cpu(), bufs.acc_tok.cpu(), bufs.bonus.cpu(),
-                    kv_len.cpu())
+        def run_e2e(n):
+            got = 0
+            for i in range(n):
+                k = i & 1
+                with torch.cuda.stream(copy_stream):
+                    if i >= 2:
+                        copy_stream.wait_event(comp_done[k])     # the set's last reader is done
+                    for d, h in zip(flat(sets[k]), flat(hostA)):
+                        d.copy_(h, non_blocking=True)
+                    h2d_done[k].record(copy_stream)
+                with torch.cuda.stream(comp_stream):
+                    comp_stream.wait_event(h2d_done[k])
+                    runs[k]()
+                    comp_done[k].record(comp_stream)
+                    for d, h in zip(results, host_out[k]):
+                        h.copy_(d, non_blocking=True)
+                    out_done[k].record(comp_stream)
+                if i >= 1:                                       # results of the step before
+                    out_done[k ^ 1].synchronize()
+                    got += int(host_out[k ^ 1][0][0])
+            out_done[(n - 1) & 1].synchronize()
+            return got + int(host_out[(n - 1) & 1][0][0])
 
-        step_e2e()
-        n_e2e = max(3, args.steps // 2)
+        torch.cuda.synchronize()
+        run_e2e(2)
+        n_e2e = max(4, args.steps // 2)
         barrier()
         e0.record()
-        for _ in range(n_e2e):
-            step_e2e()
+        run_e2e(n_e2e)
+        comp_stream.synchronize()
+        torch.cuda.current_stream().wait_stream(comp_stream)
         e1.record()
         barrier()
         ms_e = e0.elapsed_time(e1)
@@ -366,7 +398,8 @@ def main():
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             ms_e = float(t.item())
         e2e = {"value": world * 1000.0 * n_e2e / ms_e, "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": n_e2e}
+               "d2h_bytes_per_step": d2h, "steps": n_e2e,
+               "pipelining": "inputs double-buffered; copies of step s+1 overlap step s"}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

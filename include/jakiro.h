@@ -89,6 +89,12 @@ int jk_set_tensor_path(jk_ctx* ctx, int32_t enable);
 /* 1 if the tensor-core kernels will run the contractions of this context (bf16, enabled, rows
  * within their limit, driver entry point for tensor maps found), else 0. */
 int jk_tensor_path_active(jk_ctx* ctx);
+/* Which tensor-core kernel runs jk_tree_verify_attn for bf16: 0 = chosen per call from the sizes
+ * (default), 1 = one CTA per (query block, key slice), 2 = the persistent kernel that deals key
+ * tiles evenly to one CTA per SM (falls back to 1 where its limits do not hold).  Both compute
+ * the operation of arXiv 2502.06282 Sec. 2.1 step 2 with the mask of Fig. 4; the choice only
+ * affects speed.  Returns JK_ERR_SHAPE for another value. */
+int jk_set_attn_kernel(jk_ctx* ctx, int32_t mode);
 
 /* Diagnostics (the paper has no counterpart): with max_launches > 0 every kernel launch of this
  * context is bracketed by a pair of CUDA events on its stream (up to max_launches launches

@@ -25,7 +25,8 @@ EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", 
            "jk_last_cuda_error", "jk_read_status", "jk_set_tensor_path", "jk_draft_expand",
            "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
            "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
-           "jk_profile_stage_name", "jk_tree_verify_attn_static", "jk_tensor_path_active"]
+           "jk_profile_stage_name", "jk_tree_verify_attn_static", "jk_tensor_path_active",
+           "jk_set_attn_kernel"]
 
 
 class JkConfig(C.Structure):
@@ -70,6 +71,7 @@ def lib() -> C.CDLL:
         L.jk_read_status.argtypes = [vp, vp, C.POINTER(i32)]
         L.jk_set_tensor_path.argtypes = [vp, i32]
         L.jk_tensor_path_active.argtypes = [vp]
+        L.jk_set_attn_kernel.argtypes = [vp, i32]
         L.jk_draft_expand.argtypes = [vp, vp, C.POINTER(JkDraftWeights), i32, i32, i32, vp, vp,
                                       vp, i32, i32, vp, vp, vp, C.POINTER(JkPool), vp, vp, vp,
                                       i64, vp, vp, vp]
@@ -166,6 +168,9 @@ class Context:
             self.close()
         except Exception:
             pass
+
+    def set_attn_kernel(self, mode: int):
+        self._check(lib().jk_set_attn_kernel(self._h, int(mode)), "jk_set_attn_kernel")
 
     def set_tensor_path(self, enable: bool):
         self._check(lib().jk_set_tensor_path(self._h, int(enable)), "jk_set_tensor_path")

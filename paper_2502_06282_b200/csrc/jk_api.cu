@@ -123,6 +123,13 @@ extern "C" int jk_set_tensor_path(jk_ctx* ctx, int32_t enable) {
   return JK_OK;
 }
 
+extern "C" int jk_set_attn_kernel(jk_ctx* ctx, int32_t mode) {
+  if (!ctx) return JK_ERR_NULL;
+  if (mode < 0 || mode > 2) return JK_ERR_SHAPE;
+  ctx->attn_kernel = mode;
+  return JK_OK;
+}
+
 extern "C" const char* jk_strerror(int code) {
   switch (code) {
     case JK_OK: return "ok";

@@ -33,7 +33,7 @@
 
 struct ask_tail {
   uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2], s_empty[2];
-  uint64_t p_full, pv_done, q_full, par_full;
+  uint64_t p_full, pv_done, q_full, par_full, o_ready;
   uint64_t pair[4];                  // the two threads of a row meet here (64 arrivals)
   uint32_t tmem_base;
   int abort_flag;
@@ -144,6 +144,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
     }
     mbar_init(&T.p_full, ASK_SM_THREADS);
     mbar_init(&T.pv_done, 1);
+    mbar_init(&T.o_ready, 1);
     mbar_init(&T.q_full, ASK_SM_THREADS);
     mbar_init(&T.par_full, ASK_SM_THREADS);
     for (int i = 0; i < 4; ++i) mbar_init(&T.pair[i], 64);
@@ -273,6 +274,9 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
           tc_commit(&T.pv_done);
           if (t + 1 < s.tile_hi && !ahead) ok = issue_s(g + 1);
         }
+        // the segment's O is complete: pass that on through a barrier this thread arrives on
+        ok = ok && mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
+        if (ok) mbar_arrive(&T.o_ready);
         x += (uint32_t)(s.tile_hi - s.tile_lo);
       }
     }
@@ -445,7 +449,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
       if (!ok) break;
       // ---- the segment's partial (max, sum, O) of every row
       {
-        const bool okd = mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
+        const bool okd = mbar_wait(&T.o_ready, (uint32_t)seg & 1u, abort_flag, status);
         ok = __all_sync(0xffffffffu, okd);
       }
       if (!ok) break;
@@ -605,8 +609,7 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                       (size_t)ASK_ROWS * ASK_KEYS * 2 + sizeof(ask_tail) + 1024;
   const int n_cta = ctx->sm_count;
   const int ms = L.attn_max_split;
-  const char* mu_env = getenv("JK_ATTN_MINU");
-  const int min_units = mu_env ? atoi(mu_env) : 1;
+  const int min_units = 1;
   JK_PROF(ctx, st, JK_ST_ATTN);
   if (D == 128)
     jk_launch_pdl(k_tree_attn_sk<128>, dim3(n_cta), dim3(ASK_THREADS), smem, st, *mk, *mv,

@@ -370,9 +370,17 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                const int32_t* parent, float scale, void* out) {
   const jk_config& c = ctx->cfg;
   const jk_ws_layout& L = ctx->lay;
-  const char* sk_env = getenv("JK_ATTN_SK");
-  if (sk_env && sk_env[0] == '1' && jk_attn_sk_usable(ctx, B, M, cache_rows))
-    return jk_attn_sk(ctx, st, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale, out);
+  // The persistent kernel wins once every SM has several key tiles to walk; below that its longer
+  // set-up costs more than its pipelining saves.
+  {
+    const int Gq = c.n_q_heads / c.n_kv_heads;
+    const long long units = (long long)B * c.n_kv_heads * ((Gq * M + ATC_ROWS - 1) / ATC_ROWS) *
+                            ((cache_rows + ATC_KEYS - 1) / ATC_KEYS);
+    const bool want = ctx->attn_kernel == 2 ||
+                      (ctx->attn_kernel == 0 && units >= 4ll * ctx->sm_count);
+    if (want && jk_attn_sk_usable(ctx, B, M, cache_rows))
+      return jk_attn_sk(ctx, st, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale, out);
+  }
   const CUtensorMap *mk = nullptr, *mv = nullptr;
   if (jk_attn_tc_maps(ctx, kc, vc, sb, sh, cache_rows, &mk, &mv) != JK_OK) return JK_ERR_CUDA;
   atc_state* s = (atc_state*)ctx->attn_tc_state;

@@ -13,10 +13,11 @@ from tests.jk_testutil import TOL, dev, host, rel_err
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, parent_np, ragged=False, layer=0):
+def _run(w, parent_np, ragged=False, layer=0, kernel=0):
     q, k, v, kv_len = synth.attn_inputs(w, layer, ragged)
     ctx = jk.Context.for_workload(w)
     assert ctx.tensor_path_active == (w.dtype == "bf16")
+    ctx.set_attn_kernel(kernel)
     qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
     out = torch.empty_like(qd)
     ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, dev(kv_len), dev(parent_np),
@@ -48,6 +49,13 @@ def test_attn_tiny(name, kind):
     assert rel_err(got, ref) <= TOL[w.dtype]
 
 
+@pytest.mark.parametrize("kind", ["chain", "star", "binary", "random"])
+def test_attn_tiny_persistent_kernel(kind):
+    w = synth.WORKLOADS["tiny_bf16"]
+    got, ref = _run(w, _trees(w, kind), kernel=2)
+    assert rel_err(got, ref) <= TOL[w.dtype]
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("P,M,Hq,Hkv,d,B", [
     (0, 1, 2, 2, 64, 1),          # empty prefix, single node
@@ -62,8 +70,10 @@ def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype=dtype, prefix=P, tree_size=M,
                      n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, batch=B, depth=6,
                      seed=900 + P + M)
-    got, ref = _run(w, _trees(w, "random"), ragged=True)
-    assert rel_err(got, ref) <= TOL[dtype]
+    # bf16: both tensor-core kernels (1 = CTA per key slice, 2 = persistent); f32: CUDA cores
+    for kernel in ((1, 2) if dtype == "bf16" else (0,)):
+        got, ref = _run(w, _trees(w, "random"), ragged=True, kernel=kernel)
+        assert rel_err(got, ref) <= TOL[dtype], kernel
 
 
 @pytest.mark.parametrize("name,heads,ragged", [
@@ -72,13 +82,16 @@ def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     ("llama3_8b", (0, 17), False),              # GQA 32/8, P = 4096: two query blocks per kv head
     ("llama2_70b_layer", (9, 63), False),       # GQA 64/8, P = 4096: four query blocks per kv head
 ])
-def test_attn_full_shapes_sampled_heads(name, heads, ragged):
-    """Full-size shapes, launch configuration as benchmarked; the oracle checks a few q heads."""
+@pytest.mark.parametrize("kernel", [0, 1, 2])
+def test_attn_full_shapes_sampled_heads(name, heads, ragged, kernel):
+    """Full-size shapes (0 = the kernel the library picks, as benchmarked; 1, 2 = each kernel
+    forced); the oracle checks a few q heads."""
     w = synth.WORKLOADS[name]
     par = _trees(w, "random")
     q, k, v, kv_len = synth.attn_inputs(w, 0, ragged)
     ctx = jk.Context.for_workload(w)
     assert ctx.tensor_path_active
+    ctx.set_attn_kernel(kernel)
     qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
     out = torch.empty_like(qd)
     ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, dev(kv_len), dev(par),
@@ -104,3 +117,17 @@ def test_attn_reports_a_cache_that_is_too_short():
     ctx.tree_verify_attn(1, w.tree_size, qd, kd, vd, bad_len, dev(_trees(w, "chain")), 0.125, out)
     assert ctx.read_status() == jk.ERR["BOUNDS"]
     assert ctx.read_status() == 0          # reading clears it
+
+
+def test_attn_persistent_kernel_reports_a_cache_that_is_too_short():
+    w = synth.WORKLOADS["tiny_bf16"]
+    q, k, v, kv_len = synth.attn_inputs(w)
+    ctx = jk.Context.for_workload(w)
+    ctx.set_attn_kernel(2)
+    qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
+    out = torch.zeros_like(qd)
+    bad_len = dev(np.array([k.shape[2] - w.tree_size + 1] * w.batch, dtype=np.int32))
+    ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, bad_len, dev(_trees(w, "chain")),
+                         0.125, out)
+    assert ctx.read_status() == jk.ERR["BOUNDS"]
+    assert ctx.read_status() == 0
