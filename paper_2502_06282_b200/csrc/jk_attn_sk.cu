@@ -159,7 +159,6 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
   __syncthreads();
   // everything above touches no global memory; kv_len may be the product of the kernel before
   jk_pdl_wait();
-  jk_pdl_trigger();
   for (int i = tid; i < B; i += ASK_THREADS) {
     const int P = kv_len[i];
     const bool bad = P < 0 || P + M > cache_rows;
@@ -488,6 +487,9 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
   }
   tc_fence_before();
   __syncthreads();
+  // Only now may the next kernel of the stream be scheduled: CTAs of a dependent grid that sit
+  // on this SM in their grid-dependency wait were measured to slow this kernel's own warps.
+  jk_pdl_trigger();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);

@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ kv_len,
     const int32_t* __restrict__ parent, float scale, int M, int Hq, int Hkv, int n_split,
     int n_qblk, int cache_rows, float* __restrict__ part_o, float* __restrict__ part_ml,
-    int32_t* __restrict__ counters, __nv_bfloat16* __restrict__ out, int32_t* status) {
+    __nv_bfloat16* __restrict__ out, int32_t* status) {
   constexpr int KB = D / 64;                       // 64-element blocks along d
   constexpr int Q_BYTES = ATC_ROWS * D * 2;
   constexpr int KP_BYTES = 2 * ATC_ROWS * 64 * 2;  // K tile (KB blocks) or P tile (2 blocks)
@@ -71,7 +71,6 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   const int node = row_valid ? (row0 + tid) % M : 0;
   const size_t n_out = (size_t)gridDim.z * M * Hq;
   const size_t orow = ((size_t)b * M + node) * Hq + kvh * G + g_idx;
-  int32_t* counter = counters + ((size_t)b * Hkv + kvh) * n_qblk + qblk;
   const int tiles_total = (Ltot + ATC_KEYS - 1) / ATC_KEYS;
   const int tiles_per = (tiles_total + n_split - 1) / n_split;
   const int t0 = split * tiles_per;
@@ -397,7 +396,6 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                       sizeof(atc_tail) + 1024;
   float* part_o = (float*)(ctx->ws + L.attn_o);
   float* part_ml = (float*)(ctx->ws + L.attn_ml);
-  int32_t* counters = (int32_t*)(ctx->ws + L.attn_cnt);
   int32_t* status = (int32_t*)(ctx->ws + L.status);
   const dim3 grid(n_split * n_qblk, c.n_kv_heads, B);
   if (!s->smem_set) {
@@ -411,12 +409,12 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   if (D == 128)
     jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(128), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                  scale, M, c.n_q_heads, c.n_kv_heads, n_split,
-                                                 n_qblk, cache_rows, part_o, part_ml, counters,
+                                                 n_qblk, cache_rows, part_o, part_ml,
                                                  (__nv_bfloat16*)out, status);
   else
     jk_launch_pdl(k_tree_attn_tc<64>, dim3(grid), dim3(128), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                 scale, M, c.n_q_heads, c.n_kv_heads, n_split,
-                                                n_qblk, cache_rows, part_o, part_ml, counters,
+                                                n_qblk, cache_rows, part_o, part_ml,
                                                 (__nv_bfloat16*)out, status);
   JK_LAUNCH_CHECK(ctx);
   return jk_attn_combine_launch(ctx, st, n_split, (size_t)B * M * c.n_q_heads, out);
