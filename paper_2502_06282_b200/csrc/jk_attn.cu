@@ -241,12 +241,13 @@ int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_o
   const float* part_o = (const float*)(ctx->ws + L.attn_o);
   const float* part_ml = (const float*)(ctx->ws + L.attn_ml);
   JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
+  const dim3 grid((unsigned)((n_out + 7) / 8));
   if (ctx->cfg.head_dim == 128)
-    k_attn_combine<__nv_bfloat16, 128><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(
-        part_o, part_ml, n_split, n_out, (__nv_bfloat16*)out);
+    jk_launch_pdl(k_attn_combine<__nv_bfloat16, 128>, grid, dim3(256), 0, st, part_o, part_ml,
+                  n_split, n_out, (__nv_bfloat16*)out);
   else
-    k_attn_combine<__nv_bfloat16, 64><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(
-        part_o, part_ml, n_split, n_out, (__nv_bfloat16*)out);
+    jk_launch_pdl(k_attn_combine<__nv_bfloat16, 64>, grid, dim3(256), 0, st, part_o, part_ml,
+                  n_split, n_out, (__nv_bfloat16*)out);
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
 }

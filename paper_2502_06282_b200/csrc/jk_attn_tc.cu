@@ -56,12 +56,11 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   const int G = Hq / Hkv;
   const int tid = threadIdx.x, warp = tid >> 5;
   jk_pdl_wait();
-  jk_pdl_trigger();
   const int P = kv_len[b];
   const int Ltot = P + M;
   if (P < 0 || Ltot > cache_rows) {
     if (tid == 0) jk_set_status(status, JK_ERR_BOUNDS);
-    return;
+    return;                                    // (a CTA that exits counts as having released)
   }
   const int n_rows = G * M;
   const int row0 = qblk * ATC_ROWS;
@@ -297,6 +296,9 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
       tmem_dealloc(tmem_base, TMEM_COLS);
     }
   }
+  // Only now may the next kernel of the stream be scheduled: CTAs of a dependent grid that sit on
+  // an SM in their grid-dependency wait were measured to slow the warps still working there.
+  jk_pdl_trigger();
   if (row_valid && ok) {
     part_ml[((size_t)split * n_out + orow) * 2] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
     part_ml[((size_t)split * n_out + orow) * 2 + 1] = l_run;
