@@ -29,6 +29,10 @@ if ROOT not in sys.path:
 METRIC = "draft_verify_steps_per_s"
 UNIT = "steps/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per algorithmic byte of one expert gate/up launch, from the ncu
+# capture summarised in profiles/k_tc_gemm_llama2_7b.txt (366.95 MB moved for 360.71 MB of
+# weights); the traffic is weight bytes plus a few MB, so it scales with the experts touched.
+GATE_UP_TRAFFIC_RATIO = 366.95 / 360.71
 
 
 def parse_args():
@@ -330,7 +334,11 @@ def main():
         kernels[name] = ent
     dom = max((k for k in kernels if "GBps" in kernels[k]), key=lambda k: kernels[k]["ms_per_step"])
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak,
-                "unit": "GB/s", "frac": kernels[dom]["frac_of_peak"], "traffic": None,
+                "unit": "GB/s", "frac": kernels[dom]["frac_of_peak"],
+                "traffic": (GATE_UP_TRAFFIC_RATIO * algo_bytes_per_step[dom]
+                            / kernels[dom]["launches_per_step"]) if dom == "expert_gate_up" else None,
+                "traffic_source": ("ncu capture of a two-expert launch, scaled by the weight bytes "
+                                   "of an average launch" if dom == "expert_gate_up" else None),
                 "peak_source": f"of {peak_src}",
                 "algo_bytes_per_launch": algo_bytes_per_step[dom] / kernels[dom]["launches_per_step"],
                 "us_per_launch": kernels[dom]["us_per_launch"]}
