@@ -64,7 +64,6 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->attn_max_split = ms;
   L->attn_o = take(rows * c.head_dim * 4 * ms);
   L->attn_ml = take(rows * 2 * 4 * ms);
-  L->attn_cnt = take((size_t)c.max_batch * c.n_q_heads * 4);
   L->rs_arg = take(BM * 4);
   L->rs_max = take(BM * 4);
   L->rs_sum = take(BM * 4);
@@ -110,10 +109,6 @@ extern "C" int jk_set_workspace(jk_ctx* ctx, void* stream, void* dev_ptr, size_t
   ctx->ws_bytes = bytes;
   jk_tc_destroy(ctx);   // tensor maps over an earlier workspace are stale
   JK_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 16, (cudaStream_t)stream));
-  // arrival counters of the attention kernel start at zero and return to zero after every call
-  JK_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0,
-                                     (size_t)ctx->cfg.max_batch * ctx->cfg.n_q_heads * 4,
-                                     (cudaStream_t)stream));
   return JK_OK;
 }
 

@@ -34,14 +34,13 @@ struct jk_ws_layout {
   size_t gemm_part;     // f32 partial tiles of the tensor-core GEMMs
   size_t attn_o;        // f32 [split, B*M*Hq, d]
   size_t attn_ml;       // f32 [split, B*M*Hq, 2]
-  size_t attn_cnt;      // i32 [B, Hkv, query blocks] arrival counters (zero between calls)
   size_t rs_arg;        // i32 [B, M]        per tree node: top-1 token of the target row
   size_t rs_max;        // f32 [B, M]
   size_t rs_sum;        // f32 [B, M]
   size_t pbuf;          // f32 [B, V]
   size_t qbuf;          // f32 [B, K, V]
   size_t p_old;         // i32 [B]
-  size_t qs_arg;        // i32 [B, S, K]     (unused top-1 of the draft rows)
+  size_t qs_arg;        // i32 [B, S, K]     top-1 of every stored draft row (written, not read)
   size_t qs_max;        // f32 [B, S, K]     max of every stored draft logits row
   size_t qs_sum;        // f32 [B, S, K]     its sum of exp((x - max)/T)
   size_t total;
