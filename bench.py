@@ -164,7 +164,8 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.layers:
         w = synth.scaled(w, n_layers=args.layers)
-    w = synth.scaled(w, seed=w.seed + 17 * rank)       # every rank drafts its own sequences
+    from paper_2502_06282_b200 import replicas
+    w = replicas.rank_workload(w, rank)                # every rank drafts its own sequences
     config = {"workload": f"{w.name}: H={w.hidden} I={w.inter} V={w.vocab} N={w.n_experts} "
                           f"K={w.top_k} heads={w.n_q_heads}/{w.n_kv_heads}x{w.head_dim} "
                           f"P={w.prefix} M={w.tree_size} D={w.depth} k_e={w.k_per_expert} "
@@ -301,12 +302,9 @@ def main():
     ctx.profile_enable(0)
     assert ctx.read_status() == 0, "device status word reports an error"
     n_acc = int(bufs.n_acc[0])
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(ms, "cuda")
     ms_per_step = ms / args.steps
-    value = world * 1000.0 / ms_per_step
+    value = replicas.job_steps_per_s(world, ms_per_step)
 
     # ---------------------------------------------------------------- per-kernel roofline
     peak, peak_src = measured_peaks()
@@ -401,11 +399,8 @@ def main():
         e1.record()
         barrier()
         ms_e = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms_e], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e = float(t.item())
-        e2e = {"value": world * 1000.0 * n_e2e / ms_e, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        ms_e = replicas.max_over_ranks(ms_e, "cuda")
+        e2e = {"value": replicas.job_steps_per_s(world, ms_e / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": n_e2e,
                "pipelining": "inputs double-buffered; copies of step s+1 overlap step s"}
 
