@@ -65,6 +65,8 @@ def test_attn_tiny_persistent_kernel(kind):
     (777, 60, 16, 2, 128, 2),     # GQA 8: several query blocks per kv head
     (1500, 60, 32, 32, 128, 2),   # many heads: each CTA walks several key tiles (running max)
     (900, 33, 16, 16, 64, 3),     # the same with head size 64
+    (8192, 128, 8, 2, 128, 2),    # the longest prefix and largest tree of the sweep: 65 key tiles
+    (4096, 64, 8, 8, 64, 8),      # batch 8, ragged lengths, head size 64
 ])
 def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype=dtype, prefix=P, tree_size=M,
