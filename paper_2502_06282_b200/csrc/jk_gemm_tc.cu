@@ -437,7 +437,7 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
 
 // logits = b W_head^T (Eq. 4) assembled from the partial tiles, optionally stored, and the
 // per-chunk top-k statistics of jk_topk.cuh.   grid (chunks, logits rows), JK_TOPK_THREADS threads.
-__global__ void __launch_bounds__(JK_TOPK_THREADS) k_tc_fix_lmhead_topk(
+__global__ void __launch_bounds__(JK_TOPK_THREADS, 2) k_tc_fix_lmhead_topk(
     const tc_params p, int n_cta, int V, int k_e, int chunks, const float* __restrict__ partial,
     float* __restrict__ logits, int rows_per_b, long long stride_b, float* __restrict__ tk_val,
     int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {

@@ -12,7 +12,7 @@
 
 #include "jk_common.cuh"
 
-#define JK_TOPK_THREADS 1024
+#define JK_TOPK_THREADS 512
 #define JK_TOPK_WARPS (JK_TOPK_THREADS / 32)
 #define JK_TOPK_PER (JK_TOPK_CHUNK / JK_TOPK_THREADS)
 
