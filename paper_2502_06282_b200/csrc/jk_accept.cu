@@ -11,18 +11,12 @@
 // tree node.
 // ------------------------------------------------------------------------------------------
 template <typename TL>
-__global__ void __launch_bounds__(512) k_row_stats(const TL* __restrict__ tl, int V, float inv_t,
-                                                   int32_t* __restrict__ rs_arg,
-                                                   float* __restrict__ rs_max,
-                                                   float* __restrict__ rs_sum) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
+__device__ __forceinline__ void row_stats_row(const TL* __restrict__ r, size_t row, int V,
+                                              float inv_t, int32_t* __restrict__ rs_arg,
+                                              float* __restrict__ rs_max,
+                                              float* __restrict__ rs_sum, float* red, float* wv,
+                                              int* wi) {
   constexpr int VN = jk_vec<TL>::N;
-  __shared__ float red[33];
-  __shared__ float wv[16];
-  __shared__ int wi[16];
-  const size_t row = blockIdx.x;
-  const TL* r = tl + row * V;
   float bv = -INFINITY;
   int bi = INT_MAX;
   const int vmain = V / VN * VN;
@@ -61,6 +55,27 @@ __global__ void __launch_bounds__(512) k_row_stats(const TL* __restrict__ tl, in
     s += expf((jk_to_float(r[k]) - mx) * inv_t);
   s = jk_block_sum(s, red);
   if (threadIdx.x == 0) { rs_arg[row] = am; rs_max[row] = mx; rs_sum[row] = s; }
+}
+
+// Blocks 0 .. rows-1 take the target rows, the rest (sampling mode) the stored draft rows: one
+// launch for both sets.
+template <typename TL>
+__global__ void __launch_bounds__(512) k_row_stats(
+    const TL* __restrict__ tl, int rows, const float* __restrict__ dl, int V, float inv_t,
+    int32_t* __restrict__ rs_arg, float* __restrict__ rs_max, float* __restrict__ rs_sum,
+    int32_t* __restrict__ qs_arg, float* __restrict__ qs_max, float* __restrict__ qs_sum) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  __shared__ float red[33];
+  __shared__ float wv[16];
+  __shared__ int wi[16];
+  if ((int)blockIdx.x < rows) {
+    const size_t row = blockIdx.x;
+    row_stats_row<TL>(tl + row * V, row, V, inv_t, rs_arg, rs_max, rs_sum, red, wv, wi);
+  } else {
+    const size_t row = blockIdx.x - rows;
+    row_stats_row<float>(dl + row * V, row, V, inv_t, qs_arg, qs_max, qs_sum, red, wv, wi);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -414,22 +429,20 @@ extern "C" int jk_accept_and_compact(
   int32_t* status = (int32_t*)(ws + L.status);
   const float inv_t = mode == 1 ? 1.f / temperature : 1.f;
   const int rows = batch * tree_size;
+  // max and sum of exp of every stored draft row too (sampling), before the serial walk
+  const int q_rows = mode == 1 ? batch * n_slots * c.top_k : 0;
   JK_PROF(ctx, st, JK_ST_ROWSTATS);
   if (tl_dtype == JK_BF16)
-    jk_launch_pdl(k_row_stats<__nv_bfloat16>, dim3(rows), dim3(512), 0, st, (const __nv_bfloat16*)target_logits, c.vocab,
-                                                     inv_t, rs_arg, rs_max, rs_sum);
+    jk_launch_pdl(k_row_stats<__nv_bfloat16>, dim3(rows + q_rows), dim3(512), 0, st,
+                  (const __nv_bfloat16*)target_logits, rows, draft_logits, c.vocab, inv_t, rs_arg,
+                  rs_max, rs_sum, (int32_t*)(ws + L.qs_arg), (float*)(ws + L.qs_max),
+                  (float*)(ws + L.qs_sum));
   else
-    jk_launch_pdl(k_row_stats<float>, dim3(rows), dim3(512), 0, st, (const float*)target_logits, c.vocab, inv_t, rs_arg,
-                                             rs_max, rs_sum);
+    jk_launch_pdl(k_row_stats<float>, dim3(rows + q_rows), dim3(512), 0, st,
+                  (const float*)target_logits, rows, draft_logits, c.vocab, inv_t, rs_arg, rs_max,
+                  rs_sum, (int32_t*)(ws + L.qs_arg), (float*)(ws + L.qs_max),
+                  (float*)(ws + L.qs_sum));
   JK_LAUNCH_CHECK(ctx);
-  if (mode == 1) {
-    // max and sum of exp of every stored draft row, in parallel, before the serial walk
-    JK_PROF(ctx, st, JK_ST_ROWSTATS);
-    jk_launch_pdl(k_row_stats<float>, dim3(batch * n_slots * c.top_k), dim3(512), 0, st, 
-        draft_logits, c.vocab, inv_t, (int32_t*)(ws + L.qs_arg), (float*)(ws + L.qs_max),
-        (float*)(ws + L.qs_sum));
-    JK_LAUNCH_CHECK(ctx);
-  }
   walk_out o{kv_len, (int32_t*)(ws + L.p_old), n_acc, acc_idx, acc_tok, bonus_tok};
   JK_PROF(ctx, st, JK_ST_WALK);
   if (mode == 0) {
