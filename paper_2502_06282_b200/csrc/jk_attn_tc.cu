@@ -6,9 +6,10 @@
 // tiles.  Per tile of 128 keys:
 //   TMA brings K [128 keys x d] and V [128 keys x d] into swizzled shared memory;
 //   S = Q K^T on the tensor core into tensor memory (128 x 128 fp32);
-//   every thread owns one query row: it reads its row of S, applies the tree mask (a 128-bit
-//   visibility word built from the node's ancestor set and the prefix length), keeps a running
-//   max and sum, and writes P = exp(S - max) as bf16 into the shared memory K just left;
+//   two threads own one query row: each reads the whole row of S for the maximum (so the two agree
+//   without an exchange), applies the tree mask (a 128-bit visibility word built from the node's
+//   ancestor set and the prefix length), keeps the running max and the sum of its 64 keys, and
+//   writes P = exp(S - max) for those keys as bf16 into the shared memory K just left;
 //   O (+)= P V on the tensor core, V taken MN-major straight from its row-major tile; when the
 //   running max moved, O is first rescaled in tensor memory.
 // The CTA writes an unnormalised partial (max, sum, O) per row; the merge kernel of jk_attn.cu
@@ -28,10 +29,13 @@ struct atc_tail {
   uint32_t tmem_base;
   int abort_flag;
   int parent[JK_MAX_TREE];
+  float xsum[2][ATC_ROWS];             // [key half][row]: the half's sum of exponentials
 };
 
+#define ATC_THREADS 256
+
 template <int D>
-__global__ void __launch_bounds__(128) k_tree_attn_tc(
+__global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
     const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ kv_len,
     const int32_t* __restrict__ parent, float scale, int M, int Hq, int Hkv, int n_split,
@@ -54,7 +58,10 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   const int split = blockIdx.x % n_split, qblk = blockIdx.x / n_split;
   const int kvh = blockIdx.y, b = blockIdx.z;
   const int G = Hq / Hkv;
+  // two threads per query row: tensor-memory lane quarter = warp % 4, key half = warp / 4
   const int tid = threadIdx.x, warp = tid >> 5;
+  const int quarter = warp & 3, half = warp >> 2;
+  const int row = quarter * 32 + (tid & 31);
   jk_pdl_wait();
   const int P = kv_len[b];
   const int Ltot = P + M;
@@ -64,10 +71,10 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   }
   const int n_rows = G * M;
   const int row0 = qblk * ATC_ROWS;
-  const bool row_valid = row0 + tid < n_rows;
-  const bool warp_has_rows = row0 + (tid & ~31) < n_rows;
-  const int g_idx = row_valid ? (row0 + tid) / M : 0;
-  const int node = row_valid ? (row0 + tid) % M : 0;
+  const bool row_valid = row0 + row < n_rows;
+  const bool warp_has_rows = row0 + quarter * 32 < n_rows;
+  const int g_idx = row_valid ? (row0 + row) / M : 0;
+  const int node = row_valid ? (row0 + row) % M : 0;
   const size_t n_out = (size_t)gridDim.z * M * Hq;
   const size_t orow = ((size_t)b * M + node) * Hq + kvh * G + g_idx;
   const int tiles_total = (Ltot + ATC_KEYS - 1) / ATC_KEYS;
@@ -105,11 +112,11 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
     if (tid < M) T.parent[tid] = parent[(size_t)b * M + tid];
     // Q block -> shared memory in the K-major 128-byte-swizzled layout the MMA reads
     // (all loads are issued before the first store, so that they overlap)
-    constexpr int QV = ATC_ROWS * (D / 8) / 128;   // 16-byte vectors per thread
+    constexpr int QV = ATC_ROWS * (D / 8) / ATC_THREADS;   // 16-byte vectors per thread
     uint4 qv[QV];
 #pragma unroll
     for (int it = 0; it < QV; ++it) {
-      const int idx = tid + it * 128;
+      const int idx = tid + it * ATC_THREADS;
       const int rr = idx / (D / 8), ch = idx % (D / 8);
       qv[it] = make_uint4(0u, 0u, 0u, 0u);
       if (row0 + rr < n_rows) {
@@ -120,7 +127,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
     }
 #pragma unroll
     for (int it = 0; it < QV; ++it) {
-      const int idx = tid + it * 128;
+      const int idx = tid + it * ATC_THREADS;
       const int rr = idx / (D / 8), ch = idx % (D / 8);
       const int kb = ch >> 3, cb = ch & 7;
       *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = qv[it];
@@ -140,7 +147,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
         c = (pp < c) ? pp : -1;
       }
     }
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const uint32_t idesc_s = instr_desc_bf16_ex(ATC_KEYS, 0);
     const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
     const float sl2 = scale * 1.4426950408889634f;
@@ -188,63 +195,69 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
       // (warps whose 32 rows all lie past the last query row skip the row work: their rows of P
       // and O are never stored)
       if (warp_has_rows) {
-      // the whole row of S in registers: one round of tensor-memory loads
-      uint32_t s0[32], s1[32], s2[32], s3[32];
-      tmem_ld32(tmem_base + lane_base + 0u, s0);
-      tmem_ld32(tmem_base + lane_base + 32u, s1);
-      tmem_ld32(tmem_base + lane_base + 64u, s2);
-      tmem_ld32(tmem_base + lane_base + 96u, s3);
-      tmem_ld_wait();
-      const unsigned b0 = (unsigned)vis_lo, b1 = (unsigned)(vis_lo >> 32);
-      const unsigned b2 = (unsigned)vis_hi, b3 = (unsigned)(vis_hi >> 32);
-      float mx = -INFINITY;
+        // pass 1: the row maximum over all 128 keys.  Both threads of a row compute it from the
+        // same values in the same order, so they agree bit for bit without an exchange.
+        float mx = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s0[j]));
-        if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s1[j]));
-        if ((b2 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s2[j]));
-        if ((b3 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(s3[j]));
-      }
-      const float m_new = fmaxf(m_run, mx);
-      const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
-                                               : fast_exp2((m_run - m_new) * sl2);
-      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-      float lsum = 0.f;
-      auto emit = [&](const uint32_t (&sr)[32], unsigned bits, int c) {
-        uint32_t packed[16];
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(sr[j]) - m_use) * sl2) : 0.f;
-          const float p1 = ((bits >> (j + 1)) & 1u)
-                               ? fast_exp2((__uint_as_float(sr[j + 1]) - m_use) * sl2) : 0.f;
-          lsum += p0 + p1;
-          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-          packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h);
-        }
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const int ch = c * 4 + jj;             // 16-byte chunk of the 128-key row
-          const int kb = ch >> 3, cb = ch & 7;
-          *reinterpret_cast<uint4*>(skp + kb * 16384 + tid * 128 + ((cb ^ (tid & 7)) << 4)) =
-              make_uint4(packed[4 * jj], packed[4 * jj + 1], packed[4 * jj + 2], packed[4 * jj + 3]);
-        }
-      };
-      emit(s0, b0, 0); emit(s1, b1, 1); emit(s2, b2, 2); emit(s3, b3, 3);
-      l_run = l_run * alpha + lsum;
-      m_run = m_new;
-      // rescale the running output when some row of this warp moved its maximum
-      if (tile > t0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+        for (int hh = 0; hh < 4; ++hh) {
+          uint32_t r0[32];
+          tmem_ld32(tmem_base + lane_base + (uint32_t)(hh * 32), r0);
           tmem_ld_wait();
+          const unsigned long long v = (hh & 2) ? vis_hi : vis_lo;
+          const unsigned b0 = (hh & 1) ? (unsigned)(v >> 32) : (unsigned)v;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-          tmem_st32(tmem_base + lane_base + O_COL + (uint32_t)(c * 32), r);
+          for (int j = 0; j < 32; ++j)
+            if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
         }
-        tmem_st_wait();
-      }
+        const float m_new = fmaxf(m_run, mx);
+        const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
+                                                 : fast_exp2((m_run - m_new) * sl2);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        // pass 2: P = exp(S - max) as bf16 for this thread's 64 keys, over the K tile (S, its only
+        // reader, has completed)
+        float lsum = 0.f;
+        unsigned char* prow = skp + half * 16384 + row * 128;
+        const unsigned long long vh = half ? vis_hi : vis_lo;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + lane_base + (uint32_t)(half * 64 + hh * 32), r);
+          tmem_ld_wait();
+          const unsigned bits = hh ? (unsigned)(vh >> 32) : (unsigned)vh;
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(r[j]) - m_use) * sl2) : 0.f;
+            const float p1 = ((bits >> (j + 1)) & 1u)
+                                 ? fast_exp2((__uint_as_float(r[j + 1]) - m_use) * sl2) : 0.f;
+            lsum += p0 + p1;
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            const int cb = hh * 4 + cc;
+            *reinterpret_cast<uint4*>(prow + ((cb ^ (row & 7)) << 4)) =
+                make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+          }
+        }
+        l_run = l_run * alpha + lsum;
+        m_run = m_new;
+        // rescale this thread's half of the running output when some row of the warp moved its
+        // maximum (the previous tile's P V product has completed: the loop waits for it)
+        if (tile > t0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+          for (int c = 0; c < D / 64; ++c) {
+            uint32_t r[32];
+            const uint32_t oa = tmem_base + lane_base + O_COL + (uint32_t)(half * (D / 2) + c * 32);
+            tmem_ld32(oa, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+            tmem_st32(oa, r);
+          }
+          tmem_st_wait();
+        }
       }
       fence_proxy_async_smem();
       tc_fence_before();
@@ -268,13 +281,12 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
       if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
     }
     if (ok) {
-      float* po = part_o + ((size_t)split * n_out + orow) * D;
-      const uint32_t lane_base2 = (uint32_t)(warp * 32) << 16;
+      float* po = part_o + ((size_t)split * n_out + orow) * D + half * (D / 2);
 #pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < D / 64; ++c) {
         uint32_t r[32];
         if (!warp_has_rows) break;
-        tmem_ld32(tmem_base + lane_base2 + O_COL + (uint32_t)(c * 32), r);
+        tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(half * (D / 2) + c * 32), r);
         tmem_ld_wait();
         if (row_valid) {
 #pragma unroll
@@ -289,6 +301,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
       const unsigned long long ts = global_ns();
       while (global_ns() - ts < 2000000ull) { /* 2 ms: far longer than any TMA copy */ }
     }
+    T.xsum[half][row] = l_run;
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -299,9 +312,9 @@ __global__ void __launch_bounds__(128) k_tree_attn_tc(
   // Only now may the next kernel of the stream be scheduled: CTAs of a dependent grid that sit on
   // an SM in their grid-dependency wait were measured to slow the warps still working there.
   jk_pdl_trigger();
-  if (row_valid && ok) {
+  if (row_valid && ok && half == 0) {
     part_ml[((size_t)split * n_out + orow) * 2] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
-    part_ml[((size_t)split * n_out + orow) * 2 + 1] = l_run;
+    part_ml[((size_t)split * n_out + orow) * 2 + 1] = have_keys ? l_run + T.xsum[1][row] : 0.f;
   }
 }
 
@@ -409,12 +422,12 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   }
   JK_PROF(ctx, st, JK_ST_ATTN);
   if (D == 128)
-    jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(128), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+    jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(ATC_THREADS), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                  scale, M, c.n_q_heads, c.n_kv_heads, n_split,
                                                  n_qblk, cache_rows, part_o, part_ml,
                                                  (__nv_bfloat16*)out, status);
   else
-    jk_launch_pdl(k_tree_attn_tc<64>, dim3(grid), dim3(128), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+    jk_launch_pdl(k_tree_attn_tc<64>, dim3(grid), dim3(ATC_THREADS), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                 scale, M, c.n_q_heads, c.n_kv_heads, n_split,
                                                 n_qblk, cache_rows, part_o, part_ml,
                                                 (__nv_bfloat16*)out, status);
