@@ -402,7 +402,8 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   const int n_qblk = (G * M + ATC_ROWS - 1) / ATC_ROWS;
   const int base = n_qblk * c.n_kv_heads * B;
   const int tiles_max = (cache_rows + ATC_KEYS - 1) / ATC_KEYS;
-  int n_split = (2 * ctx->sm_count + base - 1) / base;
+  // as many key slices as keep all CTAs resident at once (two per SM): one wave
+  int n_split = (2 * ctx->sm_count) / base;
   if (n_split > tiles_max) n_split = tiles_max;
   if (n_split > L.attn_max_split) n_split = L.attn_max_split;
   if (n_split < 1) n_split = 1;
