@@ -64,8 +64,7 @@ __global__ void __launch_bounds__(512) k_row_stats(
     const TL* __restrict__ tl, int rows, const float* __restrict__ dl, int V, float inv_t,
     int32_t* __restrict__ rs_arg, float* __restrict__ rs_max, float* __restrict__ rs_sum,
     int32_t* __restrict__ qs_arg, float* __restrict__ qs_max, float* __restrict__ qs_sum) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
+  jk_pdl_wait();      // (its dependent is released when this kernel's CTAs exit: measured faster)
   __shared__ float red[33];
   __shared__ float wv[16];
   __shared__ int wi[16];
@@ -110,8 +109,7 @@ __global__ void __launch_bounds__(128) k_walk_greedy(
     int M, int max_depth, int V, const int32_t* __restrict__ tok,
     const int32_t* __restrict__ parent, const int32_t* __restrict__ rs_arg, walk_out o,
     int cache_rows, int32_t* status) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
+  jk_pdl_wait();      // (its dependent is released when this kernel's CTAs exit: measured faster)
   __shared__ int s_next;
   __shared__ int path[16], path_tok[16];
   const int b = blockIdx.x;
@@ -153,8 +151,7 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     const float* __restrict__ rs_sum, const float* __restrict__ qs_max,
     const float* __restrict__ qs_sum, float* __restrict__ pbuf_all, float* __restrict__ qbuf_all,
     walk_out o, int cache_rows, int32_t* status) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
+  jk_pdl_wait();      // (its dependent is released when this kernel's CTAs exit: measured faster)
   __shared__ float red[66];
   __shared__ int s_parent[JK_MAX_TREE], s_tok[JK_MAX_TREE], s_branch[JK_MAX_TREE];
   __shared__ int kids[JK_MAX_TREE];
@@ -364,8 +361,7 @@ __global__ void __launch_bounds__(256) k_compact(
     long long stride_b, long long stride_h, int row_bytes, int cache_rows, int max_depth, int M,
     const int32_t* __restrict__ p_old, const int32_t* __restrict__ n_acc,
     const int32_t* __restrict__ acc_idx, int elem_size) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
+  jk_pdl_wait();      // (its dependent is released when this kernel's CTAs exit: measured faster)
   const int which = blockIdx.z;                  // layer*2 + (0 = K, 1 = V)
   const int b = blockIdx.y, kvh = blockIdx.x;
   const int n = n_acc[b];
