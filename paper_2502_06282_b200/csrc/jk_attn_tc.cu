@@ -281,19 +281,37 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
     }
     if (ok) {
-      float* po = part_o + ((size_t)split * n_out + orow) * D + half * (D / 2);
+      // The partial O goes through shared memory (over the K/P and V tiles: every MMA has
+      // completed) so that it leaves in whole 512-byte rows: a thread per row storing straight
+      // from its registers would touch 32 different rows with every store instruction.
+      // 16-byte chunk c of row t sits at chunk index c * 128 + (t ^ c), which the row-per-lane
+      // writes and the chunk-per-lane reads both reach without bank conflicts.
+      float4* so4 = reinterpret_cast<float4*>(skp);
+      constexpr int NC4 = D / 4;                       // chunks of a row
+      if (warp_has_rows) {
 #pragma unroll 1
-      for (int c = 0; c < D / 64; ++c) {
-        uint32_t r[32];
-        if (!warp_has_rows) break;
-        tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(half * (D / 2) + c * 32), r);
-        tmem_ld_wait();
-        if (row_valid) {
+        for (int c = 0; c < D / 64; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + lane_base + O_COL + (uint32_t)(half * (D / 2) + c * 32), r);
+          tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            *reinterpret_cast<float4*>(po + c * 32 + j) =
-                make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                            __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+          for (int j = 0; j < 8; ++j) {
+            const int c4 = half * (NC4 / 2) + c * 8 + j;
+            so4[c4 * ATC_ROWS + (row ^ (c4 & 31))] =
+                make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                            __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+          }
+        }
+      }
+      __syncthreads();
+      const int lane = tid & 31;
+      const int rows_here = min(ATC_ROWS, n_rows - row0);
+      if (lane < NC4) {
+        for (int r = warp; r < rows_here; r += ATC_THREADS / 32) {
+          const int gg = (row0 + r) / M, ii = (row0 + r) % M;
+          const size_t orr = ((size_t)b * M + ii) * Hq + kvh * G + gg;
+          *reinterpret_cast<float4*>(part_o + ((size_t)split * n_out + orr) * D + lane * 4) =
+              so4[lane * ATC_ROWS + (r ^ (lane & 31))];
         }
       }
     } else if (tid == 0) {
