@@ -535,12 +535,30 @@ __global__ void __launch_bounds__(256) k_attn_combine_sk(
   const uint32_t item = (uint32_t)((head / G) * n_qblk + ((head % G) * M + node) / ASK_ROWS);
   const uint32_t start = base + item * Tb;
   const int n_split = (int)(ask_owner(start + Tb - 1u, pl) - ask_owner(start, pl)) + 1;
+  const float* po = part_o + row * D + lane * DPL;      // partial s is s * n_out * D further
+  const size_t sstride = n_out * D;
+  auto load_batch = [&](int s0, float (&v)[4][DPL]) {   // four independent vector loads in flight
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int s = s0 + j < n_split ? s0 + j : n_split - 1;
+      if (DPL == 4) {
+        const float4 x = *reinterpret_cast<const float4*>(po + (size_t)s * sstride);
+        v[j][0] = x.x; v[j][1] = x.y; v[j][DPL - 2] = x.z; v[j][DPL - 1] = x.w;
+      } else {
+        const float2 x = *reinterpret_cast<const float2*>(po + (size_t)s * sstride);
+        v[j][0] = x.x; v[j][DPL - 1] = x.y;
+      }
+    }
+  };
+  // the first batch of partial outputs is asked for before anything waits on the (max, sum) pairs
+  float v[4][DPL];
+  load_batch(0, v);
   // lane s holds (max, sum) of partial s (n_split < 32); one load round for all partials
   float ms = -INFINITY, ls = 0.f;
   if (lane < n_split) {
-    const float2 v = *reinterpret_cast<const float2*>(part_ml + ((size_t)lane * n_out + row) * 2);
-    ms = v.x;
-    ls = v.y;
+    const float2 x = *reinterpret_cast<const float2*>(part_ml + ((size_t)lane * n_out + row) * 2);
+    ms = x.x;
+    ls = x.y;
   }
   const float m = jk_warp_max(ms);
   const float w_lane = (ms == -INFINITY) ? 0.f : __expf(ms - m);
@@ -549,14 +567,7 @@ __global__ void __launch_bounds__(256) k_attn_combine_sk(
 #pragma unroll
   for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
   for (int s0 = 0; s0 < n_split; s0 += 4) {
-    float v[4][DPL];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {                 // four independent loads in flight
-      const int s = s0 + j;
-#pragma unroll
-      for (int t = 0; t < DPL; ++t)
-        v[j][t] = s < n_split ? part_o[((size_t)s * n_out + row) * D + lane * DPL + t] : 0.f;
-    }
+    if (s0 > 0) load_batch(s0, v);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float w = __shfl_sync(0xffffffffu, w_lane, (s0 + j) & 31);
