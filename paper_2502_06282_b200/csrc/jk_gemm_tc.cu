@@ -625,12 +625,6 @@ static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUten
   return JK_OK;
 }
 
-static int tc_zdim(int base_blocks, int n_rows, int n_cta) {
-  int z = 1;
-  while (z < n_rows && base_blocks * z < 2 * n_cta) z <<= 1;
-  return z;
-}
-
 // Expert FFNs of the draft layer (Eq. 3) on the tensor core: gate/up GEMM, SiLU * up, down GEMM,
 // then the combined feature and the branch features (LM-head input).
 int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
