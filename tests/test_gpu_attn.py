@@ -133,3 +133,23 @@ def test_attn_persistent_kernel_reports_a_cache_that_is_too_short():
                          0.125, out)
     assert ctx.read_status() == jk.ERR["BOUNDS"]
     assert ctx.read_status() == 0
+
+
+@pytest.mark.parametrize("kernel", [1, 2])
+def test_attn_is_bitwise_reproducible(kernel):
+    """Slices are merged in a fixed order: two calls on the same inputs give the same bits."""
+    w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype="bf16", prefix=1500, tree_size=60,
+                     n_q_heads=32, n_kv_heads=8, head_dim=128, batch=2, depth=6, seed=77)
+    q, k, v, kv_len = synth.attn_inputs(w, 0, True)
+    ctx = jk.Context.for_workload(w)
+    ctx.set_attn_kernel(kernel)
+    qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
+    par, kvd = dev(_trees(w, "random")), dev(kv_len)
+    outs = []
+    for _ in range(2):
+        out = torch.empty_like(qd)
+        ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, kvd, par, 1.0 / math.sqrt(w.head_dim), out)
+        torch.cuda.synchronize()
+        outs.append(out.view(torch.int16).cpu())
+    assert ctx.read_status() == 0
+    assert torch.equal(outs[0], outs[1])
