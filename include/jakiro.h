@@ -53,8 +53,10 @@ typedef enum {
 
 typedef enum { JK_F32 = 0, JK_BF16 = 1 } jk_dtype;
 
-/* Limits: top_k <= n_experts <= 8, k_per_expert <= 16, max_tree <= 128,
- * max_batch * max_frontier <= 128, head_dim 64 or 128, hidden/inter multiples of 8. */
+/* Limits: top_k <= n_experts <= 8, k_per_expert <= 16, max_tree <= 128, max_depth <= 16,
+ * max_batch * max_frontier <= 128, head_dim 64 or 128, hidden/inter multiples of 8,
+ * ceil(vocab / 4096) * k_per_expert <= 512; a step's candidate pool holds at most 4096 entries
+ * per sequence. */
 typedef struct {
   int32_t hidden, n_experts, top_k, inter, vocab;
   int32_t n_q_heads, n_kv_heads, head_dim;
@@ -204,7 +206,10 @@ int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_s
 
 /*
  * jk_tree_verify_attn for callers that cannot allocate device memory.  (The paper has no
- * counterpart: this is a packaging variant of the call above, same arithmetic.)
+ * counterpart: this is a packaging variant of the call above.  It computes the same operation
+ * with the CUDA-core kernel for both dtypes - fp32 products and an fp32 softmax - where
+ * jk_tree_verify_attn uses the tensor-core kernels for bf16, which round the softmax weights to
+ * bf16 and run several times faster; the two agree within the bf16 tolerance, not bit for bit.)
  *
  * Meant for processes that have given all free HBM to their own pools at start-up, so that a
  * later cudaMalloc for a workspace fails, and for decode loops that cannot afford the
@@ -214,19 +219,20 @@ int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_s
  * uses no allocating library routine.
  *
  *   Arguments as jk_tree_verify_attn, plus
- *   status   i32 [1] device, optional: receives JK_ERR_BOUNDS if kv_len[b] + M > cache_rows
- *            (atomic compare-and-swap on 0, so the caller clears it); with NULL the error is
- *            only recorded inside the built-in array, which the next call clears.
+ *   status   i32 [1] device, required (NULL returns JK_ERR_NULL): receives JK_ERR_BOUNDS if
+ *            kv_len[b] + M > cache_rows, in which case `out` is not written.  It is set by an
+ *            atomic compare-and-swap on 0, so the caller clears it before the call and reads it
+ *            after synchronising the stream.
  *   Limit    batch * tree_size * n_q_heads * (head_dim + 2) * 4 bytes <= 8 MiB (e.g. 60 nodes x
  *            32 heads x 128 uses 1 MiB per key slice); beyond it the call returns
  *            JK_ERR_CAPACITY, launches nothing, and jk_last_cuda_error(ctx) says why.
  *   Set-up   the first call on each device (with that device current) looks up the array's
  *            device address; make that first call before starting any stream capture.
  *   Sharing  all contexts, streams and threads of the process share the one array per GPU, and
- *            it keeps the previous call's contents.  Nothing in it has to start at zero except
- *            the internal status word, which the call clears itself; but two of these calls
- *            that overlap on the same GPU race on the partials and give wrong results: run
- *            them one after the other.
+ *            it keeps the previous call's contents.  Nothing in it has to start at zero (every
+ *            partial a call reads it has written itself); but two of these calls that overlap
+ *            on the same GPU race on the partials and give wrong results: run them one after
+ *            the other.
  */
 int jk_tree_verify_attn_static(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
                                const void* q, const void* k_cache, const void* v_cache,

@@ -8,8 +8,8 @@ step of the paper after the other, with no blocking, fusion or reordering.
 
 What each function follows:
 
-  rmsnorm               the layer norm the paper leaves out of Eq. 1-5 "for
-                        brevity" (Sec. 3.1.2); read as a LLaMA-style pre-MLP
+  rmsnorm               the layer norm that Eq. 1-5 leave out (Sec. 3.1.2, the
+                        note after Eq. 5); read as a LLaMA-style pre-MLP
                         RMSNorm in front of router and experts
   router_scores         Eq. 2: softmax over the N expert centroids
   topk_gate             Eq. 5: the K largest scores keep their value, the rest
@@ -19,7 +19,8 @@ What each function follows:
                         f^top1, f^top2 that Eq. 4 and Eq. 6 feed to the head
   head_logits           Eq. 4: the LM head shared with the target model
   branch_topk           per-expert top-k children with cumulative log-prob,
-                        "top-k construction principle of the Eagle tree"
+                        the Eagle-style tree growth of Sec. 3.1.2 (last
+                        paragraph)
   frontier_select       dynamic-tree frontier (Sec. 3.1.2, last paragraph)
   draft_expand          one draft layer: all of the above for F frontier nodes
   grow_tree             D draft layers in sequence -> candidate pool

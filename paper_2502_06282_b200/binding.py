@@ -141,6 +141,17 @@ class Context:
             base = (self.workspace.data_ptr() + 255) // 256 * 256
             self._check(lib().jk_set_workspace(self._h, _stream(), base, n), "jk_set_workspace")
 
+    def set_workspace(self, buf: torch.Tensor, offset: int = 0):
+        """jk_set_workspace on a caller-made uint8 device buffer: the workspace starts at the
+        first 256-byte boundary at or after buf[offset]; the buffer must stay alive."""
+        n = lib().jk_workspace_bytes(self._h)
+        base = (buf.data_ptr() + offset + 255) // 256 * 256
+        if base + n > buf.data_ptr() + buf.numel():
+            raise ValueError("buffer too small for the workspace")
+        self.workspace = buf
+        self._check(lib().jk_set_workspace(self._h, _stream(), base, n), "jk_set_workspace")
+        return base - buf.data_ptr()
+
     @classmethod
     def for_workload(cls, w, **kw) -> "Context":
         return cls(hidden=w.hidden, n_experts=w.n_experts, top_k=w.top_k, inter=w.inter,
@@ -239,9 +250,11 @@ class Context:
         self._check(rc, "jk_tree_verify_attn")
 
     def tree_verify_attn_static(self, batch, tree_size, q, k_cache, v_cache, kv_len, parent,
-                                scale, out, status=None, cache_rows=None):
+                                scale, out, status, cache_rows=None):
         """jk_tree_verify_attn_static: the same attention without any workspace, for callers
-        that cannot allocate device memory; scratch is the library's built-in 8 MiB array."""
+        that cannot allocate device memory; scratch is the library's built-in 8 MiB array.
+        `status` is a caller-owned int32 device word (cleared by the caller) that receives
+        JK_ERR_BOUNDS when a cache is too short."""
         rows = k_cache.shape[2] if cache_rows is None else cache_rows
         rc = lib().jk_tree_verify_attn_static(self._h, _stream(), batch, tree_size, _ptr(q),
                                               _ptr(k_cache), _ptr(v_cache), k_cache.stride(0),

@@ -330,15 +330,26 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     const float total = scan_s[nt - 1];
     const float thr = ub * total;
     const float before = scan_s[t] - loc;
-    if (before <= thr && scan_s[t] > thr) {          // the crossing lies in this thread's run
+    // The crossing lies in this thread's run (the scan is non-decreasing, so the test picks the
+    // first run whose end passes the threshold; several can pass it only when later runs are
+    // empty, and atomicMin keeps the first).
+    const bool mine = before <= thr && scan_s[t] > thr;
+    if (mine) {
       float run = before;
+      int last_pos = -1;
       for (int v = v0; v < v1; ++v) {
-        run += p_at(v);
-        if (run > thr) { atomicMin(&s_found, v); break; }
+        const float pv = p_at(v);
+        run += pv;
+        if (pv > 0.f) last_pos = v;
+        if (run > thr) { last_pos = v; break; }
       }
+      // The run was first added pairwise and now one by one: rounding can leave the sequential
+      // sum at or below the threshold.  The draw then belongs to this run's last token with
+      // p > 0 (the pairwise sum passed the threshold, so the run has one).
+      if (last_pos >= 0) atomicMin(&s_found, last_pos);
     }
     __syncthreads();
-    if (s_found == INT_MAX) {            // rounding left no bin: last token with p > 0
+    if (s_found == INT_MAX) {            // no run passed the threshold: last token with p > 0
       __syncthreads();
       if (t == 0) s_found = -1;
       __syncthreads();

@@ -315,7 +315,8 @@ static __device__ __align__(256) unsigned char g_attn_static_scratch[JK_ATTN_STA
 static void* g_attn_static_ptr[JK_ATTN_STATIC_MAX_DEVICES];   // device address, per device
 
 template <typename T, int D>
-static int attn_static_impl(jk_ctx* ctx, cudaStream_t st, unsigned char* scratch, int B, int M,
+static int attn_static_impl(jk_ctx* ctx, cudaStream_t st, int dev, unsigned char* scratch, int B,
+                            int M,
                             const void* q, const void* kc, const void* vc, int64_t sb, int64_t sh,
                             int cache_rows, const int32_t* kv_len, const int32_t* parent,
                             float scale, void* out, int32_t* status) {
@@ -338,18 +339,20 @@ static int attn_static_impl(jk_ctx* ctx, cudaStream_t st, unsigned char* scratch
   if (n_split > max_by_mem) n_split = max_by_mem;
   if (n_split > JK_ATTN_MAX_SPLIT) n_split = JK_ATTN_MAX_SPLIT;
   if (n_split < 1) n_split = 1;
-  // first 256 bytes: a status word for callers that pass none; it must start at zero
-  int32_t* status_word = status ? status : reinterpret_cast<int32_t*>(scratch);
-  if (!status) JK_CUDA_CHECK(ctx, cudaMemsetAsync(scratch, 0, 16, st));
   float* part_o = reinterpret_cast<float*>(scratch + 256);
   float* part_ml = part_o + (size_t)n_split * n_out * D;
   const size_t smem = sizeof(attn_smem<D>);
   auto kern = k_tree_attn<T, D>;
-  JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem));
+  // the shared-memory limit is a per-device property of the kernel: raised once per device
+  static bool smem_set[JK_ATTN_STATIC_MAX_DEVICES];
+  if (!smem_set[dev]) {
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)smem));
+    smem_set[dev] = true;
+  }
   kern<<<dim3(n_split * n_qblk, c.n_kv_heads, B), 256, smem, st>>>(
       (const T*)q, (const T*)kc, (const T*)vc, sb, sh, cache_rows, kv_len, parent, scale, M,
-      c.n_q_heads, c.n_kv_heads, n_split, n_qblk, part_o, part_ml, status_word);
+      c.n_q_heads, c.n_kv_heads, n_split, n_qblk, part_o, part_ml, status);
   JK_LAUNCH_CHECK(ctx);
   k_attn_combine<T, D><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
                                                                     n_out, (T*)out);
@@ -363,7 +366,10 @@ extern "C" int jk_tree_verify_attn_static(jk_ctx* ctx, void* stream, int32_t bat
                                           int64_t cache_stride_h, int32_t cache_rows,
                                           const int32_t* kv_len, const int32_t* parent,
                                           float softmax_scale, void* out, int32_t* status) {
-  if (!ctx || !q || !k_cache || !v_cache || !kv_len || !parent || !out) return JK_ERR_NULL;
+  // `status` is required: this call has no context workspace whose status word could record a
+  // cache that is too short, and an error nobody can read is worse than an argument error.
+  if (!ctx || !q || !k_cache || !v_cache || !kv_len || !parent || !out || !status)
+    return JK_ERR_NULL;
   const jk_config& c = ctx->cfg;
   if (batch < 1 || tree_size < 1 || cache_rows < tree_size) return JK_ERR_SHAPE;
   if (batch > c.max_batch || tree_size > c.max_tree) return JK_ERR_CAPACITY;
@@ -394,7 +400,7 @@ extern "C" int jk_tree_verify_attn_static(jk_ctx* ctx, void* stream, int32_t bat
   unsigned char* scratch = static_cast<unsigned char*>(g_attn_static_ptr[dev]);
   cudaStream_t st = (cudaStream_t)stream;
 #define JK_ATTN_STATIC_CASE(T, D)                                                             \
-  return attn_static_impl<T, D>(ctx, st, scratch, batch, tree_size, q, k_cache, v_cache,      \
+  return attn_static_impl<T, D>(ctx, st, dev, scratch, batch, tree_size, q, k_cache, v_cache, \
                                 cache_stride_b, cache_stride_h, cache_rows, kv_len, parent,   \
                                 softmax_scale, out, status)
   if (c.dtype == JK_BF16) {

@@ -440,6 +440,22 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         }
         l_run = l_run * alpha + lsum;
         m_run = m_new;
+        // Cache rows past the last live key (only a sequence's last tile has any) may hold
+        // anything, NaN bit patterns included, and 0 * NaN would poison every output row: they
+        // are cleared in the V tile before the second product reads it.
+        const int live = P + M - tile * ASK_KEYS;
+        if (live < ASK_KEYS) {
+          const bool okv = mbar_wait(&T.v_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
+          ok = __all_sync(0xffffffffu, okv);
+          if (!ok) break;
+          const int n16 = (ASK_KEYS - live) * 8;               // 16-byte pieces per 64-wide block
+          unsigned char* vt = sv + bf * KV_BYTES;
+          for (int idx = sm_tid; idx < n16 * KB; idx += ASK_SM_THREADS) {
+            const int kb = idx / n16, rem = idx % n16;
+            *reinterpret_cast<uint4*>(vt + kb * 16384 + (live + (rem >> 3)) * 128 + ((rem & 7) << 4)) =
+                make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
         fence_proxy_async_smem();
         tc_fence_before();
         mbar_arrive(&T.s_empty[bf]);
@@ -585,7 +601,7 @@ __global__ void __launch_bounds__(256) k_attn_combine_sk(
 
 // jk_attn_tc.cu: tensor maps of the two caches
 int jk_attn_tc_maps(jk_ctx* ctx, const void* kc, const void* vc, int64_t sb, int64_t sh,
-                    int cache_rows, const CUtensorMap** mk, const CUtensorMap** mv);
+                    int cache_rows, CUtensorMap* mk, CUtensorMap* mv);
 
 // The kernel needs room for at least three partials per query block, sequence counts that fit
 // its shared arrays, and unit indices that stay in 32 bits.
@@ -604,7 +620,7 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                const int32_t* parent, float scale, void* out) {
   const jk_config& c = ctx->cfg;
   const jk_ws_layout& L = ctx->lay;
-  const CUtensorMap *mk = nullptr, *mv = nullptr;
+  CUtensorMap mk, mv;
   int rc = jk_attn_tc_maps(ctx, kc, vc, sb, sh, cache_rows, &mk, &mv);
   if (rc != JK_OK) return rc;
   const int D = c.head_dim;
@@ -625,11 +641,11 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   const int min_units = 1;
   JK_PROF(ctx, st, JK_ST_ATTN);
   if (D == 128)
-    jk_launch_pdl(k_tree_attn_sk<128>, dim3(n_cta), dim3(ASK_THREADS), smem, st, *mk, *mv,
+    jk_launch_pdl(k_tree_attn_sk<128>, dim3(n_cta), dim3(ASK_THREADS), smem, st, mk, mv,
                   (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
                   ms, min_units, cache_rows, part_o, part_ml, status);
   else
-    jk_launch_pdl(k_tree_attn_sk<64>, dim3(n_cta), dim3(ASK_THREADS), smem, st, *mk, *mv,
+    jk_launch_pdl(k_tree_attn_sk<64>, dim3(n_cta), dim3(ASK_THREADS), smem, st, mk, mv,
                   (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
                   ms, min_units, cache_rows, part_o, part_ml, status);
   JK_LAUNCH_CHECK(ctx);

@@ -259,11 +259,26 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
           tmem_st_wait();
         }
       }
+      // Cache rows past the last live key (only the sequence's last tile has any) may hold
+      // anything, NaN bit patterns included, and 0 * NaN would poison every output row: they are
+      // cleared in the V tile before the second product reads it.
+      const int live = Ltot - tile * ATC_KEYS;
+      if (live < ATC_KEYS) {
+        ok = ok && mbar_wait(&T.bar_v, ph, abort_flag, status);
+        if (ok) {
+          const int n16 = (ATC_KEYS - live) * 8;               // 16-byte pieces per 64-wide block
+          for (int idx = tid; idx < n16 * KB; idx += ATC_THREADS) {
+            const int kb = idx / n16, rem = idx % n16;
+            *reinterpret_cast<uint4*>(sv + kb * 16384 + (live + (rem >> 3)) * 128 + ((rem & 7) << 4)) =
+                make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
       fence_proxy_async_smem();
       tc_fence_before();
       __syncthreads();
       if (tid == 0) {
-        ok = mbar_wait(&T.bar_v, ph, abort_flag, status);
+        ok = ok && mbar_wait(&T.bar_v, ph, abort_flag, status);
         if (ok) {
           tc_fence_after();
           const uint32_t pa = smem_u32(skp), va = smem_u32(sv);
@@ -379,16 +394,21 @@ void jk_attn_tc_destroy(jk_ctx* ctx) {
 }
 
 // Tensor maps of a K and a V cache (cached per pointer and strides).
+// The maps are handed out by value: a later lookup may recycle the slot an earlier one returned.
 int jk_attn_tc_maps(jk_ctx* ctx, const void* kc, const void* vc, int64_t sb, int64_t sh,
-                    int cache_rows, const CUtensorMap** mk, const CUtensorMap** mv) {
+                    int cache_rows, CUtensorMap* mk, CUtensorMap* mv) {
   if (!ctx->attn_tc_state) {
     ctx->attn_tc_state = calloc(1, sizeof(atc_state));
     if (!ctx->attn_tc_state) return JK_ERR_CUDA;
   }
   atc_state* s = (atc_state*)ctx->attn_tc_state;
-  *mk = atc_map(ctx, s, kc, sb, sh, cache_rows);
-  *mv = atc_map(ctx, s, vc, sb, sh, cache_rows);
-  return (*mk && *mv) ? JK_OK : JK_ERR_CUDA;
+  const CUtensorMap* m = atc_map(ctx, s, kc, sb, sh, cache_rows);
+  if (!m) return JK_ERR_CUDA;
+  *mk = *m;
+  m = atc_map(ctx, s, vc, sb, sh, cache_rows);
+  if (!m) return JK_ERR_CUDA;
+  *mv = *m;
+  return JK_OK;
 }
 
 // jk_attn_sk.cu: the persistent pipelined kernel
@@ -414,7 +434,7 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
     if (want && jk_attn_sk_usable(ctx, B, M, cache_rows))
       return jk_attn_sk(ctx, st, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale, out);
   }
-  const CUtensorMap *mk = nullptr, *mv = nullptr;
+  CUtensorMap mk, mv;
   if (jk_attn_tc_maps(ctx, kc, vc, sb, sh, cache_rows, &mk, &mv) != JK_OK) return JK_ERR_CUDA;
   atc_state* s = (atc_state*)ctx->attn_tc_state;
   const int G = c.n_q_heads / c.n_kv_heads;
@@ -442,12 +462,12 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   }
   JK_PROF(ctx, st, JK_ST_ATTN);
   if (D == 128)
-    jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(ATC_THREADS), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+    jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(ATC_THREADS), smem, st, mk, mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                  scale, M, c.n_q_heads, c.n_kv_heads, n_split,
                                                  n_qblk, cache_rows, part_o, part_ml,
                                                  (__nv_bfloat16*)out, status);
   else
-    jk_launch_pdl(k_tree_attn_tc<64>, dim3(grid), dim3(ATC_THREADS), smem, st, *mk, *mv, (const __nv_bfloat16*)q, kv_len, parent,
+    jk_launch_pdl(k_tree_attn_tc<64>, dim3(grid), dim3(ATC_THREADS), smem, st, mk, mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                 scale, M, c.n_q_heads, c.n_kv_heads, n_split,
                                                 n_qblk, cache_rows, part_o, part_ml,
                                                 (__nv_bfloat16*)out, status);

@@ -570,8 +570,8 @@ extern "C" int jk_tensor_path_active(jk_ctx* ctx) {
 }
 
 // 2-D bf16 tensor map: `rows` x `cols` (cols contiguous), box = box_rows x 64, 128-byte swizzle.
-static const CUtensorMap* tc_map(jk_ctx* ctx, tc_state* s, const void* ptr, uint64_t rows,
-                                 uint64_t cols, uint32_t box_rows) {
+static const CUtensorMap* tc_map_lookup(jk_ctx* ctx, tc_state* s, const void* ptr, uint64_t rows,
+                                        uint64_t cols, uint32_t box_rows) {
   for (int i = 0; i < s->n_maps; ++i) {
     tc_map_entry& e = s->maps[i];
     if (e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows) return &e.map;
@@ -593,6 +593,15 @@ static const CUtensorMap* tc_map(jk_ctx* ctx, tc_state* s, const void* ptr, uint
   e.ptr = ptr; e.rows = rows; e.cols = cols; e.box_rows = box_rows;
   ++s->n_maps;
   return &e.map;
+}
+
+// The same, handed out by value: a later lookup may recycle the slot an earlier one returned.
+static bool tc_map(jk_ctx* ctx, tc_state* s, const void* ptr, uint64_t rows, uint64_t cols,
+                   uint32_t box_rows, CUtensorMap* out) {
+  const CUtensorMap* m = tc_map_lookup(ctx, s, ptr, rows, cols, box_rows);
+  if (!m) return false;
+  *out = *m;
+  return true;
 }
 
 // Launch the streaming GEMM; fills the launch-dependent fields of p and returns the grid size.
@@ -641,10 +650,11 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   const int n_pad = (int)jk_align_up(R, 16);
   int n_cta = 0;
   // gate / up
-  const CUtensorMap* ag = tc_map(ctx, s, w->w_gate, (uint64_t)N * I, H, TC_TILE_M);
-  const CUtensorMap* au = tc_map(ctx, s, w->w_up, (uint64_t)N * I, H, TC_TILE_M);
-  const CUtensorMap* bx = tc_map(ctx, s, ctx->ws + L.xn, Rp, H, n_pad);
-  if (!ag || !au || !bx) return JK_ERR_CUDA;
+  CUtensorMap ag, au, bx;
+  if (!tc_map(ctx, s, w->w_gate, (uint64_t)N * I, H, TC_TILE_M, &ag) ||
+      !tc_map(ctx, s, w->w_up, (uint64_t)N * I, H, TC_TILE_M, &au) ||
+      !tc_map(ctx, s, ctx->ws + L.xn, Rp, H, n_pad, &bx))
+    return JK_ERR_CUDA;
   p.n_groups_max = 2 * N;
   for (int e = 0; e < N; ++e)
     for (int h = 0; h < 2; ++h) {
@@ -654,16 +664,17 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   p.tiles_per_group = (I + TC_TILE_M - 1) / TC_TILE_M;
   p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
   p.n_pad = n_pad;
-  int rc = tc_launch_gemm(ctx, st, s, ag, au, bx, p, expert, JK_ST_GATEUP, &n_cta);
+  int rc = tc_launch_gemm(ctx, st, s, &ag, &au, &bx, p, expert, JK_ST_GATEUP, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_GEMM_FIXUP);
   jk_launch_pdl(k_tc_fix_silu, dim3(p.tiles_per_group, N, R), dim3(128), 0, st, 
       p, n_cta, I, R, Rp, expert, partial, (__nv_bfloat16*)(ctx->ws + L.hbuf));
   JK_LAUNCH_CHECK(ctx);
   // down
-  const CUtensorMap* ad = tc_map(ctx, s, w->w_down, (uint64_t)N * H, I, TC_TILE_M);
-  const CUtensorMap* bh = tc_map(ctx, s, ctx->ws + L.hbuf, (uint64_t)N * Rp, I, n_pad);
-  if (!ad || !bh) return JK_ERR_CUDA;
+  CUtensorMap ad, bh;
+  if (!tc_map(ctx, s, w->w_down, (uint64_t)N * H, I, TC_TILE_M, &ad) ||
+      !tc_map(ctx, s, ctx->ws + L.hbuf, (uint64_t)N * Rp, I, n_pad, &bh))
+    return JK_ERR_CUDA;
   p.n_groups_max = N;
   for (int e = 0; e < N; ++e) {
     p.group_expert[e] = e; p.group_amap[e] = 0; p.group_arow0[e] = e * H; p.group_brow0[e] = e * Rp;
@@ -671,7 +682,7 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   p.tiles_per_group = (H + TC_TILE_M - 1) / TC_TILE_M;
   p.kt = (I + TC_TILE_K - 1) / TC_TILE_K;
   p.prefetch = 1;
-  rc = tc_launch_gemm(ctx, st, s, ad, ad, bh, p, expert, JK_ST_DOWN, &n_cta);
+  rc = tc_launch_gemm(ctx, st, s, &ad, &ad, &bh, p, expert, JK_ST_DOWN, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_BRANCH);
   jk_launch_pdl(k_tc_fix_down_branch, dim3(p.tiles_per_group, R), dim3(128), 0, st, 
@@ -694,9 +705,10 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
   memset(&p, 0, sizeof(p));
   p.R = 0; p.K_top = c.top_k; p.n_experts = c.n_experts;
   const int n_pad = (int)jk_align_up(RK, 16);
-  const CUtensorMap* ah = tc_map(ctx, s, w->lm_head, V, H, TC_TILE_M);
-  const CUtensorMap* bb = tc_map(ctx, s, ctx->ws + L.bbuf, L.rk_pad, H, n_pad);
-  if (!ah || !bb) return JK_ERR_CUDA;
+  CUtensorMap ah, bb;
+  if (!tc_map(ctx, s, w->lm_head, V, H, TC_TILE_M, &ah) ||
+      !tc_map(ctx, s, ctx->ws + L.bbuf, L.rk_pad, H, n_pad, &bb))
+    return JK_ERR_CUDA;
   p.n_groups_max = 1;
   p.group_expert[0] = -1; p.group_amap[0] = 0; p.group_arow0[0] = 0; p.group_brow0[0] = 0;
   p.tiles_per_group = (V + TC_TILE_M - 1) / TC_TILE_M;
@@ -704,7 +716,7 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
   p.n_pad = n_pad;
   int n_cta = 0;
   p.prefetch = 1;
-  int rc = tc_launch_gemm(ctx, st, s, ah, ah, bb, p, nullptr, JK_ST_LMHEAD, &n_cta);
+  int rc = tc_launch_gemm(ctx, st, s, &ah, &ah, &bb, p, nullptr, JK_ST_LMHEAD, &n_cta);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_TOPK);
   jk_launch_pdl(k_tc_fix_lmhead_topk, dim3(L.topk_chunks, RK), dim3(JK_TOPK_THREADS), 0, st, 

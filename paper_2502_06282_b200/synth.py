@@ -148,6 +148,27 @@ def draft_weights(w: Workload) -> Dict[str, np.ndarray]:
     return {k: store_round(v, w.dtype) for k, v in out.items()}
 
 
+def shared_weights(w: Workload) -> Dict[str, np.ndarray]:
+    """The parts of draft_weights that do not grow with the expert count: expert centroids, LM
+    head, norm weight (same streams as draft_weights)."""
+    r = lambda s: _rng(w.seed, s)
+    out = {
+        "router": _normal(r(1), (w.n_experts, w.hidden), 0.02),
+        "lm_head": _normal(r(5), (w.vocab, w.hidden), 0.02),
+        "norm_weight": np.ones((w.hidden,), dtype=np.float32),
+    }
+    return {k: store_round(v, w.dtype) for k, v in out.items()}
+
+
+def expert_weight(w: Workload, name: str, e: int) -> np.ndarray:
+    """One expert's matrix ("w_gate" | "w_up" [I, H], "w_down" [H, I]), N(0, 0.02), from a
+    stream of its own, for shapes whose whole expert set would not fit the host in fp32.  (Not
+    the same numbers as draft_weights, which draws all experts of a matrix from one stream.)"""
+    idx = {"w_gate": 0, "w_up": 1, "w_down": 2}[name]
+    shape = (w.hidden, w.inter) if name == "w_down" else (w.inter, w.hidden)
+    return store_round(_normal(_rng(w.seed, 1000 + 3 * e + idx), shape, 0.02), w.dtype)
+
+
 def layer_hidden(w: Workload, layer: int, n_frontier: int) -> np.ndarray:
     """u [B, F, H]: post-attention hidden state of each frontier node (the
     output of Eq. 1), N(0, 1).  Stands in for the draft's reduction layer and

@@ -31,3 +31,79 @@ def rel_err(got: np.ndarray, want: np.ndarray) -> float:
 
 def weights_to_device(wts: dict, dtype: str) -> dict:
     return {k: dev(v, dtype) for k, v in wts.items()}
+
+
+# ------------------------------------------------------------------------------------------
+# Guarded device buffers: the stand-in for a memory checker.  Every buffer sits between two
+# 256-byte canaries and starts out poisoned (0xFF bytes: NaN as a float, -1 as an int), so a
+# write outside an output shows up as a broken canary and a read of something the library never
+# wrote shows up as NaN / -1 in the results.
+# ------------------------------------------------------------------------------------------
+class Guard:
+    PAD = 256
+    CANARY = 0xA5
+    POISON = 0xFF
+
+    def __init__(self):
+        self.regions = []
+
+    def alloc(self, shape, dtype: torch.dtype) -> torch.Tensor:
+        shape = tuple(int(s) for s in shape)
+        n = int(np.prod(shape, dtype=np.int64)) * torch.empty((), dtype=dtype).element_size()
+        body = (n + 255) // 256 * 256
+        raw = torch.full((self.PAD + body + self.PAD,), self.CANARY, dtype=torch.uint8, device="cuda")
+        raw[self.PAD:self.PAD + n] = self.POISON
+        self.regions.append((raw, n))
+        return raw[self.PAD:self.PAD + n].view(dtype).view(shape)
+
+    def like(self, t: torch.Tensor, keep: bool = False) -> torch.Tensor:
+        g = self.alloc(t.shape, t.dtype)
+        if keep:
+            g.copy_(t)
+        return g
+
+    def check(self):
+        torch.cuda.synchronize()
+        for i, (raw, n) in enumerate(self.regions):
+            assert bool((raw[:self.PAD] == self.CANARY).all()), f"write before buffer {i}"
+            assert bool((raw[self.PAD + n:] == self.CANARY).all()), f"write past buffer {i}"
+
+
+def guarded_context(w, **kw):
+    """A context whose workspace is poisoned and fenced by canaries.  Returns (ctx, check)."""
+    from paper_2502_06282_b200 import binding as jk
+    ctx = jk.Context.for_workload(w, allocate=False, **kw)
+    n = ctx.workspace_bytes
+    pad = 512
+    raw = torch.full((pad + n + pad + 256,), Guard.CANARY, dtype=torch.uint8, device="cuda")
+    off = ctx.set_workspace(raw, pad)             # also clears the status word
+    torch.cuda.synchronize()
+    raw[off + 256:off + n] = Guard.POISON         # everything but the status section
+
+    def check():
+        torch.cuda.synchronize()
+        assert bool((raw[:off] == Guard.CANARY).all()), "write before the workspace"
+        assert bool((raw[off + n:] == Guard.CANARY).all()), "write past the workspace"
+
+    return ctx, check
+
+
+def guarded_step_buffers(ctx, w, guard: Guard):
+    """StepBuffers whose every tensor is a guarded, poisoned allocation."""
+    from paper_2502_06282_b200 import binding as jk
+    bufs = jk.StepBuffers(ctx, w)
+    for k in bufs.pool:
+        bufs.pool[k] = guard.like(bufs.pool[k])
+    bufs.pool_struct = ctx.pool_struct(bufs.pool)
+    for name in ("probs", "expert", "gate", "lse", "feat", "frontier"):
+        setattr(bufs, name, [guard.like(t) for t in getattr(bufs, name)])
+    bufs.parent_score = [guard.like(bufs.parent_score[0], keep=True)] + [
+        guard.like(t) for t in bufs.parent_score[1:]]
+    bufs.parent_gidx = [guard.like(bufs.parent_gidx[0], keep=True)] + [
+        guard.like(t) for t in bufs.parent_gidx[1:]]
+    if bufs.logits is not None:
+        bufs.logits = guard.like(bufs.logits)
+    bufs.tree = {k: guard.like(v) for k, v in bufs.tree.items()}
+    for name in ("anc", "n_acc", "acc_idx", "acc_tok", "bonus"):
+        setattr(bufs, name, guard.like(getattr(bufs, name)))
+    return bufs

@@ -153,3 +153,39 @@ def test_attn_is_bitwise_reproducible(kernel):
         outs.append(out.view(torch.int16).cpu())
     assert ctx.read_status() == 0
     assert torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("dtype,kernel", [("f32", 0), ("bf16", 0), ("bf16", 1), ("bf16", 2)])
+def test_attn_ignores_cache_rows_past_the_tree(dtype, kernel):
+    """The operation is defined over cache rows c < kv_len + M only (Sec. 2.1 step 2).  Rows
+    between kv_len + M and the cache capacity belong to nobody: here they hold NaN (as a pool
+    that was never cleared may), in K and in V, and must leave no trace in the output.  Ragged
+    lengths put the dead rows in the middle of a key tile for some sequences and make a whole
+    tile dead for others."""
+    w = synth.scaled(synth.WORKLOADS["tiny"], name="attn_nan", dtype=dtype, prefix=300,
+                     tree_size=37, n_q_heads=8, n_kv_heads=2, head_dim=128, batch=3, depth=6,
+                     seed=4711)
+    par = _trees(w, "random")
+    q, k, v, kv_len = synth.attn_inputs(w, 0, ragged=True)
+    kv_len[1] = 90                                     # one sequence leaves two whole tiles dead
+    k, v = k.copy(), v.copy()
+    for b in range(w.batch):
+        k[b, :, int(kv_len[b]) + w.tree_size:] = np.nan
+        v[b, :, int(kv_len[b]) + w.tree_size:] = np.nan
+    assert np.isnan(k).any()
+    ctx = jk.Context.for_workload(w)
+    ctx.set_attn_kernel(kernel)
+    kd = torch.from_numpy(k).cuda()
+    vd = torch.from_numpy(v).cuda()
+    if dtype == "bf16":
+        kd, vd = kd.to(torch.bfloat16), vd.to(torch.bfloat16)
+    qd = dev(q, w.dtype)
+    out = torch.empty_like(qd)
+    scale = 1.0 / math.sqrt(w.head_dim)
+    ctx.tree_verify_attn(w.batch, w.tree_size, qd, kd, vd, dev(kv_len), dev(par), scale, out)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    got = host(out)
+    assert not np.isnan(got).any()
+    ref = orc.tree_verify_attn(q, np.nan_to_num(k), np.nan_to_num(v), kv_len, par, scale)
+    assert rel_err(got, ref) <= TOL[dtype]

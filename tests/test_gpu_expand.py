@@ -11,27 +11,35 @@ import torch
 from oracle import jakiro_oracle as orc
 from paper_2502_06282_b200 import binding as jk
 from paper_2502_06282_b200 import synth
-from tests.jk_testutil import TOL, dev, host, rel_err, weights_to_device
+from tests.jk_testutil import (TOL, Guard, dev, guarded_context, guarded_step_buffers, host,
+                                rel_err, weights_to_device)
 
 pytestmark = pytest.mark.gpu
 
 
-def _run_gpu(w, wts_np, us_np, tensor_path=None, root_tok=5):
-    ctx = jk.Context.for_workload(w)
+def _run_gpu(w, wts_np, us_np, tensor_path=None, root_tok=5, expect_tensor_path=None, **ctx_kw):
+    """One draft (D expand calls + finalize) with every output buffer and the workspace poisoned
+    and fenced by canaries; the canaries are checked before the results are returned."""
+    ctx, check_ws = guarded_context(w, **ctx_kw)
     if tensor_path is not None:
         ctx.set_tensor_path(tensor_path)
         assert ctx.tensor_path_active == bool(tensor_path)
-    bufs = jk.StepBuffers(ctx, w)
+    if expect_tensor_path is not None:
+        assert ctx.tensor_path_active == expect_tensor_path
+    guard = Guard()
+    bufs = guarded_step_buffers(ctx, w, guard)
     wts = weights_to_device(wts_np, w.dtype)
     us = [dev(u, w.dtype) for u in us_np]
     root = torch.full((w.batch,), root_tok, dtype=torch.int32, device="cuda")
     jk.run_draft(ctx, bufs, wts, us, root)
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
+    guard.check()
+    check_ws()
     return ctx, bufs
 
 
-def _check_layers(w, wts_np, us_np, bufs):
+def _check_layers(w, wts_np, us_np, bufs, use_pre_norm=True, branch_residual=True, rms_eps=1e-5):
     tol = TOL[w.dtype]
     fs = w.frontier_sizes
     K, ke = w.top_k, w.k_per_expert
@@ -44,7 +52,7 @@ def _check_layers(w, wts_np, us_np, bufs):
         pgidx = host(bufs.parent_gidx[l])
         probs_g, exp_g, gate_g = host(bufs.probs[l]), host(bufs.expert[l]), host(bufs.gate[l])
         feat_g, lse_g = host(bufs.feat[l]), host(bufs.lse[l])
-        x = orc.rmsnorm(u, wts_np["norm_weight"], 1e-5)
+        x = orc.rmsnorm(u, wts_np["norm_weight"], rms_eps) if use_pre_norm else u
         probs_o = orc.router_scores(x, wts_np["router"])
         assert rel_err(probs_g, probs_o) <= tol
         n_cand = F * K * ke
@@ -58,7 +66,8 @@ def _check_layers(w, wts_np, us_np, bufs):
                 margin = np.sort(probs_o[b, f])[::-1]
                 if margin[K - 1] - margin[K] > 1e-3 and (K < 2 or margin[0] - margin[1] > 1e-3):
                     assert ids_o.tolist() == ids_r.tolist()
-                _, br, ff = orc.moe_features(u[b, f], x[b, f], ids_r, probs_o[b, f][ids_r], wts_np)
+                _, br, ff = orc.moe_features(u[b, f], x[b, f], ids_r, probs_o[b, f][ids_r], wts_np,
+                                             branch_residual)
                 assert rel_err(feat_g[b, f], ff) <= tol
                 lg_o = orc.head_logits(br, wts_np["lm_head"])
                 lg_g = logits_all[b, slot_base + f]
@@ -139,7 +148,7 @@ def test_expand_batched_ragged_shapes(tensor_path):
     _check_tree(w, pool, bufs, 5)
 
 
-def test_expand_f32_ragged_and_flags():
+def test_expand_f32_ragged_shapes():
     w = synth.scaled(synth.WORKLOADS["tiny"], name="ragged32", batch=2, vocab=4100, inter=520,
                      hidden=136, n_experts=5, k_per_expert=4, width=6, tree_size=25, depth=3,
                      seed=78)
@@ -147,6 +156,83 @@ def test_expand_f32_ragged_and_flags():
     ctx, bufs = _run_gpu(w, wts, us)
     pool = _check_layers(w, wts, us, bufs)
     _check_tree(w, pool, bufs, 5)
+
+
+@pytest.mark.parametrize("name,tensor_path", [("tiny", None), ("tiny_bf16", False),
+                                              ("tiny_bf16", True)])
+@pytest.mark.parametrize("use_pre_norm,branch_residual", [(False, True), (True, False),
+                                                          (False, False)])
+def test_expand_config_flags(name, tensor_path, use_pre_norm, branch_residual):
+    """The two readings the configuration can switch: no pre-MoE normalisation (router and
+    experts see u itself), and branch features without the residual (Eq. 4 taken literally as
+    Head(s_r * Expert_r)).  Hidden states three times larger than unit RMS, a norm weight that
+    is not all ones and a large epsilon make each switch change the result well beyond the
+    tolerance, so a flag that the kernels ignored could not pass."""
+    w = synth.scaled(synth.WORKLOADS[name], batch=2, depth=3, tree_size=14, seed=4242)
+    wts, us = _inputs(w)
+    gamma = 0.5 + np.random.default_rng(3).random(w.hidden).astype(np.float32)
+    wts["norm_weight"] = synth.store_round(gamma, w.dtype)
+    us = [synth.store_round(3.0 * u, w.dtype) for u in us]
+    eps = 0.75
+    ctx, bufs = _run_gpu(w, wts, us, tensor_path, use_pre_norm=use_pre_norm,
+                         branch_residual=branch_residual, rms_eps=eps)
+    pool = _check_layers(w, wts, us, bufs, use_pre_norm, branch_residual, eps)
+    _check_tree(w, pool, bufs, 5)
+    # the switch matters on these inputs: the other setting is far outside the tolerance
+    u0 = us[0].astype(np.float64)
+    other = orc.draft_expand(u0, np.zeros((w.batch, 1)), wts, w.k_per_expert, w.width,
+                             rms_eps=eps, use_pre_norm=not use_pre_norm,
+                             branch_residual=branch_residual)
+    assert rel_err(host(bufs.logits)[:, 0], other["logits"][:, 0]) > 10 * TOL[w.dtype]
+    other = orc.draft_expand(u0, np.zeros((w.batch, 1)), wts, w.k_per_expert, w.width,
+                             rms_eps=eps, use_pre_norm=use_pre_norm,
+                             branch_residual=not branch_residual)
+    assert rel_err(host(bufs.logits)[:, 0], other["logits"][:, 0]) > 10 * TOL[w.dtype]
+
+
+@pytest.mark.parametrize("name,tensor_path", [("tiny", None), ("tiny_bf16", False),
+                                              ("tiny_bf16", True)])
+def test_expand_planted_ties(name, tensor_path):
+    """Two vocabulary rows of the LM head made identical, chosen so that they are the root's best
+    left-branch tokens: their logits are equal bit for bit (same weight tile, same summation
+    order), so the top-k order and the frontier order are both decided by the tie rule (lower
+    token id, then lower candidate index)."""
+    w = synth.WORKLOADS[name]
+    wts, us = _inputs(w)
+    _, first = _run_gpu(w, wts, us, tensor_path)
+    t1 = int(host(first.pool["tok"])[0, 0])
+    t2 = t1 ^ 1
+    wts["lm_head"] = wts["lm_head"].copy()
+    wts["lm_head"][t2] = wts["lm_head"][t1]
+    ctx, bufs = _run_gpu(w, wts, us, tensor_path)
+    lg = host(bufs.logits)[0, 0, 0]
+    assert lg[t1] == lg[t2]
+    pool = _check_layers(w, wts, us, bufs)
+    assert pool["tok"][0, :2].tolist() == sorted([t1, t2])
+    assert pool["score"][0, 0] == pool["score"][0, 1]
+    fr = host(bufs.frontier[0])[0].tolist()
+    assert fr.index(0) < fr.index(1)                 # equal scores: the lower index goes first
+    _check_tree(w, pool, bufs, 5)
+
+
+def test_expand_tensor_path_row_limit_and_fallback():
+    """128 activation rows with K = 2 give 256 logits rows, the most the tensor-core GEMM takes
+    (two accumulators of 256 columns fill the tensor memory); with K = 3 the same rows give 384,
+    the context reports the tensor path as inactive and the CUDA-core kernels run instead."""
+    base = dict(name="rows", batch=8, hidden=256, inter=512, vocab=4096, depth=2, tree_size=24,
+                width=16, seed=91)
+    w = synth.scaled(synth.WORKLOADS["tiny_bf16"], k_per_expert=8, **base)
+    assert w.frontier_sizes == [1, 16]
+    wts, us = _inputs(w)
+    ctx, bufs = _run_gpu(w, wts, us, expect_tensor_path=True)
+    pool = _check_layers(w, wts, us, bufs)
+    _check_tree(w, pool, bufs, 5)
+    w3 = synth.scaled(synth.WORKLOADS["tiny_bf16"], k_per_expert=6, top_k=3, **base)
+    assert w3.frontier_sizes == [1, 16]
+    wts, us = _inputs(w3)
+    ctx, bufs = _run_gpu(w3, wts, us, expect_tensor_path=False)
+    pool = _check_layers(w3, wts, us, bufs)
+    _check_tree(w3, pool, bufs, 5)
 
 
 def test_expand_is_deterministic():
@@ -159,21 +245,37 @@ def test_expand_is_deterministic():
         assert torch.equal(a.pool[k], b.pool[k])
 
 
-def _sampled_rows(w, samples):
-    """Two draft layers at full-size shapes, launch configuration as benchmarked; the oracle
-    recomputes the (batch, frontier row) pairs in `samples[layer]`."""
-    wts = synth.draft_weights(w)
-    fs = w.frontier_sizes[:2]
+def _sampled_rows(w, samples, wts=None, wts_dev=None):
+    """len(samples) draft layers at full-size shapes, launch configuration as benchmarked; the
+    oracle recomputes the (batch, frontier row) pairs in `samples[layer]`.  `wts` may hold
+    per-expert matrices behind lazy sequences (and `wts_dev` the device copies made expert by
+    expert) for shapes whose full fp32 weight set would not fit the host."""
+    if wts is None:
+        wts = synth.draft_weights(w)
+    n_l = len(samples)
+    fs = w.frontier_sizes[:n_l]
     us = [synth.layer_hidden(w, l, F) for l, F in enumerate(fs)]
-    w2 = synth.scaled(w, depth=2, tree_size=min(w.tree_size, 12))
-    ctx, bufs = _run_gpu(w2, wts, us)
+    w2 = synth.scaled(w, depth=n_l, tree_size=min(w.tree_size, 12))
+    ctx, check_ws = guarded_context(w2)
+    guard = Guard()
+    bufs = guarded_step_buffers(ctx, w2, guard)
+    if wts_dev is None:
+        wts_dev = weights_to_device(wts, w.dtype)
+    root = torch.full((w.batch,), 5, dtype=torch.int32, device="cuda")
+    jk.run_draft(ctx, bufs, wts_dev, [dev(u, w.dtype) for u in us], root)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    guard.check()
+    check_ws()
     tol = TOL[w.dtype]
-    head64 = wts["lm_head"].astype(np.float64)
+    head64 = np.asarray(wts["lm_head"], dtype=np.float64)
     K, ke = w.top_k, w.k_per_expert
-    slot_base = 0
+    slot_base, gidx_base = 0, 0
+    pool_tok, pool_score = host(bufs.pool["tok"]), host(bufs.pool["score"])
     for l, F in enumerate(fs):
         u = us[l].astype(np.float64)
         probs_g = host(bufs.probs[l])
+        pscore = host(bufs.parent_score[l])
         for b, f in samples[l]:
             x = orc.rmsnorm(u[b, f], wts["norm_weight"], 1e-5)
             probs_o = orc.router_scores(x, wts["router"])
@@ -186,17 +288,39 @@ def _sampled_rows(w, samples):
             lg_g = host(bufs.logits[b, slot_base + f])
             assert rel_err(lg_g, lg_o) <= tol
             for r in range(K):
-                ids_t, sc_t, _ = orc.branch_topk(lg_g[r], ke,
-                                                 float(host(bufs.parent_score[l])[b, f]))
-                g0 = (0 if l == 0 else fs[0] * K * ke) + (f * K + r) * ke
-                assert host(bufs.pool["tok"])[b, g0:g0 + ke].tolist() == ids_t.tolist()
-                assert np.allclose(host(bufs.pool["score"])[b, g0:g0 + ke], sc_t, rtol=1e-5,
-                                   atol=2e-5)
+                ids_t, sc_t, _ = orc.branch_topk(lg_g[r], ke, float(pscore[b, f]))
+                g0 = gidx_base + (f * K + r) * ke
+                assert pool_tok[b, g0:g0 + ke].tolist() == ids_t.tolist()
+                assert np.allclose(pool_score[b, g0:g0 + ke], sc_t, rtol=1e-5, atol=2e-5)
+        # the frontier of every layer but the last, replayed from the GPU's scores
+        n_cand = F * K * ke
+        if l < n_l - 1:
+            for b in range(w.batch):
+                sel = orc.frontier_select(pool_score[b, gidx_base:gidx_base + n_cand],
+                                          min(w.width, n_cand))
+                assert host(bufs.frontier[l])[b].tolist() == sel.tolist()
+                assert host(bufs.parent_gidx[l + 1])[b].tolist() == (gidx_base + sel).tolist()
         slot_base += F
+        gidx_base += n_cand
+    return bufs
 
 
 def test_expand_llama2_7b_shape_sampled_rows():
     _sampled_rows(synth.WORKLOADS["llama2_7b"], [[(0, 0)], [(0, 3), (0, 8)]])
+
+
+def test_expand_llama2_7b_shape_all_layers():
+    """All six draft layers of the benchmarked step (frontier sizes 1, 10, 10, 10, 10, 10): the
+    pool offsets, slot offsets and per-sequence logits stride of the deeper layers, one or two
+    sampled rows per layer."""
+    w = synth.WORKLOADS["llama2_7b"]
+    assert w.frontier_sizes == [1, 10, 10, 10, 10, 10]
+    bufs = _sampled_rows(w, [[(0, 0)], [(0, 9)], [(0, 2)], [(0, 0), (0, 7)], [(0, 5)], [(0, 9)]])
+    pool = {k: host(v) for k, v in bufs.pool.items()}
+    t = orc.tree_finalize(pool["tok"][0], pool["score"][0], pool["parent"][0], pool["qslot"][0],
+                          5, 12, pool_branch=pool["branch"][0])
+    for key in ("tok", "parent", "depth", "branch", "qslot"):
+        assert host(bufs.tree[key])[0].tolist() == t[key].tolist(), key
 
 
 def test_expand_llama2_13b_batch4_sampled_rows():
@@ -214,3 +338,32 @@ def test_expand_llama2_70b_shape_two_experts():
     # the host-side weight generation of this test affordable
     w = synth.scaled(synth.WORKLOADS["llama2_70b_layer"], n_experts=2, name="llama2_70b_n2")
     _sampled_rows(w, [[(0, 0)], [(0, 5)]])
+
+
+class _LazyExperts:
+    """w_gate / w_up / w_down of a workload whose experts are drawn one at a time."""
+
+    def __init__(self, w, name):
+        self.w, self.name = w, name
+
+    def __getitem__(self, e):
+        return synth.expert_weight(self.w, self.name, int(e))
+
+
+def test_expand_llama2_70b_shape_four_experts():
+    """The 70B layer shape as configured (N = 4, hidden 8192, inner 28672): 5.6 GB of bf16 expert
+    weights on the device.  The host never holds more than one expert matrix in fp32: device
+    tensors are filled expert by expert and the oracle draws the experts it needs again."""
+    w = synth.WORKLOADS["llama2_70b_layer"]
+    assert w.n_experts == 4 and w.inter == 28672
+    small = synth.shared_weights(w)
+    wts = dict(small)
+    wts_dev = {k: dev(v, w.dtype) for k, v in small.items()}
+    for name, shape in (("w_gate", (w.inter, w.hidden)), ("w_up", (w.inter, w.hidden)),
+                        ("w_down", (w.hidden, w.inter))):
+        t = torch.empty((w.n_experts,) + shape, dtype=torch.bfloat16, device="cuda")
+        for e in range(w.n_experts):
+            t[e].copy_(dev(synth.expert_weight(w, name, e), w.dtype))
+        wts_dev[name] = t
+        wts[name] = _LazyExperts(w, name)
+    _sampled_rows(w, [[(0, 0)], [(0, 4)]], wts=wts, wts_dev=wts_dev)

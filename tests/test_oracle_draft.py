@@ -75,6 +75,18 @@ def test_rmsnorm_unit_rms():
     assert np.allclose(orc.rmsnorm(u, g, 0.0), x * g, atol=1e-12)
 
 
+def test_rmsnorm_epsilon_sits_inside_the_square_root():
+    # constant row c: mean square = c^2, so x = c / sqrt(c^2 + eps) in closed form.  With
+    # c = 3, eps = 16 that is 3/5; an epsilon added outside the root would give 3/19, an
+    # epsilon ignored 1, an epsilon on the sum instead of the mean 3/sqrt(9 + 16/H).
+    x = orc.rmsnorm(np.full((2, 8), 3.0), None, 16.0)
+    assert np.allclose(x, 0.6, atol=1e-15)
+    x = orc.rmsnorm(np.full((1, 4), -3.0), np.array([1.0, 2.0, -1.0, 0.5]), 16.0)
+    assert np.allclose(x, [[-0.6, -1.2, 0.6, -0.3]], atol=1e-15)
+    # a zero row stays zero instead of dividing by zero
+    assert np.all(orc.rmsnorm(np.zeros((1, 4)), None, 1e-5) == 0.0)
+
+
 # ----------------------------------------------------------------- experts (Eq. 3)
 def test_expert_ffn_against_pure_python_loops():
     rng = np.random.default_rng(4)
