@@ -92,10 +92,11 @@ int jk_set_tensor_path(jk_ctx* ctx, int32_t enable);
  * within their limit, driver entry point for tensor maps found), else 0. */
 int jk_tensor_path_active(jk_ctx* ctx);
 /* Which tensor-core kernel runs jk_tree_verify_attn for bf16: 0 = chosen per call from the sizes
- * (default), 1 = one CTA per (query block, key slice), 2 = the persistent kernel that deals key
- * tiles evenly to one CTA per SM (falls back to 1 where its limits do not hold).  Both compute
- * the operation of arXiv 2502.06282 Sec. 2.1 step 2 with the mask of Fig. 4; the choice only
- * affects speed.  Returns JK_ERR_SHAPE for another value. */
+ * (default), 1 = one CTA per (query block, key slice) with a merge kernel, 2 = the persistent
+ * kernel that deals key tiles evenly to one CTA per SM, 3 = the kernel whose key slices form a
+ * thread-block cluster and merge through distributed shared memory (2 and 3 fall back to 1 where
+ * their limits do not hold).  All compute the operation of arXiv 2502.06282 Sec. 2.1 step 2 with
+ * the mask of Fig. 4; the choice only affects speed.  Returns JK_ERR_SHAPE for another value. */
 int jk_set_attn_kernel(jk_ctx* ctx, int32_t mode);
 
 /* Diagnostics (the paper has no counterpart): with max_launches > 0 every kernel launch of this

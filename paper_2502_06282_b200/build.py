@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libjakiro.so")
-SOURCES = ["jk_api.cu", "jk_expand.cu", "jk_gemm_tc.cu", "jk_attn.cu", "jk_attn_tc.cu", "jk_attn_sk.cu",
+SOURCES = ["jk_api.cu", "jk_expand.cu", "jk_gemm_tc.cu", "jk_attn.cu", "jk_attn_tc.cu", "jk_attn_sk.cu", "jk_attn_cl.cu",
            "jk_accept.cu"]
 
 

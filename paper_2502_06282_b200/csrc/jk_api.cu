@@ -8,6 +8,7 @@ size_t jk_tc_partial_bytes(const jk_config& c);   // jk_gemm_tc.cu
 void jk_tc_destroy(jk_ctx* ctx);                  // jk_gemm_tc.cu
 static void prof_free(jk_ctx* ctx);
 void jk_attn_tc_destroy(jk_ctx* ctx);             // jk_attn_tc.cu
+void jk_attn_cl_destroy(jk_ctx* ctx);             // jk_attn_cl.cu
 
 static int validate_config(const jk_config& c) {
   if (c.dtype != JK_F32 && c.dtype != JK_BF16) return JK_ERR_DTYPE;
@@ -94,6 +95,7 @@ extern "C" int jk_destroy(jk_ctx* ctx) {
   if (!ctx) return JK_ERR_NULL;
   jk_tc_destroy(ctx);
   jk_attn_tc_destroy(ctx);
+  jk_attn_cl_destroy(ctx);
   if (ctx->prof.cap) prof_free(ctx);
   free(ctx);
   return JK_OK;
@@ -120,7 +122,7 @@ extern "C" int jk_set_tensor_path(jk_ctx* ctx, int32_t enable) {
 
 extern "C" int jk_set_attn_kernel(jk_ctx* ctx, int32_t mode) {
   if (!ctx) return JK_ERR_NULL;
-  if (mode < 0 || mode > 2) return JK_ERR_SHAPE;
+  if (mode < 0 || mode > 3) return JK_ERR_SHAPE;
   ctx->attn_kernel = mode;
   return JK_OK;
 }

@@ -411,6 +411,12 @@ int jk_attn_tc_maps(jk_ctx* ctx, const void* kc, const void* vc, int64_t sb, int
   return JK_OK;
 }
 
+// jk_attn_cl.cu: the cluster-merged kernel for small calls
+int jk_attn_cl_plan(jk_ctx* ctx, int B, int M, int cache_rows);
+int jk_attn_cl(jk_ctx* ctx, cudaStream_t st, int n_split, int B, int M, const void* q,
+               const void* kc, const void* vc, int64_t sb, int64_t sh, int cache_rows,
+               const int32_t* kv_len, const int32_t* parent, float scale, void* out);
+
 // jk_attn_sk.cu: the persistent pipelined kernel
 int jk_attn_sk_usable(const jk_ctx* ctx, int B, int M, int cache_rows);
 int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const void* kc,
@@ -433,6 +439,17 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                       (ctx->attn_kernel == 0 && units >= 8ll * ctx->sm_count);
     if (want && jk_attn_sk_usable(ctx, B, M, cache_rows))
       return jk_attn_sk(ctx, st, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale, out);
+  }
+  // Opt-in (mode 3): the slices of a query block form a cluster and merge through distributed
+  // shared memory, when a cluster size exists whose whole grid is resident at once.  It saves the
+  // partials' trip through global memory and the merge launch, but with one CTA per SM its two or
+  // three key tiles per CTA run one after the other, and at the benchmarked shapes it measured
+  // slower than one CTA per slice (17.4 against 13.8 us at the LLaMA2-7B shape).
+  if (ctx->attn_kernel == 3) {
+    const int ns = jk_attn_cl_plan(ctx, B, M, cache_rows);
+    if (ns > 0)
+      return jk_attn_cl(ctx, st, ns, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale,
+                        out);
   }
   CUtensorMap mk, mv;
   if (jk_attn_tc_maps(ctx, kc, vc, sb, sh, cache_rows, &mk, &mv) != JK_OK) return JK_ERR_CUDA;

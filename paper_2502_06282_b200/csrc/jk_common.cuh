@@ -73,10 +73,12 @@ struct jk_ctx {
   int sm_count;           // filled at the first launch
   int attn_smem_set;
   int attn_sk_smem_set;
-  int attn_kernel;        // 0 = by size, 1 = CTA per (query block, key slice), 2 = persistent
+  int attn_kernel;        // 0 = by size, 1 = CTA per (query block, key slice), 2 = persistent,
+                          // 3 = cluster-merged
   char cuda_err[256];
   void* tc_state;         // tensor-core path bookkeeping (tensor maps), host memory
   void* attn_tc_state;    // tensor maps of the KV caches seen by the attention kernel
+  void* attn_cl_state;    // cluster-merged attention kernel: occupancy answers per cluster size
   jk_prof prof;
 };
 

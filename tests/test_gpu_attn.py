@@ -50,9 +50,10 @@ def test_attn_tiny(name, kind):
 
 
 @pytest.mark.parametrize("kind", ["chain", "star", "binary", "random"])
-def test_attn_tiny_persistent_kernel(kind):
+@pytest.mark.parametrize("kernel", [1, 2, 3])
+def test_attn_tiny_every_tensor_core_kernel(kind, kernel):
     w = synth.WORKLOADS["tiny_bf16"]
-    got, ref = _run(w, _trees(w, kind), kernel=2)
+    got, ref = _run(w, _trees(w, kind), kernel=kernel)
     assert rel_err(got, ref) <= TOL[w.dtype]
 
 
@@ -72,8 +73,9 @@ def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype=dtype, prefix=P, tree_size=M,
                      n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, batch=B, depth=6,
                      seed=900 + P + M)
-    # bf16: both tensor-core kernels (1 = CTA per key slice, 2 = persistent); f32: CUDA cores
-    for kernel in ((1, 2) if dtype == "bf16" else (0,)):
+    # bf16: every tensor-core kernel (1 = CTA per key slice, 2 = persistent, 3 = cluster-merged);
+    # f32: CUDA cores
+    for kernel in ((1, 2, 3) if dtype == "bf16" else (0,)):
         got, ref = _run(w, _trees(w, "random"), ragged=True, kernel=kernel)
         assert rel_err(got, ref) <= TOL[dtype], kernel
 
@@ -84,9 +86,9 @@ def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     ("llama3_8b", (0, 17), False),              # GQA 32/8, P = 4096: two query blocks per kv head
     ("llama2_70b_layer", (9, 63), False),       # GQA 64/8, P = 4096: four query blocks per kv head
 ])
-@pytest.mark.parametrize("kernel", [0, 1, 2])
+@pytest.mark.parametrize("kernel", [0, 1, 2, 3])
 def test_attn_full_shapes_sampled_heads(name, heads, ragged, kernel):
-    """Full-size shapes (0 = the kernel the library picks, as benchmarked; 1, 2 = each kernel
+    """Full-size shapes (0 = the kernel the library picks, as benchmarked; 1, 2, 3 = each kernel
     forced); the oracle checks a few q heads."""
     w = synth.WORKLOADS[name]
     par = _trees(w, "random")
@@ -121,11 +123,12 @@ def test_attn_reports_a_cache_that_is_too_short():
     assert ctx.read_status() == 0          # reading clears it
 
 
-def test_attn_persistent_kernel_reports_a_cache_that_is_too_short():
+@pytest.mark.parametrize("kernel", [2, 3])
+def test_attn_tensor_core_kernels_report_a_cache_that_is_too_short(kernel):
     w = synth.WORKLOADS["tiny_bf16"]
     q, k, v, kv_len = synth.attn_inputs(w)
     ctx = jk.Context.for_workload(w)
-    ctx.set_attn_kernel(2)
+    ctx.set_attn_kernel(kernel)
     qd, kd, vd = dev(q, w.dtype), dev(k, w.dtype), dev(v, w.dtype)
     out = torch.zeros_like(qd)
     bad_len = dev(np.array([k.shape[2] - w.tree_size + 1] * w.batch, dtype=np.int32))
@@ -135,7 +138,7 @@ def test_attn_persistent_kernel_reports_a_cache_that_is_too_short():
     assert ctx.read_status() == 0
 
 
-@pytest.mark.parametrize("kernel", [1, 2])
+@pytest.mark.parametrize("kernel", [1, 2, 3])
 def test_attn_is_bitwise_reproducible(kernel):
     """Slices are merged in a fixed order: two calls on the same inputs give the same bits."""
     w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype="bf16", prefix=1500, tree_size=60,
@@ -155,7 +158,8 @@ def test_attn_is_bitwise_reproducible(kernel):
     assert torch.equal(outs[0], outs[1])
 
 
-@pytest.mark.parametrize("dtype,kernel", [("f32", 0), ("bf16", 0), ("bf16", 1), ("bf16", 2)])
+@pytest.mark.parametrize("dtype,kernel", [("f32", 0), ("bf16", 0), ("bf16", 1), ("bf16", 2),
+                                          ("bf16", 3)])
 def test_attn_ignores_cache_rows_past_the_tree(dtype, kernel):
     """The operation is defined over cache rows c < kv_len + M only (Sec. 2.1 step 2).  Rows
     between kv_len + M and the cache capacity belong to nobody: here they hold NaN (as a pool
