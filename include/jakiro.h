@@ -107,6 +107,10 @@ int jk_set_attn_kernel(jk_ctx* ctx, int32_t mode);
  * device memory is allocated. */
 int jk_profile_enable(jk_ctx* ctx, int32_t max_launches);
 int jk_profile_collect(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count);
+/* As jk_profile_collect, but the recorded event pairs are kept.  When the calls were recorded into
+ * a CUDA graph (stream capture with profiling enabled turns every event record into a graph
+ * node), every replay of the graph records the same events again: read them after each replay. */
+int jk_profile_read(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count);
 int32_t jk_profile_stage_count(void);
 const char* jk_profile_stage_name(int32_t stage);
 

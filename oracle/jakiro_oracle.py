@@ -33,6 +33,20 @@ What each function follows:
                         resampling (Sec. 2.1 steps 2-3), applied sibling by
                         sibling down the tree
   compact_kv            move the accepted nodes' KV rows behind the prefix
+  grow_static_tree      the same draft layers under a predefined (Eagle-1 style)
+                        tree shape instead of the score-driven one (Sec. 3.1.2,
+                        last paragraph: both policies are usable)
+  contrastive_features  Eq. 6-7: f^moe and f^const from the two selected
+                        experts' outputs (Sec. 3.2)
+  draft_expand_contrastive, grow_tree_hybrid
+                        Eq. 8 and the hybrid schedule of Sec. 3.2: autoregressive
+                        passes from logits^moe, and logits^const of the last pass
+                        proposing one token further, so that a tree of depth D
+                        costs D-1 draft passes
+  rope, draft_pre_block Eq. 1 and the Eagle-style input path described before
+                        it (Sec. 3.1.2): token embedding and the parent's
+                        feature concatenated, the reduction layer, then
+                        u = Attn(h) + h with the draft layer's own KV cache
 
 Parity status: every function is pinned by tests/test_oracle_*.py to closed
 forms, brute force or invariants, with two exceptions that stay
@@ -40,7 +54,10 @@ forms, brute force or invariants, with two exceptions that stay
 branch feature (the printed Eq. 4 is ambiguous; only b_1 + b_2 - u = f ties it
 to Eq. 3), and (2) exact losslessness of accept_sampling when the children
 are deterministic top-k tokens rather than samples from q (pinned only in the
-sampled-children mode).
+sampled-children mode).  Readings the paper leaves open in the later functions
+(where the proposals of logits^const hang in the tree, no normalisation and
+LLaMA-style rotary positions in the draft attention) are stated at the
+functions; their arithmetic is pinned, the readings themselves cannot be.
 """
 from __future__ import annotations
 
@@ -467,3 +484,249 @@ def compact_kv(cache: np.ndarray, prefix_len: int, acc_idx: Sequence[int]) -> np
     for j, a in enumerate(acc_idx):
         out[:, prefix_len + 1 + j, :] = cache[:, prefix_len + int(a), :]
     return out
+
+
+# --------------------------------------------------------------------------
+# static tree policy (Sec. 3.1.2, last paragraph)
+# --------------------------------------------------------------------------
+def grow_static_tree(u_of_path, weights: Dict[str, np.ndarray], paths: Sequence[Tuple[int, ...]],
+                     k_e: int, root_tok: int, top_k: int = 2, **kw) -> Dict[str, np.ndarray]:
+    """One sequence under a predefined tree shape.  `paths` lists the tree's
+    nodes below the root as tuples of child ranks: rank c of a node is its
+    c-th candidate in child order (left branch ranks 0..k_e-1, then the right
+    branch), so (0,) is the root's best left-branch child and (k_e, 0) the best
+    left-branch child of the root's best right-branch child.  Every prefix of
+    a listed path must be listed.  A node is expanded iff it has listed
+    children; which tokens fill the shape depends on the draft, the shape
+    itself never does.  `u_of_path(path)` returns the hidden state u [H] of the
+    node at `path` (() = root).  Nodes are numbered root first, then by
+    (depth, path) ascending, which keeps parent[i] < i, depth non-decreasing
+    and every node's children contiguous in child order.  Returns tok, parent,
+    depth, branch, score per node and the logits [K, V] of every expanded
+    node (dict keyed by path)."""
+    paths = sorted(set(tuple(p) for p in paths), key=lambda p: (len(p), p))
+    listed = set(paths)
+    for p in paths:
+        if len(p) > 1 and p[:-1] not in listed:
+            raise ValueError("a listed node whose parent is not listed")
+        if not 0 <= p[-1] < top_k * k_e:
+            raise ValueError("child rank outside the candidate list")
+    order = [()] + paths
+    index = {p: i for i, p in enumerate(order)}
+    n = len(order)
+    tok = np.zeros(n, dtype=np.int32)
+    parent = np.full(n, -1, dtype=np.int32)
+    depth = np.zeros(n, dtype=np.int32)
+    branch = np.zeros(n, dtype=np.int32)
+    score = np.zeros(n, dtype=F64)
+    tok[0] = root_tok
+    logits_of = {}
+    expanded = [p for p in order if any(q[:-1] == p for q in paths)]
+    for p in expanded:
+        u = np.asarray(u_of_path(p), dtype=F64)[None, None, :]
+        out = draft_expand(u, np.array([[score[index[p]]]]), weights, k_e, 1, top_k, **kw)
+        logits_of[p] = out["logits"][0, 0]
+        cand_tok = out["tok"][0, 0].reshape(-1)          # child order: branch, then rank
+        cand_score = out["score"][0, 0].reshape(-1)
+        for q in paths:
+            if q[:-1] == p:
+                i = index[q]
+                tok[i] = cand_tok[q[-1]]
+                score[i] = cand_score[q[-1]]
+                parent[i] = index[p]
+                depth[i] = len(q)
+                branch[i] = q[-1] // k_e
+    return {"tok": tok, "parent": parent, "depth": depth, "branch": branch, "score": score,
+            "logits": logits_of, "order": order}
+
+
+# --------------------------------------------------------------------------
+# contrastive head and hybrid parallel decoding (Sec. 3.2, Eq. 6-8)
+# --------------------------------------------------------------------------
+def contrastive_features(y: np.ndarray, gates: np.ndarray, alpha: float, beta: float
+                         ) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 6-7 for one node.  y [2, H] are the outputs f^top1, f^top2 of the
+    two selected experts (larger score first), gates their scores:
+    f^moe = s^top1 f^top1 + s^top2 f^top2, f^const = beta f^top1 - alpha f^top2."""
+    y = np.asarray(y, dtype=F64)
+    f_moe = gates[0] * y[0] + gates[1] * y[1]
+    f_const = beta * y[0] - alpha * y[1]
+    return f_moe, f_const
+
+
+def draft_expand_contrastive(u: np.ndarray, parent_score: np.ndarray,
+                             weights: Dict[str, np.ndarray], k_e: int, width: int, alpha: float,
+                             beta: float, last_pass: bool, rms_eps: float = 1e-5,
+                             use_pre_norm: bool = True, branch_residual: bool = True
+                             ) -> Dict[str, np.ndarray]:
+    """One draft pass in the contrastive mode (Eq. 6-8) for u [B, F, H].  Row 0
+    of a node's logits is Head(f^moe), row 1 is Head(f^const); with
+    branch_residual the residual u is added to both head inputs, as it is in
+    Eq. 3 (then row 0 is the head of the combined feature f of Eq. 3 itself).
+    Children: the k_e best tokens of row 0 are the node's children, scored as
+    in branch_topk.  Row 1 predicts the token after the next one (the
+    parallel-decoding head of Sec. 3.2): its k_e best tokens hang under the
+    node's best row-0 child, with score = that child's score + their
+    log-probability under row 1.  They count only in the last pass of a step
+    (score -inf otherwise) and are never expanded.  Reading: the paper does not
+    say under which child the row-1 proposals hang; the best one is the choice
+    that keeps the candidate count of a pass unchanged."""
+    u = np.asarray(u, dtype=F64)
+    B, F, H = u.shape
+    V = weights["lm_head"].shape[0]
+    x = rmsnorm(u, weights.get("norm_weight"), rms_eps) if use_pre_norm else u.copy()
+    probs = router_scores(x, weights["router"])
+    expert = np.zeros((B, F, 2), dtype=np.int32)
+    gate = np.zeros((B, F, 2), dtype=F64)
+    feat = np.zeros((B, F, H), dtype=F64)
+    logits = np.zeros((B, F, 2, V), dtype=F64)
+    tok = np.zeros((B, F, 2, k_e), dtype=np.int32)
+    score = np.zeros((B, F, 2, k_e), dtype=F64)
+    lse = np.zeros((B, F, 2), dtype=F64)
+    for b in range(B):
+        for f in range(F):
+            ids, g = topk_gate(probs[b, f], 2)
+            expert[b, f], gate[b, f] = ids, g
+            y, _, ff = moe_features(u[b, f], x[b, f], ids, g, weights, True)
+            feat[b, f] = ff                                   # Eq. 3, fed to the next pass
+            f_moe, f_const = contrastive_features(y, g, alpha, beta)
+            if branch_residual:
+                f_moe, f_const = f_moe + u[b, f], f_const + u[b, f]
+            logits[b, f] = head_logits(np.stack([f_moe, f_const]), weights["lm_head"])
+            tok[b, f, 0], score[b, f, 0], lse[b, f, 0] = branch_topk(
+                logits[b, f, 0], k_e, float(parent_score[b, f]))
+            tok[b, f, 1], score[b, f, 1], lse[b, f, 1] = branch_topk(
+                logits[b, f, 1], k_e, float(score[b, f, 0, 0]))
+            if not last_pass:
+                score[b, f, 1, :] = -np.inf
+    n_cand = F * 2 * k_e
+    wsel = min(width, F * k_e)
+    frontier = np.zeros((B, wsel), dtype=np.int32)
+    for b in range(B):
+        # only row-0 children can be expanded: the others are masked out of the selection
+        sc = score[b].copy()
+        sc[:, 1, :] = -np.inf
+        frontier[b] = frontier_select(sc.reshape(-1), wsel)
+    return {"probs": probs, "expert": expert, "gate": gate, "feat": feat, "logits": logits,
+            "tok": tok, "score": score, "lse": lse, "frontier": frontier, "n_cand": n_cand}
+
+
+def grow_tree_hybrid(u_layers: Sequence[np.ndarray], weights: Dict[str, np.ndarray], k_e: int,
+                     width: int, alpha: float, beta: float, **kw) -> Dict[str, np.ndarray]:
+    """The hybrid schedule of Sec. 3.2: len(u_layers) = D-1 contrastive passes
+    build a tree of depth up to D, because the last pass's row-1 proposals sit
+    one level below its row-0 children.  Pool layout as in grow_tree; the
+    parent of a row-1 candidate is the generation index of its node's best
+    row-0 child."""
+    B = u_layers[0].shape[0]
+    tok_l, score_l, parent_l, qslot_l, branch_l, logits_l = [], [], [], [], [], []
+    parent_score = np.zeros((B, 1), dtype=F64)
+    parent_gidx = np.full((B, 1), -1, dtype=np.int32)
+    gidx_base, slot_base = 0, 0
+    for l, u in enumerate(u_layers):
+        F = u.shape[1]
+        last = l == len(u_layers) - 1
+        out = draft_expand_contrastive(u, parent_score, weights, k_e, width, alpha, beta, last, **kw)
+        n_cand = F * 2 * k_e
+        par = np.zeros((B, F, 2, k_e), dtype=np.int32)
+        for f in range(F):
+            par[:, f, 0, :] = parent_gidx[:, f:f + 1]
+            par[:, f, 1, :] = gidx_base + (f * 2 + 0) * k_e + 0
+        q = np.full((B, n_cand), -1, dtype=np.int32)
+        if not last:
+            for b in range(B):
+                q[b, out["frontier"][b]] = slot_base + F + np.arange(out["frontier"].shape[1])
+        tok_l.append(out["tok"].reshape(B, n_cand))
+        score_l.append(out["score"].reshape(B, n_cand))
+        parent_l.append(par.reshape(B, n_cand))
+        qslot_l.append(q)
+        branch_l.append(np.tile(np.repeat(np.arange(2), k_e), F)[None].repeat(B, 0))
+        logits_l.append(out["logits"])
+        parent_score = np.take_along_axis(out["score"].reshape(B, n_cand), out["frontier"], 1)
+        parent_gidx = (gidx_base + out["frontier"]).astype(np.int32)
+        gidx_base += n_cand
+        slot_base += F
+    return {"tok": np.concatenate(tok_l, 1), "score": np.concatenate(score_l, 1),
+            "parent": np.concatenate(parent_l, 1), "qslot": np.concatenate(qslot_l, 1),
+            "branch": np.concatenate(branch_l, 1).astype(np.int32),
+            "logits": np.concatenate(logits_l, 1)}
+
+
+# --------------------------------------------------------------------------
+# draft pre-MoE block (Eq. 1 and the paragraph before it)
+# --------------------------------------------------------------------------
+def rope(x: np.ndarray, pos: float, theta: float) -> np.ndarray:
+    """Rotary position embedding of one head vector x [d] at position `pos`,
+    LLaMA convention: the vector is split in halves (x1, x2), pair i is
+    (x1[i], x2[i]) and rotates by pos / theta^(2 i / d)."""
+    x = np.asarray(x, dtype=F64)
+    d = x.shape[-1]
+    half = d // 2
+    ang = pos / theta ** (2.0 * np.arange(half) / d)
+    c, s_ = np.cos(ang), np.sin(ang)
+    x1, x2 = x[:half], x[half:]
+    return np.concatenate([x1 * c - x2 * s_, x2 * c + x1 * s_])
+
+
+def draft_pre_block(tok: np.ndarray, f_prev: np.ndarray, pw: Dict[str, np.ndarray],
+                    k_cache: np.ndarray, v_cache: np.ndarray, prefix_len: int,
+                    slots: Sequence[int], slot_parent: np.ndarray, n_q_heads: int,
+                    n_kv_heads: int, theta: float, scale: float
+                    ) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Eq. 1 for the F nodes of one draft layer of one sequence.
+    tok [F]: the nodes' tokens; f_prev [F, H]: each node's parent feature (the
+    f of Eq. 3 the parent's pass produced; for the root the target model's
+    last feature).  pw: emb [V, H], w_fc [H, 2H], b_fc [H] or None, w_q
+    [Hq d, H], w_k, w_v [Hkv d, H], w_o [H, Hq d].
+      h = W_fc [emb(tok) ; f_prev] (+ b_fc)          (the reduction layer)
+      q, k, v = W_q h, W_k h, W_v h per head, q and k rotated to position
+      prefix_len + depth of the node; k, v are stored in the draft layer's own
+      cache [Hkv, cap, d] at row prefix_len + slot (slots = the nodes' rows
+      among the step's expanded nodes, root = 0);
+      Attn: every node attends over the committed prefix rows and the rows of
+      itself and its ancestors (slot_parent [S], -1 for the root);
+      u = W_o Attn + h.
+    No normalisation is applied (Eagle-style drafts drop the input norm of
+    their single layer; the note after Eq. 5 leaves norms out).  Returns
+    (u [F, H], h [F, H], and the updated caches)."""
+    emb = np.asarray(pw["emb"], dtype=F64)
+    F = len(tok)
+    H = emb.shape[1]
+    d = pw["w_q"].shape[0] // n_q_heads
+    G = n_q_heads // n_kv_heads
+    kc = np.array(k_cache, dtype=F64, copy=True)
+    vc = np.array(v_cache, dtype=F64, copy=True)
+    depth = np.zeros(len(slot_parent), dtype=np.int64)
+    for s_ in range(1, len(slot_parent)):
+        if slot_parent[s_] >= 0:
+            depth[s_] = depth[slot_parent[s_]] + 1
+    h = np.zeros((F, H), dtype=F64)
+    qs = np.zeros((F, n_q_heads, d), dtype=F64)
+    for i in range(F):
+        x = np.concatenate([emb[int(tok[i])], np.asarray(f_prev[i], dtype=F64)])
+        h[i] = np.asarray(pw["w_fc"], dtype=F64) @ x
+        if pw.get("b_fc") is not None:
+            h[i] = h[i] + np.asarray(pw["b_fc"], dtype=F64)
+        pos = prefix_len + int(depth[slots[i]])
+        q = (np.asarray(pw["w_q"], dtype=F64) @ h[i]).reshape(n_q_heads, d)
+        k = (np.asarray(pw["w_k"], dtype=F64) @ h[i]).reshape(n_kv_heads, d)
+        v = (np.asarray(pw["w_v"], dtype=F64) @ h[i]).reshape(n_kv_heads, d)
+        for hh in range(n_q_heads):
+            qs[i, hh] = rope(q[hh], pos, theta)
+        for hh in range(n_kv_heads):
+            kc[hh, prefix_len + slots[i]] = rope(k[hh], pos, theta)
+            vc[hh, prefix_len + slots[i]] = v[hh]
+    u = np.zeros((F, H), dtype=F64)
+    for i in range(F):
+        anc = []
+        t = int(slots[i])
+        while t >= 0:
+            anc.append(t)
+            t = int(slot_parent[t])
+        cols = list(range(prefix_len)) + [prefix_len + a for a in sorted(anc)]
+        o = np.zeros((n_q_heads, d), dtype=F64)
+        for hh in range(n_q_heads):
+            kk, vv = kc[hh // G, cols], vc[hh // G, cols]
+            o[hh] = softmax(scale * (kk @ qs[i, hh])) @ vv
+        u[i] = np.asarray(pw["w_o"], dtype=F64) @ o.reshape(-1) + h[i]
+    return u, h, kc, vc

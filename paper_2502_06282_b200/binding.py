@@ -26,7 +26,7 @@ EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", 
            "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
            "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
            "jk_profile_stage_name", "jk_tree_verify_attn_static", "jk_tensor_path_active",
-           "jk_set_attn_kernel"]
+           "jk_set_attn_kernel", "jk_profile_read"]
 
 
 class JkConfig(C.Structure):
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
                                             vp, vp, vp, vp]
         L.jk_profile_enable.argtypes = [vp, i32]
         L.jk_profile_collect.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
+        L.jk_profile_read.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
         L.jk_profile_stage_count.argtypes = []
         L.jk_profile_stage_name.argtypes = [i32]
         L.jk_profile_stage_name.restype = C.c_char_p
@@ -198,12 +199,14 @@ class Context:
     def profile_enable(self, max_launches: int):
         self._check(lib().jk_profile_enable(self._h, max_launches), "jk_profile_enable")
 
-    def profile_collect(self) -> Dict[str, tuple]:
-        """{stage name: (total ms, launches)} since the last collect; synchronises."""
+    def profile_collect(self, keep: bool = False) -> Dict[str, tuple]:
+        """{stage name: (total ms, launches)} since the last collect; synchronises.  keep=True
+        leaves the recorded event pairs in place (jk_profile_read), for graph replays."""
         n = lib().jk_profile_stage_count()
         ms = (C.c_float * n)()
         cnt = (C.c_int32 * n)()
-        self._check(lib().jk_profile_collect(self._h, _stream(), ms, cnt), "jk_profile_collect")
+        fn = lib().jk_profile_read if keep else lib().jk_profile_collect
+        self._check(fn(self._h, _stream(), ms, cnt), "jk_profile_collect")
         return {lib().jk_profile_stage_name(i).decode(): (float(ms[i]), int(cnt[i]))
                 for i in range(n) if cnt[i]}
 

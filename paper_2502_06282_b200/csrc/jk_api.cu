@@ -193,7 +193,7 @@ extern "C" int jk_profile_enable(jk_ctx* ctx, int32_t max_launches) {
   return JK_OK;
 }
 
-extern "C" int jk_profile_collect(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count) {
+static int prof_sum(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count, bool reset) {
   if (!ctx || !host_ms || !host_count) return JK_ERR_NULL;
   for (int s = 0; s < JK_N_STAGES; ++s) { host_ms[s] = 0.f; host_count[s] = 0; }
   jk_prof& p = ctx->prof;
@@ -205,8 +205,16 @@ extern "C" int jk_profile_collect(jk_ctx* ctx, void* stream, float* host_ms, int
     host_ms[p.stage[i]] += ms;
     host_count[p.stage[i]] += 1;
   }
-  p.n = 0;
+  if (reset) p.n = 0;
   return JK_OK;
+}
+
+extern "C" int jk_profile_collect(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count) {
+  return prof_sum(ctx, stream, host_ms, host_count, true);
+}
+
+extern "C" int jk_profile_read(jk_ctx* ctx, void* stream, float* host_ms, int32_t* host_count) {
+  return prof_sum(ctx, stream, host_ms, host_count, false);
 }
 
 extern "C" int32_t jk_profile_stage_count(void) { return JK_N_STAGES; }
