@@ -66,6 +66,11 @@ typedef struct {
   int32_t use_pre_norm;     /* 1: router and experts see RMSNorm(u) * norm_weight (the
                                normalisation Sec. 3.1.2 leaves out of Eq. 1-5); 0: u     */
   int32_t branch_residual;  /* 1: branch feature = g_r * Expert_r(x) + u; 0: g_r * Expert_r(x) */
+  int32_t head_mode;        /* 0: decoupled heads, one logits row per selected expert (Eq. 4);
+                               1: contrastive heads (Sec. 3.2, Eq. 6-8; needs top_k = 2): row 0 is
+                               Head(f^moe), row 1 is Head(f^const), see jk_draft_expand            */
+  float contrast_alpha;     /* alpha and beta of Eq. 7: f^const = beta f^top1 - alpha f^top2       */
+  float contrast_beta;
 } jk_config;
 
 typedef struct jk_ctx jk_ctx;
@@ -167,6 +172,18 @@ typedef struct {
  *                      width = 0 skips the selection (last layer)
  *   next_parent_score  f32 [B, W'] their scores
  *   next_parent_gidx   i32 [B, W'] their generation indices
+ * Static tree policy (Sec. 3.1.2, last paragraph: the predefined tree of Eagle-1 is as usable as
+ * the dynamic one): with static_select != NULL the next frontier is not chosen by score but
+ * read from static_select, i32 [width] device, the flat child indices of the predefined shape in
+ * frontier order, the same for every sequence; an index outside 0 .. F*K*k_e-1 sets JK_ERR_BOUNDS.
+ * Contrastive mode (cfg.head_mode = 1; Sec. 3.2, Eq. 6-8): the head inputs are
+ *   row 0: f^moe = g_1 y_1 + g_2 y_2 (+ u), row 1: f^const = beta y_1 - alpha y_2 (+ u).
+ * The k_e best tokens of row 0 are the node's children as above.  Row 1 is the parallel-decoding
+ * head: its k_e best tokens hang one level lower, under the node's best row-0 child (their pool
+ * parent is that child's generation index, their score its score plus their log-probability
+ * under row 1); they count only in a step's last pass (width = 0), get the score -inf in the
+ * others, and are never chosen for the next frontier, so W' = min(width, F*k_e).  A step of tree
+ * depth D then takes D-1 calls.
  * Errors: NULL/ALIGN/SHAPE/CAPACITY (B > max_batch, F > max_frontier)/WORKSPACE/CUDA.
  */
 int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* host_w,
@@ -175,7 +192,8 @@ int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* host_w,
                     int32_t gidx_base, int32_t slot_base,
                     float* out_probs, int32_t* out_expert, float* out_gate,
                     const jk_pool* host_pool, float* out_lse, void* out_feat, float* out_logits,
-                    int64_t logits_stride_b, int32_t* next_frontier, float* next_parent_score, int32_t* next_parent_gidx);
+                    int64_t logits_stride_b, int32_t* next_frontier, float* next_parent_score,
+                    int32_t* next_parent_gidx, const int32_t* static_select);
 
 /*
  * Build the verification tree from the pool (Sec. 3.1.2; mask as in Fig. 4): node 0 is the
@@ -185,11 +203,15 @@ int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* host_w,
  *   root_tok i32 [B]; outputs i32 [B, M]: tok, parent (-1 for the root), depth, branch, qslot
  *   (root: 0); anc u64 [B, M, 2]: bit t of the 128-bit set is 1 iff t is the node itself or
  *   one of its ancestors.
+ *   static_keep  i32 [M-1] device or NULL.  Static tree policy: the generation indices of the
+ *   predefined shape's nodes, ascending, the same for every sequence, kept instead of the M-1
+ *   best by score; a list that is not ascending, reaches past pool_n or keeps a node without
+ *   its parent sets JK_ERR_BOUNDS.
  */
 int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const jk_pool* host_pool,
                      int32_t pool_n, const int32_t* root_tok, int32_t tree_size,
                      int32_t* tok, int32_t* parent, int32_t* depth, int32_t* branch,
-                     int32_t* qslot, uint64_t* anc);
+                     int32_t* qslot, uint64_t* anc, const int32_t* static_keep);
 
 /*
  * Tree-masked attention of one target layer over all M tree tokens (Sec. 2.1 step 2):

@@ -33,7 +33,8 @@ class JkConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "hidden", "n_experts", "top_k", "inter", "vocab", "n_q_heads", "n_kv_heads", "head_dim",
         "max_batch", "max_tree", "max_depth", "max_frontier", "k_per_expert", "dtype")] + [
-        ("rms_eps", C.c_float), ("use_pre_norm", C.c_int32), ("branch_residual", C.c_int32)]
+        ("rms_eps", C.c_float), ("use_pre_norm", C.c_int32), ("branch_residual", C.c_int32),
+        ("head_mode", C.c_int32), ("contrast_alpha", C.c_float), ("contrast_beta", C.c_float)]
 
 
 class JkDraftWeights(C.Structure):
@@ -74,9 +75,9 @@ def lib() -> C.CDLL:
         L.jk_set_attn_kernel.argtypes = [vp, i32]
         L.jk_draft_expand.argtypes = [vp, vp, C.POINTER(JkDraftWeights), i32, i32, i32, vp, vp,
                                       vp, i32, i32, vp, vp, vp, C.POINTER(JkPool), vp, vp, vp,
-                                      i64, vp, vp, vp]
+                                      i64, vp, vp, vp, vp]
         L.jk_tree_finalize.argtypes = [vp, vp, i32, C.POINTER(JkPool), i32, vp, i32, vp, vp, vp,
-                                       vp, vp, vp]
+                                       vp, vp, vp, vp]
         L.jk_tree_verify_attn.argtypes = [vp, vp, i32, i32, vp, vp, vp, i64, i64, i32, vp, vp,
                                           f32, vp]
         L.jk_tree_verify_attn_static.argtypes = L.jk_tree_verify_attn.argtypes + [vp]
@@ -121,12 +122,13 @@ class Context:
 
     def __init__(self, *, hidden, n_experts, top_k, inter, vocab, n_q_heads, n_kv_heads,
                  head_dim, max_batch, max_tree, max_depth, max_frontier, k_per_expert, dtype,
-                 rms_eps=1e-5, use_pre_norm=True, branch_residual=True, device="cuda",
-                 allocate=True):
+                 rms_eps=1e-5, use_pre_norm=True, branch_residual=True, head_mode=0,
+                 contrast_alpha=0.0, contrast_beta=1.0, device="cuda", allocate=True):
         self.cfg = JkConfig(hidden, n_experts, top_k, inter, vocab, n_q_heads, n_kv_heads,
                             head_dim, max_batch, max_tree, max_depth, max_frontier,
                             k_per_expert, JK_BF16 if dtype == "bf16" else JK_F32, rms_eps,
-                            int(use_pre_norm), int(branch_residual))
+                            int(use_pre_norm), int(branch_residual), int(head_mode),
+                            float(contrast_alpha), float(contrast_beta))
         self.dtype = dtype
         self.tdtype = torch_dtype(dtype)
         self._h = C.c_void_p()
@@ -154,11 +156,13 @@ class Context:
         return base - buf.data_ptr()
 
     @classmethod
-    def for_workload(cls, w, **kw) -> "Context":
+    def for_workload(cls, w, frontier_sizes=None, **kw) -> "Context":
+        fs = w.frontier_sizes if frontier_sizes is None else frontier_sizes
+        kw.setdefault("head_mode", getattr(w, "head_mode", 0))
         return cls(hidden=w.hidden, n_experts=w.n_experts, top_k=w.top_k, inter=w.inter,
                    vocab=w.vocab, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
                    head_dim=w.head_dim, max_batch=w.batch, max_tree=w.tree_size,
-                   max_depth=w.depth, max_frontier=max(w.frontier_sizes),
+                   max_depth=w.depth, max_frontier=max(fs),
                    k_per_expert=w.k_per_expert, dtype=w.dtype, **kw)
 
     def _check(self, rc: int, where: str):
@@ -223,7 +227,8 @@ class Context:
 
     def draft_expand(self, weights, batch, n_frontier, width, u, parent_score, parent_gidx,
                      gidx_base, slot_base, out_probs, out_expert, out_gate, pool, out_lse,
-                     out_feat, out_logits, next_frontier, next_parent_score, next_parent_gidx):
+                     out_feat, out_logits, next_frontier, next_parent_score, next_parent_gidx,
+                     static_select=None):
         ws = weights if isinstance(weights, JkDraftWeights) else self.weights_struct(weights)
         ps = pool if isinstance(pool, JkPool) else self.pool_struct(pool)
         rc = lib().jk_draft_expand(
@@ -232,15 +237,16 @@ class Context:
             _ptr(out_expert), _ptr(out_gate), C.byref(ps), _ptr(out_lse), _ptr(out_feat),
             _ptr(out_logits), 0 if out_logits is None else out_logits.stride(0),
             _ptr(next_frontier), _ptr(next_parent_score),
-            _ptr(next_parent_gidx))
+            _ptr(next_parent_gidx), _ptr(static_select))
         self._check(rc, "jk_draft_expand")
 
     def tree_finalize(self, batch, pool, pool_n, root_tok, tree_size, tok, parent, depth, branch,
-                      qslot, anc):
+                      qslot, anc, static_keep=None):
         ps = pool if isinstance(pool, JkPool) else self.pool_struct(pool)
         rc = lib().jk_tree_finalize(self._h, _stream(), batch, C.byref(ps), pool_n,
                                     _ptr(root_tok), tree_size, _ptr(tok), _ptr(parent),
-                                    _ptr(depth), _ptr(branch), _ptr(qslot), _ptr(anc))
+                                    _ptr(depth), _ptr(branch), _ptr(qslot), _ptr(anc),
+                                    _ptr(static_keep))
         self._check(rc, "jk_tree_finalize")
 
     def tree_verify_attn(self, batch, tree_size, q, k_cache, v_cache, kv_len, parent, scale, out,
@@ -286,30 +292,34 @@ class Context:
 class StepBuffers:
     """Device buffers of one draft-and-verify step for a workload, allocated once."""
 
-    def __init__(self, ctx: Context, w, keep_logits: bool = True, device="cuda"):
+    def __init__(self, ctx: Context, w, keep_logits: bool = True, device="cuda",
+                 frontier_sizes=None):
+        """frontier_sizes: the expanded nodes per draft pass when they do not follow from the
+        workload's width (a predefined tree shape); default w.frontier_sizes."""
         B, K, ke, V, H = w.batch, w.top_k, w.k_per_expert, w.vocab, w.hidden
-        fs = w.frontier_sizes
-        Fm = max(fs)
+        fs = list(w.frontier_sizes if frontier_sizes is None else frontier_sizes)
+        self.frontier_sizes = fs
+        self.pool_n = sum(f * K * ke for f in fs)
+        self.n_slots = sum(fs)
         i32 = dict(dtype=torch.int32, device=device)
         f32 = dict(dtype=torch.float32, device=device)
         self.w = w
-        self.pool = {"tok": torch.empty(B, w.pool_size, **i32),
-                     "score": torch.empty(B, w.pool_size, **f32),
-                     "parent": torch.empty(B, w.pool_size, **i32),
-                     "qslot": torch.empty(B, w.pool_size, **i32),
-                     "branch": torch.empty(B, w.pool_size, **i32)}
+        self.pool = {"tok": torch.empty(B, self.pool_n, **i32),
+                     "score": torch.empty(B, self.pool_n, **f32),
+                     "parent": torch.empty(B, self.pool_n, **i32),
+                     "qslot": torch.empty(B, self.pool_n, **i32),
+                     "branch": torch.empty(B, self.pool_n, **i32)}
         self.pool_struct = ctx.pool_struct(self.pool)
         self.probs = [torch.empty(B, F, w.n_experts, **f32) for F in fs]
         self.expert = [torch.empty(B, F, K, **i32) for F in fs]
         self.gate = [torch.empty(B, F, K, **f32) for F in fs]
         self.lse = [torch.empty(B, F, K, **f32) for F in fs]
         self.feat = [torch.empty(B, F, H, dtype=ctx.tdtype, device=device) for F in fs]
-        self.logits = torch.empty(B, w.n_slots, K, V, **f32) if keep_logits else None
-        self.frontier = [torch.empty(B, min(w.width, F * K * ke), **i32) for F in fs]
-        self.parent_score = [torch.zeros(B, 1, **f32)] + [
-            torch.empty(B, min(w.width, F * K * ke), **f32) for F in fs]
-        self.parent_gidx = [torch.full((B, 1), -1, **i32)] + [
-            torch.empty(B, min(w.width, F * K * ke), **i32) for F in fs]
+        self.logits = torch.empty(B, self.n_slots, K, V, **f32) if keep_logits else None
+        nxt = fs[1:] + [1]                      # nodes chosen by pass l = nodes expanded by pass l+1
+        self.frontier = [torch.empty(B, n, **i32) for n in nxt]
+        self.parent_score = [torch.zeros(B, 1, **f32)] + [torch.empty(B, n, **f32) for n in nxt]
+        self.parent_gidx = [torch.full((B, 1), -1, **i32)] + [torch.empty(B, n, **i32) for n in nxt]
         M = w.tree_size
         self.tree = {k: torch.empty(B, M, **i32) for k in ("tok", "parent", "depth", "branch",
                                                            "qslot")}
@@ -321,11 +331,13 @@ class StepBuffers:
 
 
 def run_draft(ctx: Context, bufs: StepBuffers, weights, u_layers: Sequence[torch.Tensor],
-              root_tok: torch.Tensor, finalize: bool = True):
-    """D calls of jk_draft_expand, one per tree layer, then jk_tree_finalize.  The expanded
-    nodes' logits are kept in bufs.logits at slot order when that buffer exists."""
+              root_tok: torch.Tensor, finalize: bool = True, static_plan=None):
+    """One jk_draft_expand call per draft pass, then jk_tree_finalize.  The expanded nodes'
+    logits are kept in bufs.logits at slot order when that buffer exists.  static_plan (from
+    static_tree.plan_from_paths, with device arrays): the predefined tree shape that replaces the
+    score-driven choice of frontier and final tree."""
     w = bufs.w
-    fs = w.frontier_sizes
+    fs = bufs.frontier_sizes
     B, K, ke = w.batch, w.top_k, w.k_per_expert
     gidx_base = 0
     slot_base = 0
@@ -334,16 +346,19 @@ def run_draft(ctx: Context, bufs: StepBuffers, weights, u_layers: Sequence[torch
         out_logits = None
         if bufs.logits is not None:      # rows slot_base..slot_base+F-1 of every sequence
             out_logits = bufs.logits[:, slot_base:slot_base + F]
-        ctx.draft_expand(weights, B, F, 0 if last else w.width, u_layers[l],
+        width = 0 if last else fs[l + 1]
+        ctx.draft_expand(weights, B, F, width, u_layers[l],
                          bufs.parent_score[l], bufs.parent_gidx[l], gidx_base, slot_base,
                          bufs.probs[l], bufs.expert[l], bufs.gate[l], bufs.pool_struct,
                          bufs.lse[l], bufs.feat[l], out_logits,
                          None if last else bufs.frontier[l],
                          None if last else bufs.parent_score[l + 1],
-                         None if last else bufs.parent_gidx[l + 1])
+                         None if last else bufs.parent_gidx[l + 1],
+                         None if (last or static_plan is None) else static_plan["select"][l])
         gidx_base += F * K * ke
         slot_base += F
     if finalize:
-        ctx.tree_finalize(B, bufs.pool_struct, w.pool_size, root_tok, w.tree_size,
+        ctx.tree_finalize(B, bufs.pool_struct, bufs.pool_n, root_tok, w.tree_size,
                           bufs.tree["tok"], bufs.tree["parent"], bufs.tree["depth"],
-                          bufs.tree["branch"], bufs.tree["qslot"], bufs.anc)
+                          bufs.tree["branch"], bufs.tree["qslot"], bufs.anc,
+                          None if static_plan is None else static_plan["keep"])

@@ -26,6 +26,8 @@ static int validate_config(const jk_config& c) {
   if (c.n_kv_heads < 1 || c.n_q_heads < c.n_kv_heads || c.n_q_heads % c.n_kv_heads)
     return JK_ERR_SHAPE;
   if (!(c.rms_eps >= 0.f)) return JK_ERR_SHAPE;
+  if (c.head_mode != 0 && c.head_mode != 1) return JK_ERR_SHAPE;
+  if (c.head_mode == 1 && c.top_k != 2) return JK_ERR_SHAPE;      // Eq. 6-7 contrast two experts
   // the top-k merge keeps chunks * k_e candidates in 16 registers per lane
   if ((size_t)((c.vocab + JK_TOPK_CHUNK - 1) / JK_TOPK_CHUNK) * c.k_per_expert > 512) return JK_ERR_SHAPE;
   return JK_OK;
@@ -157,18 +159,28 @@ extern "C" int jk_read_status(jk_ctx* ctx, void* stream, int32_t* host_status) {
 }
 
 // ---------------------------------------------------------------- per-kernel timing
+// While the stream is being captured into a graph an ordinary event record only adds a
+// dependency; the "external" flavour becomes an event-record node that every replay executes,
+// which is what a timing pair needs.
+static cudaError_t prof_record(cudaEvent_t ev, cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) cs = cudaStreamCaptureStatusNone;
+  return cudaEventRecordWithFlags(ev, st, cs == cudaStreamCaptureStatusActive
+                                              ? cudaEventRecordExternal : cudaEventRecordDefault);
+}
+
 void jk_prof_begin(jk_ctx* ctx, cudaStream_t st, int stage) {
   jk_prof& p = ctx->prof;
   if (p.n >= p.cap) return;
   p.stage[p.n] = stage;
   p.stream = st;
-  if (cudaEventRecord(p.ev[2 * p.n], st) == cudaSuccess) p.open = 1;
+  if (prof_record(p.ev[2 * p.n], st) == cudaSuccess) p.open = 1;
 }
 
 void jk_prof_end(jk_ctx* ctx) {
   jk_prof& p = ctx->prof;
   p.open = 0;
-  if (cudaEventRecord(p.ev[2 * p.n + 1], p.stream) == cudaSuccess) ++p.n;
+  if (prof_record(p.ev[2 * p.n + 1], p.stream) == cudaSuccess) ++p.n;
 }
 
 static void prof_free(jk_ctx* ctx) {

@@ -225,20 +225,32 @@ __global__ void __launch_bounds__(256) k_down(
 }
 
 // Eq. 3 and the branch features: f = u + sum_r g_r y_r; b_r = g_r y_r (+ u)
+// Contrastive mode (Eq. 6-7, K = 2): b_0 = f^moe = g_1 y_1 + g_2 y_2 (+ u), b_1 = f^const =
+// beta y_1 - alpha y_2 (+ u).
 template <typename T>
 __global__ void __launch_bounds__(256) k_branch(
     const T* __restrict__ u, const float* __restrict__ ybuf, const int32_t* __restrict__ expert,
-    const float* __restrict__ gate, int K, int H, int Rp, int branch_residual,
-    T* __restrict__ bbuf, T* __restrict__ out_feat) {
+    const float* __restrict__ gate, int K, int H, int Rp, int branch_residual, int head_mode,
+    float alpha, float beta, T* __restrict__ bbuf, T* __restrict__ out_feat) {
   const int r = blockIdx.x;
   for (int h = threadIdx.x; h < H; h += blockDim.x) {
     const float uv = jk_to_float(u[(size_t)r * H + h]);
     float f = uv;
-    for (int k = 0; k < K; ++k) {
-      const int e = expert[r * K + k];
-      const float gy = gate[r * K + k] * ybuf[((size_t)e * Rp + r) * H + h];
-      f += gy;
-      bbuf[((size_t)r * K + k) * H + h] = jk_from_float<T>(branch_residual ? gy + uv : gy);
+    if (head_mode == 1) {
+      const float y0 = ybuf[((size_t)expert[r * K] * Rp + r) * H + h];
+      const float y1 = ybuf[((size_t)expert[r * K + 1] * Rp + r) * H + h];
+      const float g0y = gate[r * K] * y0, g1y = gate[r * K + 1] * y1;
+      const float fm = g0y + g1y, fc = beta * y0 - alpha * y1;
+      f = (uv + g0y) + g1y;
+      bbuf[((size_t)r * K) * H + h] = jk_from_float<T>(branch_residual ? fm + uv : fm);
+      bbuf[((size_t)r * K + 1) * H + h] = jk_from_float<T>(branch_residual ? fc + uv : fc);
+    } else {
+      for (int k = 0; k < K; ++k) {
+        const int e = expert[r * K + k];
+        const float gy = gate[r * K + k] * ybuf[((size_t)e * Rp + r) * H + h];
+        f += gy;
+        bbuf[((size_t)r * K + k) * H + h] = jk_from_float<T>(branch_residual ? gy + uv : gy);
+      }
     }
     out_feat[(size_t)r * H + h] = jk_from_float<T>(f);
   }
@@ -299,25 +311,30 @@ __global__ void __launch_bounds__(JK_TOPK_THREADS) k_topk_partial(
 }
 
 // Merge the chunk partials of every logits row of one sequence, append the children to the
-// pool, then pick the next frontier.  One block per sequence.
+// pool, then pick the next frontier (by score, or from the predefined shape's list).  One block
+// per sequence.  In contrastive mode (head_mode 1) the row-1 children hang under the node's best
+// row-0 child and only row-0 children can become frontier nodes.
 __global__ void __launch_bounds__(1024) k_expand_finish(
-    int F, int K, int k_e, int chunks, int width,
+    int F, int K, int k_e, int chunks, int width, int head_mode,
     const float* __restrict__ tk_val, const int32_t* __restrict__ tk_idx,
     const float* __restrict__ tk_ms, const float* __restrict__ parent_score,
     const int32_t* __restrict__ parent_gidx, int gidx_base, int slot_base,
-    jk_pool pool, float* __restrict__ out_lse, int32_t* __restrict__ next_frontier,
-    float* __restrict__ next_parent_score, int32_t* __restrict__ next_parent_gidx) {
+    jk_pool pool, float* __restrict__ out_lse, int rows_per_b_lse, long long lse_stride_b,
+    int32_t* __restrict__ next_frontier, float* __restrict__ next_parent_score,
+    int32_t* __restrict__ next_parent_gidx, const int32_t* __restrict__ static_select,
+    int32_t* status) {
   jk_pdl_wait();
   jk_pdl_trigger();
   constexpr int PER_MAX = 16;                   // candidates per lane held in registers
-  __shared__ float sc[JK_MAX_POOL];
+  __shared__ float sc[JK_MAX_POOL];             // cumulative score of every child
+  __shared__ float lp[JK_MAX_POOL];             // its log-probability under its own logits row
+  __shared__ int tk[JK_MAX_POOL];
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   const int rows = F * K;
   const size_t pb = (size_t)b * pool.stride_b;
   const int nc = chunks * k_e;
   for (int lr = warp; lr < rows; lr += nw) {
-    const int f = lr / K, r = lr % K;
     const size_t row = (size_t)b * rows + lr;
     // candidates of this row: the chunks' partial winners (loaded once)
     float cv[PER_MAX];
@@ -337,9 +354,8 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
       s += tk_ms[(row * chunks + c) * 2 + 1] * expf(tk_ms[(row * chunks + c) * 2] - m);
     s = jk_warp_sum(s);
     const float lse = m + logf(s);
-    if (out_lse && lane == 0) out_lse[row] = lse;
-    const float ps = parent_score[(size_t)b * F + f];
-    const int pg = parent_gidx[(size_t)b * F + f];
+    if (out_lse && lane == 0)
+      out_lse[(size_t)b * (size_t)lse_stride_b + lr] = lse;
     unsigned taken = 0u;
     for (int it = 0; it < k_e; ++it) {
       float bv = -INFINITY;
@@ -358,25 +374,60 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
       if (wi == bi && bj >= 0 && wi != INT_MAX) taken |= 1u << bj;
       if (lane == 0) {
         const int flat = lr * k_e + it;
-        const int g = gidx_base + flat;
-        const float score = ps + (wv - lse);
-        pool.tok[pb + g] = wi;
-        pool.score[pb + g] = score;
-        pool.parent[pb + g] = pg;
-        pool.qslot[pb + g] = -1;
-        pool.branch[pb + g] = r;
-        sc[flat] = score;
+        lp[flat] = wv - lse;
+        tk[flat] = wi;
       }
     }
   }
   __syncthreads();
-  if (width <= 0 || !next_frontier) return;
   const int n = rows * k_e;
-  const int wsel = min(width, n);
+  const bool last_pass = width <= 0;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int lr = i / k_e, f = lr / K, r = lr % K;
+    const float ps = parent_score[(size_t)b * F + f];
+    int pg = parent_gidx[(size_t)b * F + f];
+    float base = ps;
+    if (head_mode == 1 && r == 1) {
+      const int best0 = (f * K) * k_e;                      // the node's best row-0 child
+      base = ps + lp[best0];
+      pg = gidx_base + best0;
+    }
+    float score = base + lp[i];
+    if (head_mode == 1 && r == 1 && !last_pass) score = -INFINITY;
+    const int g = gidx_base + i;
+    pool.tok[pb + g] = tk[i];
+    pool.score[pb + g] = score;
+    pool.parent[pb + g] = pg;
+    pool.qslot[pb + g] = -1;
+    pool.branch[pb + g] = r;
+    sc[i] = score;
+  }
+  __syncthreads();
+  if (width <= 0 || !next_frontier) return;
+  const int n_sel = head_mode == 1 ? F * k_e : n;           // children that may be expanded
+  const int wsel = min(width, n_sel);
+  if (static_select) {
+    for (int i = threadIdx.x; i < wsel; i += blockDim.x) {
+      int idx = static_select[i];
+      if (idx < 0 || idx >= n || (head_mode == 1 && (idx / k_e) % K == 1)) {
+        jk_set_status(status, JK_ERR_BOUNDS);
+        idx = 0;
+      }
+      next_frontier[(size_t)b * wsel + i] = idx;
+      next_parent_score[(size_t)b * wsel + i] = sc[idx];
+      next_parent_gidx[(size_t)b * wsel + i] = gidx_base + idx;
+      pool.qslot[pb + gidx_base + idx] = slot_base + F + i;
+    }
+    return;
+  }
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    if (head_mode == 1 && (i / k_e) % K == 1) continue;
     const float v = sc[i];
     int rank = 0;
-    for (int j = 0; j < n; ++j) rank += jk_better(sc[j], j, v, i) ? 1 : 0;
+    for (int j = 0; j < n; ++j) {
+      if (head_mode == 1 && (j / k_e) % K == 1) continue;
+      rank += jk_better(sc[j], j, v, i) ? 1 : 0;
+    }
     if (rank < wsel) {
       next_frontier[(size_t)b * wsel + rank] = i;
       next_parent_score[(size_t)b * wsel + rank] = v;
@@ -393,29 +444,43 @@ __global__ void __launch_bounds__(1024) k_tree_finalize(
     jk_pool pool, int pool_n, const int32_t* __restrict__ root_tok, int M,
     int32_t* __restrict__ tok, int32_t* __restrict__ parent, int32_t* __restrict__ depth,
     int32_t* __restrict__ branch, int32_t* __restrict__ qslot, unsigned long long* __restrict__ anc,
-    int32_t* status) {
+    const int32_t* __restrict__ static_keep, int32_t* status) {
   jk_pdl_wait();
   jk_pdl_trigger();
   __shared__ float sc[JK_MAX_POOL];
   __shared__ short newid[JK_MAX_POOL];      // 0 = dropped, else node index
   __shared__ int par_s[JK_MAX_TREE];
   __shared__ int scan[1024];
+  __shared__ int keep_s[JK_MAX_TREE];
   const int b = blockIdx.x;
   const size_t pb = (size_t)b * pool.stride_b;
   const int t = threadIdx.x;
   for (int g = t; g < pool_n; g += blockDim.x) sc[g] = pool.score[pb + g];
-  __syncthreads();
   const int m1 = M - 1;
+  if (static_keep && t < m1) {
+    // the predefined shape's list: ascending generation indices inside the pool
+    const int g = static_keep[t];
+    const int prev = t > 0 ? static_keep[t - 1] : -1;
+    if (g < 0 || g >= pool_n || g <= prev) jk_set_status(status, JK_ERR_BOUNDS);
+    keep_s[t] = g;
+  }
+  __syncthreads();
   // each thread owns a contiguous slice so that the prefix sum runs in generation order
   const int per = (pool_n + blockDim.x - 1) / blockDim.x;
   const int g0 = t * per, g1 = min(pool_n, g0 + per);
   int cnt = 0;
   unsigned keepmask = 0;                     // per <= 4 for pool_n <= 4096
   for (int g = g0; g < g1; ++g) {
-    const float v = sc[g];
-    int rank = 0;
-    for (int j = 0; j < pool_n; ++j) rank += jk_better(sc[j], j, v, g) ? 1 : 0;
-    if (rank < m1) { keepmask |= 1u << (g - g0); ++cnt; }
+    bool keep = false;
+    if (static_keep) {
+      for (int j = 0; j < m1; ++j) keep |= keep_s[j] == g;
+    } else {
+      const float v = sc[g];
+      int rank = 0;
+      for (int j = 0; j < pool_n; ++j) rank += jk_better(sc[j], j, v, g) ? 1 : 0;
+      keep = rank < m1;
+    }
+    if (keep) { keepmask |= 1u << (g - g0); ++cnt; }
   }
   scan[t] = cnt;
   __syncthreads();
@@ -477,7 +542,7 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
                        int32_t* out_expert, float* out_gate, const jk_pool* pool, float* out_lse,
                        void* out_feat, float* out_logits, int64_t logits_stride_b,
                        int32_t* next_frontier, float* next_parent_score,
-                       int32_t* next_parent_gidx) {
+                       int32_t* next_parent_gidx, const int32_t* static_select) {
   const jk_config& c = ctx->cfg;
   const jk_ws_layout& L = ctx->lay;
   const int R = B * F, K = c.top_k, RK = R * K, H = c.hidden, I = c.inter, V = c.vocab;
@@ -513,7 +578,8 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
     JK_LAUNCH_CHECK(ctx);
     JK_PROF(ctx, st, JK_ST_BRANCH);
     k_branch<T><<<R, 256, 0, st>>>((const T*)u, ybuf, out_expert, out_gate, K, H, Rp,
-                                   c.branch_residual, bbuf, (T*)out_feat);
+                                   c.branch_residual, c.head_mode, c.contrast_alpha,
+                                   c.contrast_beta, bbuf, (T*)out_feat);
     JK_LAUNCH_CHECK(ctx);
     JK_PROF(ctx, st, JK_ST_LMHEAD);
     k_lmhead<T><<<(V + 31) / 32, 256, 0, st>>>((const T*)w->lm_head, bbuf, RK, H, V, logits,
@@ -526,12 +592,16 @@ static int expand_impl(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, 
     JK_LAUNCH_CHECK(ctx);
   }
   JK_PROF(ctx, st, JK_ST_FINISH);
+  // out_lse follows the per-sequence layout of out_logits: rows slot_base.. of a [B, S, K]
+  // array when the logits go to rows slot_base.. of a [B, S, K, V] one
+  const long long lse_sb = (out_logits && logits_stride_b) ? logits_stride_b / V : rows_per_b;
   jk_launch_pdl(k_expand_finish, dim3(B), dim3(1024), 0, st, F, K, c.k_per_expert, L.topk_chunks, width,
-                                     (const float*)(ws + L.tk_val),
+                                     c.head_mode, (const float*)(ws + L.tk_val),
                                      (const int32_t*)(ws + L.tk_idx),
                                      (const float*)(ws + L.tk_ms), parent_score, parent_gidx,
-                                     gidx_base, slot_base, *pool, out_lse, next_frontier,
-                                     next_parent_score, next_parent_gidx);
+                                     gidx_base, slot_base, *pool, out_lse, rows_per_b, lse_sb,
+                                     next_frontier, next_parent_score, next_parent_gidx,
+                                     static_select, (int32_t*)(ws + L.status));
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
 }
@@ -543,7 +613,8 @@ extern "C" int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights
                                int32_t* out_expert, float* out_gate, const jk_pool* pool,
                                float* out_lse, void* out_feat, float* out_logits,
                                int64_t logits_stride_b, int32_t* next_frontier,
-                               float* next_parent_score, int32_t* next_parent_gidx) {
+                               float* next_parent_score, int32_t* next_parent_gidx,
+                               const int32_t* static_select) {
   if (!ctx || !w || !u || !parent_score || !parent_gidx || !out_expert || !out_gate || !pool ||
       !out_feat)
     return JK_ERR_NULL;
@@ -558,9 +629,10 @@ extern "C" int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights
   const int n_cand = n_frontier * c.top_k * c.k_per_expert;
   if (n_cand > JK_MAX_POOL) return JK_ERR_SHAPE;
   if (pool->stride_b < (int64_t)gidx_base + n_cand) return JK_ERR_SHAPE;
-  if (logits_stride_b < 0 || logits_stride_b % 4 ||
+  if (logits_stride_b < 0 || logits_stride_b % 4 || logits_stride_b % c.vocab ||
       (logits_stride_b && logits_stride_b < (int64_t)n_frontier * c.top_k * c.vocab))
     return JK_ERR_SHAPE;
+  if (static_select && width <= 0) return JK_ERR_SHAPE;
   const void* ptrs[] = {u, w->router, w->w_gate, w->w_up, w->w_down, w->lm_head, w->norm_weight,
                         out_feat, out_logits};
   for (const void* p : ptrs)
@@ -574,17 +646,17 @@ extern "C" int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights
                                       parent_gidx, gidx_base, slot_base, out_probs, out_expert,
                                       out_gate, pool, out_lse, out_feat, out_logits,
                                       logits_stride_b, next_frontier, next_parent_score,
-                                      next_parent_gidx);
+                                      next_parent_gidx, static_select);
   return expand_impl<float>(ctx, st, w, batch, n_frontier, width, u, parent_score, parent_gidx,
                             gidx_base, slot_base, out_probs, out_expert, out_gate, pool, out_lse,
                             out_feat, out_logits, logits_stride_b, next_frontier,
-                            next_parent_score, next_parent_gidx);
+                            next_parent_score, next_parent_gidx, static_select);
 }
 
 extern "C" int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const jk_pool* pool,
                                 int32_t pool_n, const int32_t* root_tok, int32_t tree_size,
                                 int32_t* tok, int32_t* parent, int32_t* depth, int32_t* branch,
-                                int32_t* qslot, uint64_t* anc) {
+                                int32_t* qslot, uint64_t* anc, const int32_t* static_keep) {
   if (!ctx || !pool || !root_tok || !tok || !parent || !depth || !branch || !qslot || !anc)
     return JK_ERR_NULL;
   if (!pool->tok || !pool->score || !pool->parent || !pool->qslot || !pool->branch)
@@ -598,7 +670,7 @@ extern "C" int jk_tree_finalize(jk_ctx* ctx, void* stream, int32_t batch, const 
   JK_PROF(ctx, st, JK_ST_FINALIZE);
   jk_launch_pdl(k_tree_finalize, dim3(batch), dim3(1024), 0, st, 
       *pool, pool_n, root_tok, tree_size, tok, parent, depth, branch, qslot,
-      (unsigned long long*)anc, (int32_t*)(ctx->ws + ctx->lay.status));
+      (unsigned long long*)anc, static_keep, (int32_t*)(ctx->ws + ctx->lay.status));
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
 }

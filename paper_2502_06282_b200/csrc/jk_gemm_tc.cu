@@ -401,8 +401,8 @@ __global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int n_ct
 __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
     const tc_params p, int n_cta, int H, const int32_t* __restrict__ expert,
     const float* __restrict__ gate, const __nv_bfloat16* __restrict__ u, int branch_residual,
-    const float* __restrict__ partial, __nv_bfloat16* __restrict__ bbuf,
-    __nv_bfloat16* __restrict__ out_feat) {
+    int head_mode, float alpha, float beta, const float* __restrict__ partial,
+    __nv_bfloat16* __restrict__ bbuf, __nv_bfloat16* __restrict__ out_feat) {
   jk_pdl_wait();
   jk_pdl_trigger();
   __shared__ tc_plan plan;
@@ -426,11 +426,22 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
   if (h >= H) return;
   const float uv = __bfloat162float(u[(size_t)r * H + h]);
   float f = uv;
-  for (int k = 0; k < K; ++k) {
-    const float y = tc_sum_list(partial, p, lists[k], total, n_cta, tiles[k], r, m);
-    const float gy = gate[r * K + k] * y;
-    f += gy;
-    bbuf[((size_t)r * K + k) * H + h] = __float2bfloat16_rn(branch_residual ? gy + uv : gy);
+  if (head_mode == 1) {
+    // contrastive heads (Eq. 6-7): b_0 = f^moe (+ u), b_1 = beta y_1 - alpha y_2 (+ u)
+    const float y0 = tc_sum_list(partial, p, lists[0], total, n_cta, tiles[0], r, m);
+    const float y1 = tc_sum_list(partial, p, lists[1], total, n_cta, tiles[1], r, m);
+    const float g0y = gate[r * K] * y0, g1y = gate[r * K + 1] * y1;
+    const float fm = g0y + g1y, fc = beta * y0 - alpha * y1;
+    f = (uv + g0y) + g1y;
+    bbuf[((size_t)r * K) * H + h] = __float2bfloat16_rn(branch_residual ? fm + uv : fm);
+    bbuf[((size_t)r * K + 1) * H + h] = __float2bfloat16_rn(branch_residual ? fc + uv : fc);
+  } else {
+    for (int k = 0; k < K; ++k) {
+      const float y = tc_sum_list(partial, p, lists[k], total, n_cta, tiles[k], r, m);
+      const float gy = gate[r * K + k] * y;
+      f += gy;
+      bbuf[((size_t)r * K + k) * H + h] = __float2bfloat16_rn(branch_residual ? gy + uv : gy);
+    }
   }
   out_feat[(size_t)r * H + h] = __float2bfloat16_rn(f);
 }
@@ -686,7 +697,8 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_BRANCH);
   jk_launch_pdl(k_tc_fix_down_branch, dim3(p.tiles_per_group, R), dim3(128), 0, st, 
-      p, n_cta, H, expert, gate, (const __nv_bfloat16*)u, c.branch_residual, partial,
+      p, n_cta, H, expert, gate, (const __nv_bfloat16*)u, c.branch_residual, c.head_mode,
+      c.contrast_alpha, c.contrast_beta, partial,
       (__nv_bfloat16*)(ctx->ws + L.bbuf), (__nv_bfloat16*)out_feat);
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;

@@ -65,14 +65,22 @@ class Workload:
     dtype: str             # "f32" | "bf16"
     n_layers: int          # L target layers verified per step
     seed: int
+    head_mode: int = 0     # 0: decoupled heads (Eq. 4); 1: contrastive heads with the hybrid
+                           # schedule of Sec. 3.2 (depth D from D-1 draft passes)
+
+    @property
+    def n_passes(self) -> int:
+        """jk_draft_expand calls per step."""
+        return self.depth - 1 if self.head_mode == 1 else self.depth
 
     @property
     def frontier_sizes(self) -> List[int]:
-        """F_1..F_D: the root alone, then at most W nodes per layer."""
+        """F_1.. of the draft passes: the root alone, then at most W nodes per pass (in the
+        contrastive mode only a node's row-0 children can be expanded)."""
+        per_node = self.k_per_expert * (1 if self.head_mode == 1 else self.top_k)
         out = [1]
-        for _ in range(1, self.depth):
-            prev_cands = out[-1] * self.top_k * self.k_per_expert
-            out.append(min(self.width, prev_cands))
+        for _ in range(1, self.n_passes):
+            out.append(min(self.width, out[-1] * per_node))
         return out
 
     @property

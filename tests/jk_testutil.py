@@ -88,10 +88,11 @@ def guarded_context(w, **kw):
     return ctx, check
 
 
-def guarded_step_buffers(ctx, w, guard: Guard):
+def guarded_step_buffers(ctx, w, guard: Guard, bufs=None):
     """StepBuffers whose every tensor is a guarded, poisoned allocation."""
     from paper_2502_06282_b200 import binding as jk
-    bufs = jk.StepBuffers(ctx, w)
+    if bufs is None:
+        bufs = jk.StepBuffers(ctx, w)
     for k in bufs.pool:
         bufs.pool[k] = guard.like(bufs.pool[k])
     bufs.pool_struct = ctx.pool_struct(bufs.pool)

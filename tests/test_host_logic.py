@@ -44,6 +44,15 @@ def test_create_and_workspace_size(lib):
     ctx.close()
 
 
+def test_contrastive_mode_needs_two_active_experts(lib):
+    with pytest.raises(jk.JakiroError) as e:
+        jk.Context(**_cfg(head_mode=1, top_k=3))
+    assert e.value.code == jk.ERR["SHAPE"]
+    with pytest.raises(jk.JakiroError):
+        jk.Context(**_cfg(head_mode=2))
+    jk.Context(**_cfg(head_mode=1, contrast_alpha=0.5, contrast_beta=1.5)).close()
+
+
 @pytest.mark.parametrize("bad", [dict(hidden=510), dict(inter=1377), dict(n_experts=9),
                                  dict(top_k=5), dict(k_per_expert=17), dict(max_tree=129),
                                  dict(max_batch=64, max_frontier=4), dict(head_dim=96),
@@ -104,10 +113,10 @@ def test_expand_and_finalize_argument_checks(lib):
     w = jk.JkDraftWeights(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, None)
     pool = jk.JkPool(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 52)
 
-    def expand(batch=1, F=1, width=4, gidx=0, wts=w, p=pool, stride=0):
+    def expand(batch=1, F=1, width=4, gidx=0, wts=w, p=pool, stride=0, static=None):
         return lib.jk_draft_expand(h, None, C.byref(wts), batch, F, width, fake, fake, fake, gidx,
                                    0, None, fake, fake, C.byref(p), None, fake, None, stride,
-                                   fake, fake, fake)
+                                   fake, fake, fake, static)
     assert expand() == jk.ERR["WORKSPACE"]          # everything else is fine
     assert expand(batch=2) == jk.ERR["CAPACITY"]
     assert expand(F=5) == jk.ERR["CAPACITY"]
@@ -117,12 +126,46 @@ def test_expand_and_finalize_argument_checks(lib):
     assert expand(wts=jk.JkDraftWeights(0x1008, 0x1000, 0x1000, 0x1000, 0x1000, None)) \
         == jk.ERR["ALIGN"]
     assert expand(stride=6) == jk.ERR["SHAPE"]
+    assert expand(width=0, static=fake) == jk.ERR["SHAPE"]   # a static list selects nothing on the last pass
 
     def finalize(pool_n=52, M=16, batch=1):
         return lib.jk_tree_finalize(h, None, batch, C.byref(pool), pool_n, fake, M, fake, fake,
-                                    fake, fake, fake, fake)
+                                    fake, fake, fake, fake, None)
     assert finalize() == jk.ERR["WORKSPACE"]
     assert finalize(pool_n=10) == jk.ERR["SHAPE"]    # fewer candidates than tree nodes
     assert finalize(pool_n=60) == jk.ERR["SHAPE"]    # more than the pool's stride
     assert finalize(M=17) == jk.ERR["CAPACITY"]
     ctx.close()
+
+
+def test_static_tree_plan_matches_the_oracles_node_order():
+    """plan_from_paths (product-side index bookkeeping) against the oracle's own ordering of a
+    predefined tree: same node order, parents, depths and branches."""
+    import numpy as np
+    from oracle import jakiro_oracle as orc
+    from paper_2502_06282_b200.static_tree import plan_from_paths
+    paths = [(0,), (1,), (3,), (0, 0), (0, 2), (3, 1), (0, 0, 3), (0, 0, 0), (3, 1, 1), (3, 1, 2)]
+    K, ke = 2, 2
+    plan = plan_from_paths(paths, K, ke)
+    rng = np.random.default_rng(0)
+    w = {"router": rng.standard_normal((4, 8)), "w_gate": rng.standard_normal((4, 6, 8)),
+         "w_up": rng.standard_normal((4, 6, 8)), "w_down": rng.standard_normal((4, 8, 6)),
+         "lm_head": rng.standard_normal((11, 8)), "norm_weight": np.ones(8)}
+    t = orc.grow_static_tree(lambda p: rng.standard_normal(8), w, paths, ke, root_tok=1)
+    assert plan["order"] == t["order"][1:]
+    assert plan["frontier_sizes"] == [1, 2, 2]
+    assert plan["keep"] == sorted(plan["keep"]) and len(plan["keep"]) == len(paths)
+    # generation index -> (pass, frontier row, candidate): the parent of a kept node is the
+    # node that sits at that frontier row of the pass
+    bases = np.cumsum([0] + [F * K * ke for F in plan["frontier_sizes"]])
+    frontier = [[()]]
+    for sel, base in zip(plan["select"], bases[:-1]):
+        frontier.append([plan["order"][plan["keep"].index(base + s)] for s in sel])
+    for p, g in zip(plan["order"], plan["keep"]):
+        l = int(np.searchsorted(bases, g, side="right") - 1)
+        f, c = divmod(int(g - bases[l]), K * ke)
+        assert frontier[l][f] == p[:-1] and c == p[-1]
+    with pytest.raises(ValueError):
+        plan_from_paths([(0,), (1, 0)], K, ke)
+    with pytest.raises(ValueError):
+        plan_from_paths([(4,)], K, ke)
