@@ -4,6 +4,8 @@
  * One speculative-decoding step of arXiv 2502.06282 has three phases (Sec. 2.1): draft,
  * verify, refine.  This library provides the per-step kernels of each phase:
  *
+ *   jk_draft_pre           the draft layer in front of the MoE: reduction layer and attention
+ *                          (Sec. 3.1.2, Eq. 1)
  *   jk_draft_expand        one layer of the decoupled MoE draft head (Sec. 3.1.2, Eq. 2-5)
  *   jk_tree_finalize       rerank the drafted candidates into the verification tree and
  *                          build its attention mask (Sec. 3.1.2, Fig. 4)
@@ -162,7 +164,9 @@ typedef struct {
  *   out_gate     f32 [B, F, K]
  *   pool         children appended as described at jk_pool; qslot is set for the children
  *                chosen as next frontier (slot_base + F + position), -1 for the others
- *   out_lse      f32 [B, F, K]   logsumexp of each logits row (opt)
+ *   out_lse      f32 [B, F, K]   logsumexp of each logits row (opt); laid out like out_logits:
+ *                with logits_stride_b given, sequences are logits_stride_b / V elements apart,
+ *                so that a call writes rows slot_base.. of a [B, S, K] array
  *   out_feat     T   [B, F, H]   combined feature f (Eq. 3)
  *   out_logits   f32 [B, F, K, V] (opt; needed later for sampling acceptance), with
  *                logits_stride_b elements between sequences (0 = dense, F*K*V), so that a call
@@ -194,6 +198,61 @@ int jk_draft_expand(jk_ctx* ctx, void* stream, const jk_draft_weights* host_w,
                     const jk_pool* host_pool, float* out_lse, void* out_feat, float* out_logits,
                     int64_t logits_stride_b, int32_t* next_frontier, float* next_parent_score,
                     int32_t* next_parent_gidx, const int32_t* static_select);
+
+/* Weights of the draft layer in front of the MoE (Sec. 3.1.1, 3.1.2): device pointers, read-only,
+ * output-major. */
+typedef struct {
+  const void* emb;          /* T [V, H]      token embedding, shared with the target model      */
+  const void* w_fc;         /* T [H, 2H]     reduction layer, acts on [emb(tok) ; parent feature] */
+  const void* b_fc;         /* T [H] or NULL                                                     */
+  const void* w_qkv;        /* T [(Hq + 2 Hkv) d, H]  rows of W_q, then W_k, then W_v           */
+  const void* w_o;          /* T [H, Hq d]                                                       */
+} jk_pre_weights;
+
+/* State of the draft layer's attention over one step, caller-owned device memory: one entry per
+ * expanded node ("slot": root = 0, then the frontier nodes of every pass in order), S_max =
+ * stride_b slots per sequence. */
+typedef struct {
+  void* q;                  /* T   [B, S_max, Hq, d]  rotated query of every expanded node        */
+  int32_t* slot_parent;     /* i32 [B, S_max]         parent slot, -1 for the root                */
+  int32_t* slot_depth;      /* i32 [B, S_max]                                                     */
+  int64_t stride_b;         /* S_max                                                              */
+} jk_pre_state;
+
+/*
+ * The draft layer before the MoE for the F frontier nodes of one pass (Sec. 3.1.2, Eq. 1 and the
+ * paragraph before it):
+ *   h = W_fc [emb(tok) ; f_prev] (+ b_fc), with f_prev the feature f (Eq. 3, out_feat of
+ *   jk_draft_expand) of the node's parent - for the root the target model's last feature;
+ *   q, k, v = W_qkv h, q and k rotated (rotary positions, LLaMA pairing (i, i + d/2), base
+ *   rope_theta) to position kv_len[b] + depth; k and v are appended to the draft layer's own
+ *   cache at row kv_len[b] + slot; every node attends over rows 0 .. kv_len[b]-1 and the rows of
+ *   itself and its ancestors; u = W_o Attn + h (Eq. 1).
+ * No normalisation is applied in this block (Eq. 1-5 leave the norms out; Eagle-style drafts drop
+ * the input norm of their single layer).  out_u feeds jk_draft_expand of the same pass.
+ *   slot_base    slot of this pass's first node (0 for the root pass, then the running count)
+ *   node_gidx    i32 [B, F] generation index of each node = next_parent_gidx of the previous
+ *                jk_draft_expand; NULL in the root pass (then F = 1, the token is root_tok[b]
+ *                and prev_feat is T [B, H])
+ *   pool         the step's candidate pool: the nodes' tokens are pool.tok[node_gidx]
+ *   prev_gidx_base, prev_slot_base, prev_frontier   gidx_base, slot_base and F of the previous
+ *                pass; prev_feat T [B, prev_frontier, H] its out_feat.  A node's parent is
+ *                frontier row (node_gidx - prev_gidx_base) / (K k_e) of that pass.
+ *   k_cache, v_cache  T [B, Hkv, cap, d] with strides as in jk_tree_verify_attn; rows
+ *                kv_len[b] .. kv_len[b] + slot_base + F - 1 are written over the passes
+ *   out_u        T [B, F, H]
+ * The attention runs over all slot_base + F nodes expanded so far (their queries are kept in
+ * state.q), so slot_base + F <= 128 and <= max_depth * max_frontier.
+ * Errors: NULL/ALIGN/SHAPE/CAPACITY/WORKSPACE/CUDA; a token or index out of range, or a cache too
+ * short, sets JK_ERR_BOUNDS in the status word.
+ */
+int jk_draft_pre(jk_ctx* ctx, void* stream, const jk_pre_weights* host_w,
+                 const jk_pre_state* host_state, int32_t batch, int32_t n_frontier,
+                 int32_t slot_base, const int32_t* node_gidx, const jk_pool* host_pool,
+                 int32_t prev_gidx_base, int32_t prev_slot_base, int32_t prev_frontier,
+                 const void* prev_feat, const int32_t* root_tok, void* k_cache, void* v_cache,
+                 int64_t cache_stride_b, int64_t cache_stride_h, int32_t cache_rows,
+                 const int32_t* kv_len, float rope_theta, float softmax_scale, void* out_u);
 
 /*
  * Build the verification tree from the pool (Sec. 3.1.2; mask as in Fig. 4): node 0 is the

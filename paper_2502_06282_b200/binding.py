@@ -26,7 +26,7 @@ EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", 
            "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
            "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
            "jk_profile_stage_name", "jk_tree_verify_attn_static", "jk_tensor_path_active",
-           "jk_set_attn_kernel", "jk_profile_read"]
+           "jk_set_attn_kernel", "jk_profile_read", "jk_draft_pre"]
 
 
 class JkConfig(C.Structure):
@@ -45,6 +45,15 @@ class JkDraftWeights(C.Structure):
 class JkPool(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("tok", "score", "parent", "qslot", "branch")] + [
         ("stride_b", C.c_int64)]
+
+
+class JkPreWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("emb", "w_fc", "b_fc", "w_qkv", "w_o")]
+
+
+class JkPreState(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("slot_parent", C.c_void_p), ("slot_depth", C.c_void_p),
+                ("stride_b", C.c_int64)]
 
 
 _lib = None
@@ -84,6 +93,9 @@ def lib() -> C.CDLL:
         L.jk_accept_and_compact.argtypes = [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, vp, vp,
                                             vp, vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp,
                                             vp, vp, vp, vp]
+        L.jk_draft_pre.argtypes = [vp, vp, C.POINTER(JkPreWeights), C.POINTER(JkPreState), i32, i32,
+                                   i32, vp, C.POINTER(JkPool), i32, i32, i32, vp, vp, vp, vp, i64,
+                                   i64, i32, vp, f32, f32, vp]
         L.jk_profile_enable.argtypes = [vp, i32]
         L.jk_profile_collect.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
         L.jk_profile_read.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
@@ -240,6 +252,24 @@ class Context:
             _ptr(next_parent_gidx), _ptr(static_select))
         self._check(rc, "jk_draft_expand")
 
+    @staticmethod
+    def pre_weights_struct(w: Dict[str, torch.Tensor]) -> JkPreWeights:
+        return JkPreWeights(_ptr(w["emb"]), _ptr(w["w_fc"]), _ptr(w.get("b_fc")), _ptr(w["w_qkv"]),
+                            _ptr(w["w_o"]))
+
+    def draft_pre(self, pre_weights, state: JkPreState, batch, n_frontier, slot_base, node_gidx,
+                  pool, prev_gidx_base, prev_slot_base, prev_frontier, prev_feat, root_tok, k_cache,
+                  v_cache, kv_len, rope_theta, scale, out_u, cache_rows=None):
+        ws = pre_weights if isinstance(pre_weights, JkPreWeights) else self.pre_weights_struct(pre_weights)
+        ps = pool if isinstance(pool, JkPool) else self.pool_struct(pool)
+        rows = k_cache.shape[2] if cache_rows is None else cache_rows
+        rc = lib().jk_draft_pre(self._h, _stream(), C.byref(ws), C.byref(state), batch, n_frontier,
+                                slot_base, _ptr(node_gidx), C.byref(ps), prev_gidx_base,
+                                prev_slot_base, prev_frontier, _ptr(prev_feat), _ptr(root_tok),
+                                _ptr(k_cache), _ptr(v_cache), k_cache.stride(0), k_cache.stride(1),
+                                rows, _ptr(kv_len), float(rope_theta), float(scale), _ptr(out_u))
+        self._check(rc, "jk_draft_pre")
+
     def tree_finalize(self, batch, pool, pool_n, root_tok, tree_size, tok, parent, depth, branch,
                       qslot, anc, static_keep=None):
         ps = pool if isinstance(pool, JkPool) else self.pool_struct(pool)
@@ -313,7 +343,10 @@ class StepBuffers:
         self.probs = [torch.empty(B, F, w.n_experts, **f32) for F in fs]
         self.expert = [torch.empty(B, F, K, **i32) for F in fs]
         self.gate = [torch.empty(B, F, K, **f32) for F in fs]
-        self.lse = [torch.empty(B, F, K, **f32) for F in fs]
+        # log-sum-exp of every stored logits row: [B, S, K], laid out like the logits (a call
+        # writes rows slot_base.. of every sequence); dense per-pass arrays when no logits are kept
+        self.lse_all = torch.empty(B, self.n_slots, K, **f32) if keep_logits else None
+        self.lse = self.lse_views() if keep_logits else [torch.empty(B, F, K, **f32) for F in fs]
         self.feat = [torch.empty(B, F, H, dtype=ctx.tdtype, device=device) for F in fs]
         self.logits = torch.empty(B, self.n_slots, K, V, **f32) if keep_logits else None
         nxt = fs[1:] + [1]                      # nodes chosen by pass l = nodes expanded by pass l+1
@@ -328,6 +361,17 @@ class StepBuffers:
         self.acc_idx = torch.empty(B, w.depth, **i32)
         self.acc_tok = torch.empty(B, w.depth, **i32)
         self.bonus = torch.empty(B, **i32)
+
+
+def _lse_views(self):
+    out, s0 = [], 0
+    for F in self.frontier_sizes:
+        out.append(self.lse_all[:, s0:s0 + F])
+        s0 += F
+    return out
+
+
+StepBuffers.lse_views = _lse_views
 
 
 def run_draft(ctx: Context, bufs: StepBuffers, weights, u_layers: Sequence[torch.Tensor],
@@ -362,3 +406,51 @@ def run_draft(ctx: Context, bufs: StepBuffers, weights, u_layers: Sequence[torch
                           bufs.tree["tok"], bufs.tree["parent"], bufs.tree["depth"],
                           bufs.tree["branch"], bufs.tree["qslot"], bufs.anc,
                           None if static_plan is None else static_plan["keep"])
+
+
+class PreBuffers:
+    """Device state of the draft layer's pre-MoE block for one step: the rotated queries and the
+    partial tree (parent slot, depth) of every expanded node, and the hidden states u per pass."""
+
+    def __init__(self, ctx: Context, bufs: StepBuffers, device="cuda"):
+        w = bufs.w
+        S = bufs.n_slots
+        self.q = torch.empty(w.batch, S, w.n_q_heads, w.head_dim, dtype=ctx.tdtype, device=device)
+        self.slot_parent = torch.empty(w.batch, S, dtype=torch.int32, device=device)
+        self.slot_depth = torch.empty(w.batch, S, dtype=torch.int32, device=device)
+        self.state = JkPreState(_ptr(self.q), _ptr(self.slot_parent), _ptr(self.slot_depth), S)
+        self.u = [torch.empty(w.batch, F, w.hidden, dtype=ctx.tdtype, device=device)
+                  for F in bufs.frontier_sizes]
+
+
+def run_draft_chained(ctx: Context, bufs: StepBuffers, pre: PreBuffers, weights, pre_weights,
+                      root_tok: torch.Tensor, root_feat: torch.Tensor, k_cache, v_cache, kv_len,
+                      rope_theta: float, scale: float, finalize: bool = True):
+    """The whole draft of one step with nothing synthetic in between: per pass jk_draft_pre turns
+    the frontier's tokens and their parents' features into u (Eq. 1), jk_draft_expand grows the
+    tree from u (Eq. 2-5) and hands back the features the next pass starts from."""
+    w = bufs.w
+    fs = bufs.frontier_sizes
+    B, K, ke = w.batch, w.top_k, w.k_per_expert
+    gidx_base = slot_base = 0
+    prev = (0, 0, 1)                       # gidx_base, slot_base, F of the previous pass
+    for l, F in enumerate(fs):
+        last = l == len(fs) - 1
+        ctx.draft_pre(pre_weights, pre.state, B, F, slot_base,
+                      None if l == 0 else bufs.parent_gidx[l], bufs.pool_struct, prev[0], prev[1],
+                      prev[2], root_feat if l == 0 else bufs.feat[l - 1], root_tok, k_cache,
+                      v_cache, kv_len, rope_theta, scale, pre.u[l])
+        out_logits = None if bufs.logits is None else bufs.logits[:, slot_base:slot_base + F]
+        ctx.draft_expand(weights, B, F, 0 if last else fs[l + 1], pre.u[l], bufs.parent_score[l],
+                         bufs.parent_gidx[l], gidx_base, slot_base, bufs.probs[l], bufs.expert[l],
+                         bufs.gate[l], bufs.pool_struct, bufs.lse[l], bufs.feat[l], out_logits,
+                         None if last else bufs.frontier[l],
+                         None if last else bufs.parent_score[l + 1],
+                         None if last else bufs.parent_gidx[l + 1])
+        prev = (gidx_base, slot_base, F)
+        gidx_base += F * K * ke
+        slot_base += F
+    if finalize:
+        ctx.tree_finalize(B, bufs.pool_struct, bufs.pool_n, root_tok, w.tree_size,
+                          bufs.tree["tok"], bufs.tree["parent"], bufs.tree["depth"],
+                          bufs.tree["branch"], bufs.tree["qslot"], bufs.anc)

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libjakiro.so")
 SOURCES = ["jk_api.cu", "jk_expand.cu", "jk_gemm_tc.cu", "jk_attn.cu", "jk_attn_tc.cu", "jk_attn_sk.cu", "jk_attn_cl.cu",
-           "jk_accept.cu"]
+           "jk_accept.cu", "jk_pre.cu"]
 
 
 def _nvcc() -> str:

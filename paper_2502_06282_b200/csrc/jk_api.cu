@@ -60,7 +60,8 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->gemm_part_bytes = c.dtype == JK_BF16 ? jk_tc_partial_bytes(c) : 0;
   L->gemm_part = take(L->gemm_part_bytes);
   // split-KV partials, capped at 256 MiB
-  const size_t rows = BM * c.n_q_heads;
+  const size_t pre_nodes = (size_t)c.max_batch * c.max_depth * c.max_frontier;
+  const size_t rows = (BM > pre_nodes ? BM : pre_nodes) * c.n_q_heads;
   const size_t per_split = rows * (c.head_dim + 2) * 4;
   int ms = JK_ATTN_MAX_SPLIT;
   while (ms > 1 && per_split * ms > ((size_t)256 << 20)) --ms;
@@ -77,6 +78,16 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->qs_arg = take(qrows * 4);
   L->qs_max = take(qrows * 4);
   L->qs_sum = take(qrows * 4);
+  const size_t S = (size_t)c.max_depth * c.max_frontier;
+  const size_t qd = (size_t)c.n_q_heads * c.head_dim;
+  const size_t qkvd = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  L->pre_x = take(Rp * 2 * c.hidden * es);
+  L->pre_h = take(Rp * c.hidden * es);
+  L->pre_qkv = take(Rp * qkvd * 4);
+  L->pre_qd = take((size_t)c.max_batch * S * qd * es);
+  L->pre_par = take((size_t)c.max_batch * S * 4);
+  L->pre_att = take((size_t)c.max_batch * S * qd * es);
+  L->pre_ao = take(Rp * qd * es);
   L->total = off;
 }
 
@@ -89,6 +100,8 @@ extern "C" int jk_create(jk_ctx** out, const jk_config* cfg) {
   ctx->cfg = *cfg;
   build_layout(ctx->cfg, &ctx->lay);
   ctx->tensor_path = cfg->dtype == JK_BF16 ? 1 : 0;
+  ctx->st_attn = JK_ST_ATTN;
+  ctx->st_combine = JK_ST_ATTN_COMBINE;
   *out = ctx;
   return JK_OK;
 }
@@ -235,7 +248,8 @@ extern "C" const char* jk_profile_stage_name(int32_t stage) {
   static const char* names[JK_N_STAGES] = {
       "router", "expert_gate_up", "expert_down", "branch_features", "lm_head", "topk_partial",
       "expand_finish", "tree_finalize", "tree_attn", "attn_combine", "row_stats", "accept_walk",
-      "kv_compact", "gemm_fixup"};
+      "kv_compact", "gemm_fixup", "pre_gather", "pre_gemm", "pre_fixup", "pre_rope", "pre_attn",
+      "pre_attn_combine"};
   return (stage >= 0 && stage < JK_N_STAGES) ? names[stage] : "?";
 }
 

@@ -226,14 +226,14 @@ static int attn_impl(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, 
   }
   float* part_o = (float*)(ctx->ws + L.attn_o);
   float* part_ml = (float*)(ctx->ws + L.attn_ml);
-  JK_PROF(ctx, st, JK_ST_ATTN);
+  JK_PROF(ctx, st, ctx->st_attn);
   kern<<<dim3(n_split * n_qblk, c.n_kv_heads, B), 256, smem, st>>>(
       (const T*)q, (const T*)kc, (const T*)vc, sb, sh, cache_rows, kv_len, parent, scale, M,
       c.n_q_heads, c.n_kv_heads, n_split, n_qblk, part_o, part_ml,
       (int32_t*)(ctx->ws + L.status));
   JK_LAUNCH_CHECK(ctx);
   const size_t n_out = (size_t)B * M * c.n_q_heads;
-  JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
+  JK_PROF(ctx, st, ctx->st_combine);
   k_attn_combine<T, D><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
                                                                     n_out, (T*)out);
   JK_LAUNCH_CHECK(ctx);
@@ -251,7 +251,7 @@ int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_o
   const jk_ws_layout& L = ctx->lay;
   const float* part_o = (const float*)(ctx->ws + L.attn_o);
   const float* part_ml = (const float*)(ctx->ws + L.attn_ml);
-  JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
+  JK_PROF(ctx, st, ctx->st_combine);
   const dim3 grid((unsigned)((n_out + 7) / 8));
   if (ctx->cfg.head_dim == 128)
     jk_launch_pdl(k_attn_combine<__nv_bfloat16, 128>, grid, dim3(256), 0, st, part_o, part_ml,
@@ -262,6 +262,11 @@ int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_o
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
 }
+
+int jk_attn_dispatch(jk_ctx* ctx, cudaStream_t st, int batch, int tree_size, const void* q,
+                     const void* k_cache, const void* v_cache, int64_t cache_stride_b,
+                     int64_t cache_stride_h, int cache_rows, const int32_t* kv_len,
+                     const int32_t* parent, float softmax_scale, void* out);
 
 extern "C" int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
                                    const void* q, const void* k_cache, const void* v_cache,
@@ -280,7 +285,18 @@ extern "C" int jk_tree_verify_attn(jk_ctx* ctx, void* stream, int32_t batch, int
   if (!ctx->ws) return JK_ERR_WORKSPACE;
   int rc = jk_ensure_device_info(ctx);
   if (rc != JK_OK) return rc;
-  cudaStream_t st = (cudaStream_t)stream;
+  return jk_attn_dispatch(ctx, (cudaStream_t)stream, batch, tree_size, q, k_cache, v_cache,
+                          cache_stride_b, cache_stride_h, cache_rows, kv_len, parent,
+                          softmax_scale, out);
+}
+
+// The kernel choice behind jk_tree_verify_attn (arguments already validated); jk_draft_pre runs
+// the draft layer's own attention through it.
+int jk_attn_dispatch(jk_ctx* ctx, cudaStream_t st, int batch, int tree_size, const void* q,
+                     const void* k_cache, const void* v_cache, int64_t cache_stride_b,
+                     int64_t cache_stride_h, int cache_rows, const int32_t* kv_len,
+                     const int32_t* parent, float softmax_scale, void* out) {
+  const jk_config& c = ctx->cfg;
   if (c.dtype == JK_BF16 && ctx->tensor_path && softmax_scale > 0.f && jk_tc_available(ctx))
     return jk_attn_tc(ctx, st, batch, tree_size, q, k_cache, v_cache, cache_stride_b,
                       cache_stride_h, cache_rows, kv_len, parent, softmax_scale, out);

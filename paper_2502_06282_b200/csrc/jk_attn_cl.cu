@@ -606,7 +606,7 @@ int jk_attn_cl(jk_ctx* ctx, cudaStream_t st, int n_split, int B, int M, const vo
   const int D = c.head_dim;
   const dim3 grid(n_split * n_qblk, c.n_kv_heads, B);
   int32_t* status = (int32_t*)(ctx->ws + ctx->lay.status);
-  JK_PROF(ctx, st, JK_ST_ATTN);
+  JK_PROF(ctx, st, ctx->st_attn);
   if (D == 128)
     acl_launch<128>(grid, n_split, acl_smem_bytes(D), st, mk, mv, q, kv_len, parent, scale, M,
                     c.n_q_heads, c.n_kv_heads, cache_rows, out, status);

@@ -639,7 +639,7 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   const int n_cta = ctx->sm_count;
   const int ms = L.attn_max_split;
   const int min_units = 1;
-  JK_PROF(ctx, st, JK_ST_ATTN);
+  JK_PROF(ctx, st, ctx->st_attn);
   if (D == 128)
     jk_launch_pdl(k_tree_attn_sk<128>, dim3(n_cta), dim3(ASK_THREADS), smem, st, mk, mv,
                   (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
@@ -650,7 +650,7 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                   ms, min_units, cache_rows, part_o, part_ml, status);
   JK_LAUNCH_CHECK(ctx);
   const size_t n_out = (size_t)B * M * c.n_q_heads;
-  JK_PROF(ctx, st, JK_ST_ATTN_COMBINE);
+  JK_PROF(ctx, st, ctx->st_combine);
   if (D == 128)
     jk_launch_pdl(k_attn_combine_sk<128>, dim3((unsigned)((n_out + 7) / 8)), dim3(256), 0, st,
                   (const float*)part_o, (const float*)part_ml, kv_len, B, M, c.n_q_heads,

@@ -477,7 +477,7 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
     s->smem_set = 1;
   }
-  JK_PROF(ctx, st, JK_ST_ATTN);
+  JK_PROF(ctx, st, ctx->st_attn);
   if (D == 128)
     jk_launch_pdl(k_tree_attn_tc<128>, dim3(grid), dim3(ATC_THREADS), smem, st, mk, mv, (const __nv_bfloat16*)q, kv_len, parent,
                                                  scale, M, c.n_q_heads, c.n_kv_heads, n_split,

@@ -43,6 +43,14 @@ struct jk_ws_layout {
   size_t qs_arg;        // i32 [B, S, K]     top-1 of every stored draft row (written, not read)
   size_t qs_max;        // f32 [B, S, K]     max of every stored draft logits row
   size_t qs_sum;        // f32 [B, S, K]     its sum of exp((x - max)/T)
+  // draft pre-MoE block (Eq. 1); S = max_depth * max_frontier slots per sequence
+  size_t pre_x;         // T   [Rp, 2H]      [emb(tok) ; parent feature]
+  size_t pre_h;         // T   [Rp, H]       reduction layer output h
+  size_t pre_qkv;       // f32 [Rp, (Hq + 2 Hkv) d]
+  size_t pre_qd;        // T   [B * S, Hq d] rotated queries of the nodes expanded so far, dense
+  size_t pre_par;       // i32 [B * S]       their parent slots, dense
+  size_t pre_att;       // T   [B * S, Hq d] attention outputs of those nodes
+  size_t pre_ao;        // T   [Rp, Hq d]    attention outputs of this pass's nodes (O-proj input)
   size_t total;
   int attn_max_split;
   int topk_chunks;
@@ -55,7 +63,8 @@ struct jk_ws_layout {
 enum jk_stage {
   JK_ST_ROUTER = 0, JK_ST_GATEUP, JK_ST_DOWN, JK_ST_BRANCH, JK_ST_LMHEAD, JK_ST_TOPK,
   JK_ST_FINISH, JK_ST_FINALIZE, JK_ST_ATTN, JK_ST_ATTN_COMBINE, JK_ST_ROWSTATS, JK_ST_WALK,
-  JK_ST_COMPACT, JK_ST_GEMM_FIXUP, JK_N_STAGES
+  JK_ST_COMPACT, JK_ST_GEMM_FIXUP, JK_ST_PRE_GATHER, JK_ST_PRE_GEMM, JK_ST_PRE_FIXUP,
+  JK_ST_PRE_ROPE, JK_ST_PRE_ATTN, JK_ST_PRE_ATTN_COMBINE, JK_N_STAGES
 };
 struct jk_prof {
   cudaEvent_t* ev;        // 2 * cap events
@@ -73,6 +82,7 @@ struct jk_ctx {
   int sm_count;           // filled at the first launch
   int attn_smem_set;
   int attn_sk_smem_set;
+  int st_attn, st_combine;  // profiling stages the attention kernels are booked under
   int attn_kernel;        // 0 = by size, 1 = CTA per (query block, key slice), 2 = persistent,
                           // 3 = cluster-merged
   char cuda_err[256];

@@ -540,8 +540,18 @@ size_t jk_tc_partial_bytes(const jk_config& c) {
   size_t a = tc_partial_for(2ll * c.n_experts * t_i * kt_h, kt_h, np1);
   size_t b = tc_partial_for((long long)c.n_experts * t_h * kt_i, kt_i, np1);
   size_t d = tc_partial_for(t_v * kt_h, kt_h, np2);
+  // the draft layer's reduction, QKV and output projections (one group each)
+  const int qd = c.n_q_heads * c.head_dim, qkvd = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  const int kt_2h = (2 * c.hidden + TC_TILE_K - 1) / TC_TILE_K, kt_q = (qd + TC_TILE_K - 1) / TC_TILE_K;
+  const long long t_qkv = (qkvd + TC_TILE_M - 1) / TC_TILE_M;
+  size_t e1 = tc_partial_for(t_h * kt_2h, kt_2h, np1);
+  size_t e2 = tc_partial_for(t_qkv * kt_h, kt_h, np1);
+  size_t e3 = tc_partial_for(t_h * kt_q, kt_q, np1);
   size_t m = a > b ? a : b;
-  return m > d ? m : d;
+  m = m > d ? m : d;
+  m = m > e1 ? m : e1;
+  m = m > e2 ? m : e2;
+  return m > e3 ? m : e3;
 }
 
 void jk_tc_destroy(jk_ctx* ctx) {
@@ -735,6 +745,65 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
       p, n_cta, V, c.k_per_expert, L.topk_chunks, (const float*)(ctx->ws + L.gemm_part), logits,
       rows_per_b, logits_stride_b, (float*)(ctx->ws + L.tk_val), (int32_t*)(ctx->ws + L.tk_idx),
       (float*)(ctx->ws + L.tk_ms));
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Plain linear layer on the same streaming GEMM: out[r, m] = sum_k W[m, k] x[r, k] (+ bias[m])
+// (+ resid[r, m]), used by the draft layer's reduction, QKV and output projections (Eq. 1).
+// ---------------------------------------------------------------------------------------------
+// grid (tiles over the M output features, rows); one of out_bf16 / out_f32 is written
+__global__ void __launch_bounds__(128) k_tc_fix_linear(
+    const tc_params p, int n_cta, int Mrows, const float* __restrict__ partial,
+    const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ resid,
+    long long resid_ld, __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32,
+    long long out_ld) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  __shared__ tc_slot_list list;
+  const int t = blockIdx.x, r = blockIdx.y, m = threadIdx.x;
+  const long long total = (long long)p.tiles_per_group * p.kt;     // one group, always active
+  if (threadIdx.x == 0) list.n = tc_tile_slots(p, total, n_cta, t, list.slot);
+  __syncthreads();
+  const int o = t * TC_TILE_M + m;
+  if (o >= Mrows) return;
+  float v = tc_sum_list(partial, p, list, total, n_cta, t, r, m);
+  if (bias) v += __bfloat162float(bias[o]);
+  if (resid) v += __bfloat162float(resid[(size_t)r * resid_ld + o]);
+  if (out_bf16) out_bf16[(size_t)r * out_ld + o] = __float2bfloat16_rn(v);
+  else out_f32[(size_t)r * out_ld + o] = v;
+}
+
+// x: bf16 [x_rows, Kdim] (x_rows >= n_rows rounded up to 16: the workspace sections are), W: bf16
+// [Mrows, Kdim].  The weights do not depend on the kernel before: their first ring is prefetched.
+int jk_tc_linear(jk_ctx* ctx, cudaStream_t st, const void* W, int Mrows, int Kdim, const void* x,
+                 int x_rows, int n_rows, const void* bias, const void* resid, long long resid_ld,
+                 void* out_bf16, float* out_f32, long long out_ld) {
+  tc_state* s = tc_get_state(ctx);
+  if (!s || s->failed) return JK_ERR_CUDA;
+  const jk_ws_layout& L = ctx->lay;
+  tc_params p;
+  memset(&p, 0, sizeof(p));
+  p.R = 0; p.K_top = ctx->cfg.top_k; p.n_experts = ctx->cfg.n_experts;
+  const int n_pad = (int)jk_align_up(n_rows, 16);
+  if (n_pad > x_rows || n_pad > 256) return JK_ERR_SHAPE;
+  CUtensorMap aw, bx;
+  if (!tc_map(ctx, s, W, Mrows, Kdim, TC_TILE_M, &aw) || !tc_map(ctx, s, x, x_rows, Kdim, n_pad, &bx))
+    return JK_ERR_CUDA;
+  p.n_groups_max = 1;
+  p.group_expert[0] = -1; p.group_amap[0] = 0; p.group_arow0[0] = 0; p.group_brow0[0] = 0;
+  p.tiles_per_group = (Mrows + TC_TILE_M - 1) / TC_TILE_M;
+  p.kt = (Kdim + TC_TILE_K - 1) / TC_TILE_K;
+  p.n_pad = n_pad;
+  p.prefetch = 1;
+  int n_cta = 0;
+  int rc = tc_launch_gemm(ctx, st, s, &aw, &aw, &bx, p, nullptr, JK_ST_PRE_GEMM, &n_cta);
+  if (rc != JK_OK) return rc;
+  JK_PROF(ctx, st, JK_ST_PRE_FIXUP);
+  jk_launch_pdl(k_tc_fix_linear, dim3(p.tiles_per_group, n_rows), dim3(128), 0, st, p, n_cta, Mrows,
+                (const float*)(ctx->ws + L.gemm_part), (const __nv_bfloat16*)bias,
+                (const __nv_bfloat16*)resid, resid_ld, (__nv_bfloat16*)out_bf16, out_f32, out_ld);
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
 }

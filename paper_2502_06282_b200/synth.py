@@ -177,6 +177,29 @@ def expert_weight(w: Workload, name: str, e: int) -> np.ndarray:
     return store_round(_normal(_rng(w.seed, 1000 + 3 * e + idx), shape, 0.02), w.dtype)
 
 
+def pre_weights(w: Workload, bias: bool = True) -> Dict[str, np.ndarray]:
+    """Random-init weights of the draft layer in front of the MoE (Sec. 3.1.2, Eq. 1): token
+    embedding [V, H] N(0, 1), reduction layer w_fc [H, 2H] and b_fc [H], w_qkv [(Hq + 2 Hkv) d, H]
+    (W_q rows, W_k rows, W_v rows), w_o [H, Hq d], all N(0, 0.02) but the embedding."""
+    r = lambda s: _rng(w.seed, s)
+    qd, kvd = w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim
+    out = {
+        "emb": _normal(r(21), (w.vocab, w.hidden), 1.0),
+        "w_fc": _normal(r(22), (w.hidden, 2 * w.hidden), 0.02),
+        "w_qkv": _normal(r(24), (qd + 2 * kvd, w.hidden), 0.02),
+        "w_o": _normal(r(25), (w.hidden, qd), 0.02),
+    }
+    if bias:
+        out["b_fc"] = _normal(r(23), (w.hidden,), 0.02)
+    return {k: store_round(v, w.dtype) for k, v in out.items()}
+
+
+def root_feature(w: Workload) -> np.ndarray:
+    """[B, H]: the target model's feature of the last committed token (the f_{i-1} the root's
+    token is paired with), N(0, 1)."""
+    return store_round(_normal(_rng(w.seed, 26), (w.batch, w.hidden), 1.0), w.dtype)
+
+
 def layer_hidden(w: Workload, layer: int, n_frontier: int) -> np.ndarray:
     """u [B, F, H]: post-attention hidden state of each frontier node (the
     output of Eq. 1), N(0, 1).  Stands in for the draft's reduction layer and

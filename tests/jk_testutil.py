@@ -96,8 +96,13 @@ def guarded_step_buffers(ctx, w, guard: Guard, bufs=None):
     for k in bufs.pool:
         bufs.pool[k] = guard.like(bufs.pool[k])
     bufs.pool_struct = ctx.pool_struct(bufs.pool)
-    for name in ("probs", "expert", "gate", "lse", "feat", "frontier"):
+    for name in ("probs", "expert", "gate", "feat", "frontier"):
         setattr(bufs, name, [guard.like(t) for t in getattr(bufs, name)])
+    if bufs.lse_all is not None:
+        bufs.lse_all = guard.like(bufs.lse_all)
+        bufs.lse = bufs.lse_views()
+    else:
+        bufs.lse = [guard.like(t) for t in bufs.lse]
     bufs.parent_score = [guard.like(bufs.parent_score[0], keep=True)] + [
         guard.like(t) for t in bufs.parent_score[1:]]
     bufs.parent_gidx = [guard.like(bufs.parent_gidx[0], keep=True)] + [
