@@ -53,6 +53,13 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="repeat the timed pass of --steps steps until this much time has passed")
+    ap.add_argument("--pre-block", action="store_true",
+                    help="chain jk_draft_pre in front of every expand call (u no longer synthetic)")
+    ap.add_argument("--head-mode", default="decoupled", choices=["decoupled", "contrastive"],
+                    help="contrastive: the hybrid schedule of Sec. 3.2 (D-1 draft passes)")
+    ap.add_argument("--tree", default="dynamic", choices=["dynamic", "static"],
+                    help="static: a predefined tree shape instead of the score-driven one")
+    ap.add_argument("--experts", type=int, default=0, help="candidate experts N (0 = workload's)")
     ap.add_argument("--sweep", action="store_true",
                     help="per-call timings over prefix length, tree size and batch at the 70B layer shape")
     ap.add_argument("--out", default="", help="also append every JSON line to this file")
@@ -206,14 +213,28 @@ def device_weights(w, wts_np, dev):
 # ------------------------------------------------------------------------------------------
 # the CPU oracle on a bounded sample of the workload
 # ------------------------------------------------------------------------------------------
-def oracle_sample(w, wts_np, us_np, attn_np, tree_np, tl_np, dl_np, ua, ub, mode):
+def kv_len_of(attn_np):
+    return attn_np[3][0]
+
+
+def oracle_sample(w, wts_np, us_np, attn_np, tree_np, tl_np, dl_np, ua, ub, mode, n_rows=None,
+                  pre_np=None):
     """Times the oracle as it stands on: the root row of the first draft layer, one head of one
     target layer, and the full acceptance walk; scales the first two to the whole step.
     Returns (seconds one step would take, seconds the sample took, parts)."""
     from oracle import jakiro_oracle as orc
     t_start = time.perf_counter()
     t0 = time.perf_counter()
-    orc.draft_expand(us_np[0][:1], np.zeros((1, 1)), wts_np, w.k_per_expert, w.width)
+    if w.head_mode == 1:
+        orc.draft_expand_contrastive(us_np[0][:1], np.zeros((1, 1)), wts_np, w.k_per_expert, w.width,
+                                     0.5, 1.0, False)
+    else:
+        orc.draft_expand(us_np[0][:1], np.zeros((1, 1)), wts_np, w.k_per_expert, w.width)
+    if pre_np is not None:                 # the root's pass through the draft layer before the MoE
+        pw, k0, v0, root_feat, theta = pre_np
+        orc.draft_pre_block(np.array([5]), root_feat[:1], pw, k0[0], v0[0], int(kv_len_of(attn_np)),
+                            [0], np.array([-1]), w.n_q_heads, w.n_kv_heads, theta,
+                            1.0 / math.sqrt(w.head_dim))
     t_row = time.perf_counter() - t0
     q, k, v, kv_len = attn_np
     t0 = time.perf_counter()
@@ -229,7 +250,7 @@ def oracle_sample(w, wts_np, us_np, attn_np, tree_np, tl_np, dl_np, ua, ub, mode
                                 tree_np["depth"][b], tree_np["branch"][b], tree_np["qslot"][b],
                                 dl_np[b], ua[b], ub[b], 1.0)
     t_acc = time.perf_counter() - t0
-    rows = w.n_slots * w.batch
+    rows = w.n_slots * w.batch if n_rows is None else n_rows
     est = t_row * rows + t_head * w.n_q_heads * w.n_layers * w.batch + t_acc
     return est, time.perf_counter() - t_start, {"expand_row_s": t_row, "attn_head_layer_s": t_head,
                                                 "accept_s": t_acc}
@@ -255,10 +276,21 @@ def workload_text(w) -> str:
             f"D={w.depth} k_e={w.k_per_expert} W={w.width} B={w.batch} L={w.n_layers}")
 
 
+def variant(args, w):
+    from paper_2502_06282_b200 import synth
+    if args.experts:
+        w = synth.scaled(w, n_experts=args.experts, name=f"{w.name}_n{args.experts}")
+    if args.head_mode == "contrastive":
+        w = synth.scaled(w, head_mode=1, name=f"{w.name}_contrastive")
+    return w
+
+
 def make_config(args, w):
     return {"workload": workload_text(w), "mode": args.mode,
+            "draft": {"pre_block": bool(args.pre_block), "head_mode": args.head_mode,
+                      "tree": args.tree, "expand_calls": w.n_passes},
             "temperature": 1.0 if args.mode == "sampling" else 0.0,
-            "calls_per_step": {"jk_draft_expand": w.depth, "jk_tree_finalize": 1,
+            "calls_per_step": {"jk_draft_expand": w.n_passes, "jk_tree_finalize": 1,
                                "jk_tree_verify_attn": w.n_layers, "jk_accept_and_compact": 1},
             "l2": "per-step inputs exceed L2: the draft weights of every expand call and "
                   f"{w.n_layers} distinct KV caches are streamed once per step"
@@ -287,9 +319,16 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     w = synth.WORKLOADS[name]
     if args.layers:
         w = synth.scaled(w, n_layers=args.layers)
+    w = variant(args, w)
     w = replicas.rank_workload(w, rank)                # every rank drafts its own sequences
     config = make_config(args, w)
     dev_index = torch.cuda.current_device()
+    plan = None
+    fs = w.frontier_sizes
+    if args.tree == "static":
+        from paper_2502_06282_b200.static_tree import plan_from_paths
+        plan = plan_from_paths(synth.static_paths(w), w.top_k, w.k_per_expert)
+        fs = plan["frontier_sizes"]
 
     def dev(a, dtype=None):
         t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
@@ -297,13 +336,34 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
 
     # ---------------------------------------------------------------- inputs, resident in HBM
     wts_np = host_weights(w)
-    us_np = [synth.layer_hidden(w, l, F) for l, F in enumerate(w.frontier_sizes)]
+    us_np = [synth.layer_hidden(w, l, F) for l, F in enumerate(fs)]
     wts = device_weights(w, wts_np, dev)
     us = [dev(u, w.dtype) for u in us_np]
-    ctx = jk.Context.for_workload(w)
-    bufs = jk.StepBuffers(ctx, w, keep_logits=True)
+    ctx = jk.Context.for_workload(w, frontier_sizes=fs, contrast_alpha=0.5, contrast_beta=1.0)
+    bufs = jk.StepBuffers(ctx, w, keep_logits=True, frontier_sizes=fs)
     wstruct = ctx.weights_struct(wts)
     root = torch.full((w.batch,), 5, dtype=torch.int32, device="cuda")
+    dplan = None
+    if plan is not None:
+        dplan = {"select": [dev(np.asarray(x, np.int32)) for x in plan["select"]],
+                 "keep": dev(np.asarray(plan["keep"], np.int32))}
+    pre = None
+    pre_np = None
+    if args.pre_block:
+        # the draft layer in front of the MoE: its weights, its own KV cache, the root's feature
+        pre = jk.PreBuffers(ctx, bufs)
+        _, dk, dv, _ = synth.attn_inputs(w, 90)
+        dkd, dvd = dev(dk, w.dtype), dev(dv, w.dtype)
+        root_feat_np = synth.root_feature(w)
+        root_feat = dev(root_feat_np, w.dtype)
+        pw_np = synth.pre_weights(w)
+        pw = {k: dev(v, w.dtype) for k, v in pw_np.items()}
+        pstruct = ctx.pre_weights_struct(pw)
+        qd0, kvd0 = w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim
+        pre_np = ({"emb": pw_np["emb"], "w_fc": pw_np["w_fc"], "b_fc": pw_np.get("b_fc"),
+                   "w_o": pw_np["w_o"], "w_q": pw_np["w_qkv"][:qd0],
+                   "w_k": pw_np["w_qkv"][qd0:qd0 + kvd0], "w_v": pw_np["w_qkv"][qd0 + kvd0:]},
+                  dk, dv, root_feat_np, 10000.0)
     L = w.n_layers
     attn0 = synth.attn_inputs(w, 0)
     qs, ks, vs = [], [], []
@@ -320,9 +380,16 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     scale = 1.0 / math.sqrt(w.head_dim)
     # with few target layers a step's caches fit L2: a buffer larger than L2 is written between steps
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if L <= 4 else None
+    def draft(inp):
+        if pre is not None:
+            jk.run_draft_chained(ctx, bufs, pre, wstruct, pstruct, inp["root"], inp["root_feat"],
+                                 dkd, dvd, kv_len0, 10000.0, scale)
+        else:
+            jk.run_draft(ctx, bufs, wstruct, inp["us"], inp["root"], static_plan=dplan)
+
     # the tree is a function of the inputs: one untimed draft gives it, and the target logits
     # are planted on it (agreement rate 0.8 per level)
-    jk.run_draft(ctx, bufs, wstruct, us, root)
+    draft({"us": us, "root": root, "root_feat": root_feat if pre is not None else None})
     torch.cuda.synchronize()
     tree_np = {k: v.cpu().numpy() for k, v in bufs.tree.items()}
     tl_np = synth.target_logits(w, tree_np["tok"], tree_np["parent"], 0.8)
@@ -332,17 +399,20 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     mode = 1 if args.mode == "sampling" else 0
 
     inA = {"us": us, "q_all": q_all, "tl": tl, "ua": ua, "ub": ub, "root": root}
+    if pre is not None:                     # the hidden states come from jk_draft_pre instead
+        inA["us"] = []
+        inA["root_feat"] = root_feat
 
     def step(inp=inA):
         if flush is not None:
             flush.zero_()
         kv_len.copy_(kv_len0)
-        jk.run_draft(ctx, bufs, wstruct, inp["us"], inp["root"])
+        draft(inp)
         for l in range(L):
             ctx.tree_verify_attn(w.batch, w.tree_size, inp["q_all"][l], ks[l], vs[l], kv_len,
                                  bufs.tree["parent"], scale, outs[l])
         ctx.accept_and_compact(w.batch, w.tree_size, mode, 1.0, inp["tl"], bufs.tree,
-                               bufs.logits if mode else None, w.n_slots,
+                               bufs.logits if mode else None, bufs.n_slots,
                                inp["ua"] if mode else None, inp["ub"] if mode else None, L, kp, vp,
                                ks[0].stride(0), ks[0].stride(1), ks[0].shape[2], kv_len,
                                bufs.n_acc, bufs.acc_idx, bufs.acc_tok, bufs.bonus)
@@ -411,7 +481,7 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     # that graph is replayed; every replay records the same events again.  The event nodes
     # serialise neighbouring kernels, so the sum of these times exceeds the step above, whose
     # kernels overlap their neighbours' tails through programmatic dependent launch.
-    launches_cap = 16 * w.depth + 1 + 2 * L + 3 + 16
+    launches_cap = 32 * w.depth + 1 + 2 * L + 3 + 16
     n_prof = min(args.steps, 20)
     prof = {}
     ctx.profile_enable(launches_cap)
@@ -451,11 +521,15 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     touched = [len(set(e.cpu().numpy().reshape(-1).tolist())) for e in bufs.expert]
     H, I, V = w.hidden, w.inter, w.vocab
     attn_bytes, attn_flops = attention_bytes_flops(w)
-    draft_rows = w.batch * w.n_slots * w.top_k if mode else 0
+    draft_rows = w.batch * bufs.n_slots * w.top_k if mode else 0
+    n_pass = len(fs)
+    qd_, kvd_ = w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim
     algo_bytes_per_step = {
         "expert_gate_up": sum(t * 2 * I * H * es for t in touched),
         "expert_down": sum(t * H * I * es for t in touched),
-        "lm_head": w.depth * V * H * es,
+        "lm_head": n_pass * V * H * es,
+        # the draft layer's three projections: W_fc [H, 2H], W_qkv, W_o
+        "pre_gemm": n_pass * (2 * H * H + (qd_ + 2 * kvd_) * H + H * qd_) * es,
         "tree_attn": L * attn_bytes,
         # target rows, and in sampling mode the stored draft rows it also reduces
         "row_stats": w.batch * w.tree_size * V * 4 + draft_rows * V * 4,
@@ -491,11 +565,13 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
         return round(sum(kernels[n]["ms_per_step"] for n in names if n in kernels), 4)
     groups["draft_ms"] = gsum(["router", "expert_gate_up", "gemm_fixup", "expert_down",
                                "branch_features", "lm_head", "topk_partial", "expand_finish",
-                               "tree_finalize"])
+                               "tree_finalize", "pre_gather", "pre_gemm", "pre_fixup", "pre_rope",
+                               "pre_attn", "pre_attn_combine"])
     groups["verify_attn_ms"] = gsum(["tree_attn", "attn_combine"])
     groups["accept_ms"] = gsum(["row_stats", "accept_walk", "kv_compact"])
     draft_bytes = (algo_bytes_per_step["expert_gate_up"] + algo_bytes_per_step["expert_down"]
-                   + algo_bytes_per_step["lm_head"])
+                   + algo_bytes_per_step["lm_head"]
+                   + (algo_bytes_per_step["pre_gemm"] if pre is not None else 0))
     if groups["draft_ms"] > 0:
         groups["draft_frac_of_peak"] = round(draft_bytes / (groups["draft_ms"] * 1e-3) / 1e9 / peak, 4)
     step_bytes = draft_bytes + algo_bytes_per_step["tree_attn"] + w.batch * w.tree_size * V * 4
@@ -521,13 +597,11 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
         # Inputs are double-buffered on the device: the copies of step s+1 run on a copy stream
         # while step s computes, and the results of step s are read while step s+1 runs.
         pin = lambda t: t.cpu().pin_memory()
-        hostA = {"us": [pin(u) for u in us], "q_all": pin(q_all), "tl": pin(tl), "ua": pin(ua),
-                 "ub": pin(ub), "root": pin(root)}
-        inB = {"us": [u.clone() for u in us], "q_all": q_all.clone(), "tl": tl.clone(),
-               "ua": ua.clone(), "ub": ub.clone(), "root": root.clone()}
+        hostA = {k: ([pin(u) for u in v] if isinstance(v, list) else pin(v)) for k, v in inA.items()}
+        inB = {k: ([u.clone() for u in v] if isinstance(v, list) else v.clone()) for k, v in inA.items()}
         sets = [inA, inB]
         runs = [run_step, (capture(inB).replay if graph is not None else (lambda: step(inB)))]
-        flat = lambda d: d["us"] + [d["q_all"], d["tl"], d["ua"], d["ub"], d["root"]]
+        flat = lambda d: d["us"] + [d[k] for k in sorted(d) if k != "us"]
         h2d = sum(t.numel() * t.element_size() for t in flat(hostA))
         results = (bufs.n_acc, bufs.acc_idx, bufs.acc_tok, bufs.bonus, kv_len)
         d2h = sum(t.numel() * t.element_size() for t in results)
@@ -580,7 +654,7 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dl_np = bufs.logits.cpu().numpy() if mode else None
         est, _, parts = oracle_sample(w, wts_np, us_np, attn0, tree_np, tl_np, dl_np, ua_np, ub_np,
-                                      args.mode)
+                                      args.mode, n_rows=bufs.n_slots * w.batch, pre_np=pre_np)
         cpu_baseline = {"value": 1.0 / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                         "sample": sample_text(w),
                         "parts_s": {k: round(v, 4) for k, v in parts.items()}}
@@ -588,7 +662,7 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
             from threadpoolctl import threadpool_limits
             with threadpool_limits(limits=1):
                 est1, _, _ = oracle_sample(w, wts_np, us_np, attn0, tree_np, tl_np, dl_np, ua_np,
-                                           ub_np, args.mode)
+                                           ub_np, args.mode, n_rows=bufs.n_slots * w.batch, pre_np=pre_np)
             cpu_baseline["single_thread"] = {"value": 1.0 / est1, "unit": UNIT, "cores": 1}
         except Exception as exc:
             cpu_baseline["single_thread"] = {"unavailable": str(exc)}
@@ -752,6 +826,7 @@ def main():
             w = synth.WORKLOADS[name]
             if args.layers:
                 w = synth.scaled(w, n_layers=args.layers)
+            w = variant(args, w)
             run_reference(args, w, make_config(args, w))
         return
 

@@ -250,6 +250,41 @@ def random_tree(m: int, max_depth: int, seed: int) -> np.ndarray:
     return np.asarray(parent, dtype=np.int32)
 
 
+def static_paths(w: Workload) -> List[Tuple[int, ...]]:
+    """A predefined tree shape of w.tree_size - 1 nodes and depth <= w.depth for the static
+    policy, as rank paths (rank c of a node = its c-th candidate in child order).  Level 1 takes
+    the root's candidates in order; below, the first w.width nodes of a level (in path order) are
+    expanded and handed children round-robin, best left-branch rank, best right-branch rank, second
+    left, second right, ..., until the node budget is spent."""
+    per_node = w.top_k * w.k_per_expert
+    order = []
+    for j in range(w.k_per_expert):
+        for r in range(w.top_k):
+            order.append(r * w.k_per_expert + j)
+    budget = w.tree_size - 1
+    paths: List[Tuple[int, ...]] = []
+    level = [(c,) for c in range(min(per_node, budget))]
+    paths += level
+    budget -= len(level)
+    for d in range(2, w.depth + 1):
+        parents = sorted(level)[:w.width]
+        left = w.depth - d                       # levels still to come below this one
+        here = budget if left == 0 else max(len(parents), budget // (left + 1))
+        here = min(here, budget, len(parents) * per_node)
+        nxt = []
+        i = 0
+        while len(nxt) < here:
+            p = parents[i % len(parents)]
+            nxt.append(p + (order[i // len(parents)],))
+            i += 1
+        paths += nxt
+        budget -= len(nxt)
+        level = nxt
+        if budget <= 0 or not level:
+            break
+    return paths
+
+
 def tree_depths(parent: np.ndarray) -> np.ndarray:
     d = np.zeros(len(parent), dtype=np.int32)
     for i in range(1, len(parent)):
