@@ -255,6 +255,36 @@ int jk_draft_pre(jk_ctx* ctx, void* stream, const jk_pre_weights* host_w,
                  const int32_t* kv_len, float rope_theta, float softmax_scale, void* out_u);
 
 /*
+ * The target layer's own steps in front of jk_tree_verify_attn in a verification pass (Sec. 2.1
+ * step 2: the target model evaluates all tree tokens in one forward pass): QKV projection of the
+ * M tree tokens, rotary positions, K/V written at the tree slots.
+ *   x        T [B, M, H]   the layer's (normalised) input hidden states of the tree tokens
+ *   w_qkv    T [(Hq + 2 Hkv) d, H]   rows of W_q, then W_k, then W_v
+ *   depth    i32 [B, M]    as written by jk_tree_finalize: node i sits at position kv_len[b] +
+ *            depth[i] (nodes of one depth are alternatives for the same place in the sequence)
+ *   q_out    T [B, M, Hq, d]   rotated queries (LLaMA pairing (i, i + d/2), base rope_theta)
+ *   k_cache, v_cache   rotated K and V of node i go to row kv_len[b] + i
+ * More than 256 tree tokens per call (B * M) go through the projection in chunks of 256 rows,
+ * each streaming W_qkv once.  Errors as jk_tree_verify_attn; kv_len[b] + M > cache_rows sets
+ * JK_ERR_BOUNDS.
+ */
+int jk_verify_qkv(jk_ctx* ctx, void* stream, const void* w_qkv, int32_t batch, int32_t tree_size,
+                  const void* x, const int32_t* depth, void* q_out, void* k_cache, void* v_cache,
+                  int64_t cache_stride_b, int64_t cache_stride_h, int32_t cache_rows,
+                  const int32_t* kv_len, float rope_theta);
+
+/*
+ * The hidden states the next draft round starts from (Sec. 2.1 step 3 keeps the accepted path):
+ *   out[b, 0] = hidden[b, 0] (the root), out[b, 1 + j] = hidden[b, acc_idx[b, j]] for
+ *   j < n_acc[b]; rows after the accepted path are zero.
+ *   hidden T [B, M, H]; n_acc i32 [B], acc_idx i32 [B, max_depth] as written by
+ *   jk_accept_and_compact; out T [B, rows_out, H], rows_out <= max_depth + 1.
+ */
+int jk_gather_accepted(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
+                       const void* hidden, const int32_t* n_acc, const int32_t* acc_idx,
+                       int32_t rows_out, void* out);
+
+/*
  * Build the verification tree from the pool (Sec. 3.1.2; mask as in Fig. 4): node 0 is the
  * root (root_tok[b]); nodes 1..M-1 are the M-1 best pool entries by (score descending,
  * generation index ascending), listed in ascending generation index, so parent[i] < i.

@@ -43,6 +43,12 @@ What each function follows:
                         passes from logits^moe, and logits^const of the last pass
                         proposing one token further, so that a tree of depth D
                         costs D-1 draft passes
+  verify_qkv_append, gather_accepted
+                        the target layer's own steps around tree attention in a
+                        verification pass (Sec. 2.1 step 2): QKV projection of
+                        the tree tokens, rotary positions by depth, K/V written
+                        at the tree slots; and the accepted nodes' hidden states
+                        picked out for the next draft round
   rope, draft_pre_block Eq. 1 and the Eagle-style input path described before
                         it (Sec. 3.1.2): token embedding and the parent's
                         feature concatenated, the reduction layer, then
@@ -730,3 +736,49 @@ def draft_pre_block(tok: np.ndarray, f_prev: np.ndarray, pw: Dict[str, np.ndarra
             o[hh] = softmax(scale * (kk @ qs[i, hh])) @ vv
         u[i] = np.asarray(pw["w_o"], dtype=F64) @ o.reshape(-1) + h[i]
     return u, h, kc, vc
+
+
+# --------------------------------------------------------------------------
+# verification-side glue around the tree attention (Sec. 2.1 step 2)
+# --------------------------------------------------------------------------
+def verify_qkv_append(x: np.ndarray, w_q: np.ndarray, w_k: np.ndarray, w_v: np.ndarray,
+                      depth: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
+                      prefix_len: int, n_q_heads: int, n_kv_heads: int, theta: float
+                      ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """One sequence, one target layer.  x [M, H] are the layer's input hidden
+    states of the M tree tokens.  q_i = rope(W_q x_i), k_i = rope(W_k x_i),
+    v_i = W_v x_i per head, rotated to position prefix_len + depth[i] (all
+    nodes of one depth share a position: they are alternatives for the same
+    place in the sequence); k_i, v_i go to cache row prefix_len + i, which is
+    where jk_tree_verify_attn expects the tree tokens.  Returns (q [M, Hq, d],
+    caches)."""
+    x = np.asarray(x, dtype=F64)
+    M = x.shape[0]
+    d = w_q.shape[0] // n_q_heads
+    kc = np.array(k_cache, dtype=F64, copy=True)
+    vc = np.array(v_cache, dtype=F64, copy=True)
+    q_out = np.zeros((M, n_q_heads, d), dtype=F64)
+    for i in range(M):
+        pos = prefix_len + int(depth[i])
+        q = (np.asarray(w_q, dtype=F64) @ x[i]).reshape(n_q_heads, d)
+        k = (np.asarray(w_k, dtype=F64) @ x[i]).reshape(n_kv_heads, d)
+        v = (np.asarray(w_v, dtype=F64) @ x[i]).reshape(n_kv_heads, d)
+        for hh in range(n_q_heads):
+            q_out[i, hh] = rope(q[hh], pos, theta)
+        for hh in range(n_kv_heads):
+            kc[hh, prefix_len + i] = rope(k[hh], pos, theta)
+            vc[hh, prefix_len + i] = v[hh]
+    return q_out, kc, vc
+
+
+def gather_accepted(hidden: np.ndarray, acc_idx: Sequence[int], rows: int) -> np.ndarray:
+    """hidden [M, H] of one sequence's tree tokens -> [rows, H]: row 0 is the
+    root's (always committed), row 1 + j the j-th accepted node's; rows past
+    the accepted path are zero.  These are the features the next draft round
+    starts from."""
+    hidden = np.asarray(hidden)
+    out = np.zeros((rows, hidden.shape[1]), dtype=hidden.dtype)
+    out[0] = hidden[0]
+    for j, a in enumerate(acc_idx):
+        out[1 + j] = hidden[int(a)]
+    return out

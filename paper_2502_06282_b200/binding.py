@@ -26,7 +26,8 @@ EXPORTS = ["jk_create", "jk_destroy", "jk_workspace_bytes", "jk_set_workspace", 
            "jk_tree_finalize", "jk_tree_verify_attn", "jk_accept_and_compact",
            "jk_profile_enable", "jk_profile_collect", "jk_profile_stage_count",
            "jk_profile_stage_name", "jk_tree_verify_attn_static", "jk_tensor_path_active",
-           "jk_set_attn_kernel", "jk_profile_read", "jk_draft_pre"]
+           "jk_set_attn_kernel", "jk_profile_read", "jk_draft_pre",
+           "jk_verify_qkv", "jk_gather_accepted"]
 
 
 class JkConfig(C.Structure):
@@ -96,6 +97,8 @@ def lib() -> C.CDLL:
         L.jk_draft_pre.argtypes = [vp, vp, C.POINTER(JkPreWeights), C.POINTER(JkPreState), i32, i32,
                                    i32, vp, C.POINTER(JkPool), i32, i32, i32, vp, vp, vp, vp, i64,
                                    i64, i32, vp, f32, f32, vp]
+        L.jk_verify_qkv.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i64, i64, i32, vp, f32]
+        L.jk_gather_accepted.argtypes = [vp, vp, i32, i32, vp, vp, vp, i32, vp]
         L.jk_profile_enable.argtypes = [vp, i32]
         L.jk_profile_collect.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
         L.jk_profile_read.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(i32)]
@@ -269,6 +272,20 @@ class Context:
                                 _ptr(k_cache), _ptr(v_cache), k_cache.stride(0), k_cache.stride(1),
                                 rows, _ptr(kv_len), float(rope_theta), float(scale), _ptr(out_u))
         self._check(rc, "jk_draft_pre")
+
+    def verify_qkv(self, w_qkv, batch, tree_size, x, depth, q_out, k_cache, v_cache, kv_len,
+                   rope_theta, cache_rows=None):
+        rows = k_cache.shape[2] if cache_rows is None else cache_rows
+        rc = lib().jk_verify_qkv(self._h, _stream(), _ptr(w_qkv), batch, tree_size, _ptr(x),
+                                 _ptr(depth), _ptr(q_out), _ptr(k_cache), _ptr(v_cache),
+                                 k_cache.stride(0), k_cache.stride(1), rows, _ptr(kv_len),
+                                 float(rope_theta))
+        self._check(rc, "jk_verify_qkv")
+
+    def gather_accepted(self, batch, tree_size, hidden, n_acc, acc_idx, rows_out, out):
+        rc = lib().jk_gather_accepted(self._h, _stream(), batch, tree_size, _ptr(hidden),
+                                      _ptr(n_acc), _ptr(acc_idx), rows_out, _ptr(out))
+        self._check(rc, "jk_gather_accepted")
 
     def tree_finalize(self, batch, pool, pool_n, root_tok, tree_size, tok, parent, depth, branch,
                       qslot, anc, static_keep=None):

@@ -83,7 +83,8 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   const size_t qkvd = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
   L->pre_x = take(Rp * 2 * c.hidden * es);
   L->pre_h = take(Rp * c.hidden * es);
-  L->pre_qkv = take(Rp * qkvd * 4);
+  const size_t vrows = jk_align_up(BM, 16);                 // jk_verify_qkv: all tree tokens
+  L->pre_qkv = take((Rp > vrows ? Rp : vrows) * qkvd * 4);
   L->pre_qd = take((size_t)c.max_batch * S * qd * es);
   L->pre_par = take((size_t)c.max_batch * S * 4);
   L->pre_att = take((size_t)c.max_batch * S * qd * es);

@@ -73,17 +73,6 @@ __device__ __forceinline__ float4 acl_ld_f32x4(uint32_t a) {
                : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
   return v;
 }
-// D[tmem] (+)= A[tmem] * B[smem], bf16 inputs, fp32 accumulate: A is read from tensor memory
-// (128 lanes x K/2 columns, two consecutive K elements per 32-bit column)
-__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b,
-                                               uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 __device__ __forceinline__ void acl_pair_sync(int quarter) {
   // the two warps that share 32 query rows (64 threads); ids 1..4, 0 is __syncthreads
   asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");

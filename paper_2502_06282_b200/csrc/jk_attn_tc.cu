@@ -6,12 +6,13 @@
 // tiles.  Per tile of 128 keys:
 //   TMA brings K [128 keys x d] and V [128 keys x d] into swizzled shared memory;
 //   S = Q K^T on the tensor core into tensor memory (128 x 128 fp32);
-//   two threads own one query row: each reads the whole row of S for the maximum (so the two agree
-//   without an exchange), applies the tree mask (a 128-bit visibility word built from the node's
-//   ancestor set and the prefix length), keeps the running max and the sum of its 64 keys, and
-//   writes P = exp(S - max) for those keys as bf16 into the shared memory K just left;
-//   O (+)= P V on the tensor core, V taken MN-major straight from its row-major tile; when the
-//   running max moved, O is first rescaled in tensor memory.
+//   two threads own one query row, 64 keys each: one read of S into registers, the tree mask (a
+//   128-bit visibility word built from the node's ancestor set and the prefix length), the two
+//   halves' maxima exchanged through shared memory, P = exp(S - max) packed to bf16 and stored
+//   back into tensor memory over S;
+//   O (+)= P V on the tensor core, P taken from tensor memory as the A operand, V MN-major straight
+//   from its row-major tile; the reference maximum only moves when it is outgrown by more than
+//   2^8, so O is rarely rescaled.
 // The CTA writes an unnormalised partial (max, sum, O) per row; the merge kernel of jk_attn.cu
 // combines the slices.  96 KB of shared memory and 256 tensor-memory columns per CTA: two CTAs
 // share an SM and overlap each other's copy and math phases.  All mbarrier waits are bounded.
@@ -29,6 +30,7 @@ struct atc_tail {
   uint32_t tmem_base;
   int abort_flag;
   int parent[JK_MAX_TREE];
+  float xmax[2][ATC_ROWS];             // [key half][row]: the half's visible maximum of a tile
   float xsum[2][ATC_ROWS];             // [key half][row]: the half's sum of exponentials
 };
 
@@ -62,13 +64,6 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
   const int tid = threadIdx.x, warp = tid >> 5;
   const int quarter = warp & 3, half = warp >> 2;
   const int row = quarter * 32 + (tid & 31);
-  jk_pdl_wait();
-  const int P = kv_len[b];
-  const int Ltot = P + M;
-  if (P < 0 || Ltot > cache_rows) {
-    if (tid == 0) jk_set_status(status, JK_ERR_BOUNDS);
-    return;                                    // (a CTA that exits counts as having released)
-  }
   const int n_rows = G * M;
   const int row0 = qblk * ATC_ROWS;
   const bool row_valid = row0 + row < n_rows;
@@ -77,7 +72,27 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
   const int node = row_valid ? (row0 + row) % M : 0;
   const size_t n_out = (size_t)gridDim.z * M * Hq;
   const size_t orow = ((size_t)b * M + node) * Hq + kvh * G + g_idx;
-  const int tiles_total = (Ltot + ATC_KEYS - 1) / ATC_KEYS;
+  // barriers and tensor memory touch no global memory: set up before the grid-dependency wait
+  if (tid == 0) {
+    mbar_init(&T.bar_k, 1); mbar_init(&T.bar_v, 1); mbar_init(&T.bar_s, 1); mbar_init(&T.bar_o, 1);
+    T.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    tmem_alloc(&T.tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  // Before the grid-dependency wait the kernel may only read what no kernel it can overlap with
+  // writes.  That holds for kv_len and for the committed prefix rows of the caches (rows below
+  // kv_len[b]): they are written by the acceptance call of an earlier step, whose kernels release
+  // their dependents only when they exit, so they are complete before this kernel starts.  A key
+  // tile that lies wholly in the prefix is therefore asked for right away and travels while the
+  // kernel before (typically the previous layer's merge) is still running; the tree rows, Q and
+  // parent[] are fresh and wait.
+  const int P = kv_len[b];
+  const int Ltot = P + M;
+  const bool bad = P < 0 || Ltot > cache_rows;
+  const int tiles_total = bad ? 0 : (Ltot + ATC_KEYS - 1) / ATC_KEYS;
   const int tiles_per = (tiles_total + n_split - 1) / n_split;
   const int t0 = split * tiles_per;
   const int t1 = min(tiles_total, t0 + tiles_per);
@@ -86,45 +101,40 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
   uint32_t tmem_base = 0;
   float m_run = -INFINITY, l_run = 0.f;
 
+  auto issue_kv = [&](int tile) {
+    const uint64_t pol = l2_policy_evict_first();   // the cache is read once per call
+    mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb)
+      tma_load_4d_hint(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k, pol);
+    mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb)
+      tma_load_4d_hint(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v, pol);
+  };
+  const bool early = have_keys && (t0 + 1) * ATC_KEYS <= P;
+  if (early && tid == 0) issue_kv(t0);
+  jk_pdl_wait();
+  if (bad && tid == 0) jk_set_status(status, JK_ERR_BOUNDS);
+  // The query block is asked for first: its loads travel while thread 0 starts the K/V copies.
+  constexpr int QV = ATC_ROWS * (D / 8) / ATC_THREADS;   // 16-byte vectors per thread
+  uint4 qv[QV];
+#pragma unroll
+  for (int it = 0; it < QV; ++it) {
+    const int idx = tid + it * ATC_THREADS;
+    const int rr = idx / (D / 8), ch = idx % (D / 8);
+    qv[it] = make_uint4(0u, 0u, 0u, 0u);
+    if (row0 + rr < n_rows) {
+      const int gg = (row0 + rr) / M, ii = (row0 + rr) % M;
+      qv[it] = __ldg(reinterpret_cast<const uint4*>(
+          q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8));
+    }
+  }
+  const int par_mine = tid < M ? __ldg(parent + (size_t)b * M + tid) : -1;
+  if (have_keys && !early && tid == 0) issue_kv(t0);
   if (have_keys) {
-    auto issue_kv = [&](int tile) {
-      const uint64_t pol = l2_policy_evict_first();   // the cache is read once per call
-      mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
-#pragma unroll
-      for (int kb = 0; kb < KB; ++kb)
-        tma_load_4d_hint(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k, pol);
-      mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
-#pragma unroll
-      for (int kb = 0; kb < KB; ++kb)
-        tma_load_4d_hint(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v, pol);
-    };
-
-    if (tid == 0) {
-      mbar_init(&T.bar_k, 1); mbar_init(&T.bar_v, 1); mbar_init(&T.bar_s, 1); mbar_init(&T.bar_o, 1);
-      T.abort_flag = 0;
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-      issue_kv(t0);
-    }
-    if (warp == 0) {
-      tmem_alloc(&T.tmem_base, TMEM_COLS);
-      tmem_relinquish();
-    }
-    if (tid < M) T.parent[tid] = parent[(size_t)b * M + tid];
+    if (tid < M) T.parent[tid] = par_mine;
     // Q block -> shared memory in the K-major 128-byte-swizzled layout the MMA reads
-    // (all loads are issued before the first store, so that they overlap)
-    constexpr int QV = ATC_ROWS * (D / 8) / ATC_THREADS;   // 16-byte vectors per thread
-    uint4 qv[QV];
-#pragma unroll
-    for (int it = 0; it < QV; ++it) {
-      const int idx = tid + it * ATC_THREADS;
-      const int rr = idx / (D / 8), ch = idx % (D / 8);
-      qv[it] = make_uint4(0u, 0u, 0u, 0u);
-      if (row0 + rr < n_rows) {
-        const int gg = (row0 + rr) / M, ii = (row0 + rr) % M;
-        qv[it] = __ldg(reinterpret_cast<const uint4*>(
-            q + (((size_t)b * M + ii) * Hq + kvh * G + gg) * D + ch * 8));
-      }
-    }
 #pragma unroll
     for (int it = 0; it < QV; ++it) {
       const int idx = tid + it * ATC_THREADS;
@@ -133,10 +143,13 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       *reinterpret_cast<uint4*>(sq + kb * 16384 + rr * 128 + ((cb ^ (rr & 7)) << 4)) = qv[it];
     }
     fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    tmem_base = T.tmem_base;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  tmem_base = T.tmem_base;
+  if (bad) ok = false;
+  if (have_keys) {
     // ancestor set of this thread's node (Fig. 4), walked in shared memory
     unsigned long long anc_lo = 0ull, anc_hi = 0ull;
     if (row_valid) {
@@ -168,9 +181,10 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
           tc_commit(&T.bar_s);
         }
       }
-      // visibility of keys key0 .. key0+127 for this row: prefix keys, then the ancestor set
-      unsigned long long vis_lo = 0ull, vis_hi = 0ull;
+      // visibility of this thread's 64 keys (Fig. 4): prefix keys, then the ancestor set
+      unsigned long long vis = 0ull;
       if (row_valid) {
+        unsigned long long vis_lo = 0ull, vis_hi = 0ull;
         const int s = P - tile * ATC_KEYS;
         if (s >= 128) { vis_lo = ~0ull; vis_hi = ~0ull; }
         else if (s >= 0) {
@@ -187,64 +201,65 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
           if (t < 64) { vis_lo = (anc_lo >> t) | (anc_hi << (64 - t)); vis_hi = anc_hi >> t; }
           else if (t < 128) { vis_lo = anc_hi >> (t - 64); vis_hi = 0ull; }
         }
+        vis = half ? vis_hi : vis_lo;
       }
+      const unsigned b0 = (unsigned)vis, b1 = (unsigned)(vis >> 32);
       ok = ok && mbar_wait(&T.bar_s, ph, abort_flag, status);
       if (!__syncthreads_and(ok)) { ok = false; break; }
       tc_fence_after();
 
-      // (warps whose 32 rows all lie past the last query row skip the row work: their rows of P
-      // and O are never stored)
+      // ---- this thread's half row of S, read once.  (Warps whose 32 rows all lie past the last
+      // query row skip the row work: their rows of P and O are never stored.)
+      const uint32_t sa = tmem_base + lane_base + (uint32_t)half * 64u;
+      uint32_t r0[32], r1[32];
+      float mx = -INFINITY;
       if (warp_has_rows) {
-        // pass 1: the row maximum over all 128 keys.  Both threads of a row compute it from the
-        // same values in the same order, so they agree bit for bit without an exchange.
-        float mx = -INFINITY;
+        tmem_ld32(sa, r0);
+        tmem_ld32(sa + 32u, r1);
+        tmem_ld_wait();
 #pragma unroll
-        for (int hh = 0; hh < 4; ++hh) {
-          uint32_t r0[32];
-          tmem_ld32(tmem_base + lane_base + (uint32_t)(hh * 32), r0);
-          tmem_ld_wait();
-          const unsigned long long v = (hh & 2) ? vis_hi : vis_lo;
-          const unsigned b0 = (hh & 1) ? (unsigned)(v >> 32) : (unsigned)v;
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
+        for (int j = 0; j < 32; ++j) {
+          if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
+          if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r1[j]));
         }
-        const float m_new = fmaxf(m_run, mx);
-        const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
-                                                 : fast_exp2((m_run - m_new) * sl2);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        // pass 2: P = exp(S - max) as bf16 for this thread's 64 keys, over the K tile (S, its only
-        // reader, has completed)
-        float lsum = 0.f;
-        unsigned char* prow = skp + half * 16384 + row * 128;
-        const unsigned long long vh = half ? vis_hi : vis_lo;
+      }
+      T.xmax[half][row] = mx;
+      tc_fence_before();
+      // the two warps that share 32 query rows meet (64 threads; barrier ids 1..4): both halves
+      // have S in registers and their maximum out, so P may overwrite S
+      asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");
+      tc_fence_after();
+      mx = fmaxf(mx, T.xmax[half ^ 1][row]);
+      // The reference maximum moves only when the row maximum outgrows it by more than 2^8.
+      float alpha = 1.f;
+      if (mx != -INFINITY && (m_run == -INFINITY || (mx - m_run) * sl2 > 8.f)) {
+        alpha = (m_run == -INFINITY) ? 0.f : fast_exp2((m_run - mx) * sl2);
+        m_run = mx;
+      }
+      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+      // ---- P = exp(S - max) as bf16, two keys per 32-bit column, back into tensor memory over
+      // S (its only reader, this thread pair, is done with it)
+      float lsum = 0.f;
+      if (warp_has_rows) {
+        uint32_t pk[32];
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          uint32_t r[32];
-          tmem_ld32(tmem_base + lane_base + (uint32_t)(half * 64 + hh * 32), r);
-          tmem_ld_wait();
-          const unsigned bits = hh ? (unsigned)(vh >> 32) : (unsigned)vh;
-          uint32_t pk[16];
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(r[j]) - m_use) * sl2) : 0.f;
-            const float p1 = ((bits >> (j + 1)) & 1u)
-                                 ? fast_exp2((__uint_as_float(r[j + 1]) - m_use) * sl2) : 0.f;
-            lsum += p0 + p1;
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-          }
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
-            const int cb = hh * 4 + cc;
-            *reinterpret_cast<uint4*>(prow + ((cb ^ (row & 7)) << 4)) =
-                make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-          }
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = ((b0 >> j) & 1u) ? fast_exp2((__uint_as_float(r0[j]) - m_use) * sl2) : 0.f;
+          const float p1 = ((b0 >> (j + 1)) & 1u)
+                               ? fast_exp2((__uint_as_float(r0[j + 1]) - m_use) * sl2) : 0.f;
+          const float p2 = ((b1 >> j) & 1u) ? fast_exp2((__uint_as_float(r1[j]) - m_use) * sl2) : 0.f;
+          const float p3 = ((b1 >> (j + 1)) & 1u)
+                               ? fast_exp2((__uint_as_float(r1[j + 1]) - m_use) * sl2) : 0.f;
+          const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+          const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+          // the sum runs over the rounded values the second product will use
+          lsum += (__low2float(h01) + __high2float(h01)) + (__low2float(h23) + __high2float(h23));
+          pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+          pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
         }
-        l_run = l_run * alpha + lsum;
-        m_run = m_new;
+        tmem_st32(tmem_base + lane_base + (uint32_t)half * 32u, pk);
         // rescale this thread's half of the running output when some row of the warp moved its
-        // maximum (the previous tile's P V product has completed: the loop waits for it)
+        // reference (the previous tile's P V product has completed: the loop waits for it)
         if (tile > t0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
           for (int c = 0; c < D / 64; ++c) {
@@ -256,9 +271,10 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
             for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
             tmem_st32(oa, r);
           }
-          tmem_st_wait();
         }
+        tmem_st_wait();
       }
+      l_run = l_run * alpha + lsum;
       // Cache rows past the last live key (only the sequence's last tile has any) may hold
       // anything, NaN bit patterns included, and 0 * NaN would poison every output row: they are
       // cleared in the V tile before the second product reads it.
@@ -273,20 +289,20 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
                 make_uint4(0u, 0u, 0u, 0u);
           }
         }
+        fence_proxy_async_smem();
       }
-      fence_proxy_async_smem();
       tc_fence_before();
       __syncthreads();
       if (tid == 0) {
         ok = ok && mbar_wait(&T.bar_v, ph, abort_flag, status);
         if (ok) {
           tc_fence_after();
-          const uint32_t pa = smem_u32(skp), va = smem_u32(sv);
+          const uint32_t va = smem_u32(sv);
 #pragma unroll
           for (int j = 0; j < ATC_KEYS / 16; ++j)
-            tc_mma_bf16(tmem_base + O_COL, smem_desc_sw128(pa + (j >> 2) * 16384 + (j & 3) * 32),
-                        smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
-                        (tile > t0 || j > 0) ? 1u : 0u);
+            tc_mma_bf16_ts(tmem_base + O_COL, tmem_base + (uint32_t)(j * 8),
+                           smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
+                           (tile > t0 || j > 0) ? 1u : 0u);
           tc_commit(&T.bar_o);
         }
       }
@@ -296,7 +312,7 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
     }
     if (ok) {
-      // The partial O goes through shared memory (over the K/P and V tiles: every MMA has
+      // The partial O goes through shared memory (over the K and V tiles: every MMA has
       // completed) so that it leaves in whole 512-byte rows: a thread per row storing straight
       // from its registers would touch 32 different rows with every store instruction.
       // 16-byte chunk c of row t sits at chunk index c * 128 + (t ^ c), which the row-per-lane
@@ -335,20 +351,20 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       while (global_ns() - ts < 2000000ull) { /* 2 ms: far longer than any TMA copy */ }
     }
     T.xsum[half][row] = l_run;
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) {
-      tc_fence_after();
-      tmem_dealloc(tmem_base, TMEM_COLS);
-    }
   }
-  // Only now may the next kernel of the stream be scheduled: CTAs of a dependent grid that sit on
-  // an SM in their grid-dependency wait were measured to slow the warps still working there.
-  jk_pdl_trigger();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
   if (row_valid && ok && half == 0) {
     part_ml[((size_t)split * n_out + orow) * 2] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
     part_ml[((size_t)split * n_out + orow) * 2 + 1] = have_keys ? l_run + T.xsum[1][row] : 0.f;
   }
+  // Only now may the next kernel of the stream be scheduled: CTAs of a dependent grid that sit on
+  // an SM in their grid-dependency wait were measured to slow the warps still working there.
+  jk_pdl_trigger();
 }
 
 // jk_attn.cu

@@ -19,7 +19,7 @@
 #define JK_ATTN_MAX_SPLIT 32
 
 struct jk_ws_layout {
-  size_t status;        // int32[4]
+  size_t status;        // int32[4]: the only part of the workspace that has to start at zero
   size_t xn;            // T   [Rp, H]       normalised hidden states
   size_t probs;         // f32 [R, N]
   size_t expert;        // i32 [R, K]

@@ -775,8 +775,8 @@ __global__ void __launch_bounds__(128) k_tc_fix_linear(
   else out_f32[(size_t)r * out_ld + o] = v;
 }
 
-// x: bf16 [x_rows, Kdim] (x_rows >= n_rows rounded up to 16: the workspace sections are), W: bf16
-// [Mrows, Kdim].  The weights do not depend on the kernel before: their first ring is prefetched.
+// x: bf16 [x_rows, Kdim] with x_rows >= n_rows (the copy's box is n_rows rounded up to 16: rows
+// past x_rows are filled with zeros by the copy engine), W: bf16 [Mrows, Kdim].  The weights do not depend on the kernel before: their first ring is prefetched.
 int jk_tc_linear(jk_ctx* ctx, cudaStream_t st, const void* W, int Mrows, int Kdim, const void* x,
                  int x_rows, int n_rows, const void* bias, const void* resid, long long resid_ld,
                  void* out_bf16, float* out_f32, long long out_ld) {
@@ -787,7 +787,7 @@ int jk_tc_linear(jk_ctx* ctx, cudaStream_t st, const void* W, int Mrows, int Kdi
   memset(&p, 0, sizeof(p));
   p.R = 0; p.K_top = ctx->cfg.top_k; p.n_experts = ctx->cfg.n_experts;
   const int n_pad = (int)jk_align_up(n_rows, 16);
-  if (n_pad > x_rows || n_pad > 256) return JK_ERR_SHAPE;
+  if (n_rows > x_rows || n_pad > 256) return JK_ERR_SHAPE;   // (rows of the box past x_rows read as zero)
   CUtensorMap aw, bx;
   if (!tc_map(ctx, s, W, Mrows, Kdim, TC_TILE_M, &aw) || !tc_map(ctx, s, x, x_rows, Kdim, n_pad, &bx))
     return JK_ERR_CUDA;

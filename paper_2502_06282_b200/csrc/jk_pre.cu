@@ -316,3 +316,100 @@ extern "C" int jk_draft_pre(jk_ctx* ctx, void* stream, const jk_pre_weights* w,
                          k_cache, v_cache, cache_stride_b, cache_stride_h, cache_rows, kv_len,
                          rope_theta, softmax_scale, out_u);
 }
+
+// ------------------------------------------------------------------------------------------
+// Verification-side steps around the tree attention of one target layer (Sec. 2.1 step 2)
+// ------------------------------------------------------------------------------------------
+extern "C" int jk_verify_qkv(jk_ctx* ctx, void* stream, const void* w_qkv, int32_t batch,
+                             int32_t tree_size, const void* x, const int32_t* depth, void* q_out,
+                             void* k_cache, void* v_cache, int64_t cache_stride_b,
+                             int64_t cache_stride_h, int32_t cache_rows, const int32_t* kv_len,
+                             float rope_theta) {
+  if (!ctx || !w_qkv || !x || !depth || !q_out || !k_cache || !v_cache || !kv_len) return JK_ERR_NULL;
+  const jk_config& c = ctx->cfg;
+  if (batch < 1 || tree_size < 1 || cache_rows < tree_size || !(rope_theta > 0.f)) return JK_ERR_SHAPE;
+  if (batch > c.max_batch || tree_size > c.max_tree) return JK_ERR_CAPACITY;
+  if (cache_stride_h < (int64_t)cache_rows * c.head_dim) return JK_ERR_SHAPE;
+  const void* ptrs[] = {w_qkv, x, q_out, k_cache, v_cache};
+  for (const void* p : ptrs)
+    if (!jk_aligned16(p)) return JK_ERR_ALIGN;
+  const int es = jk_elem_size(c.dtype);
+  if ((cache_stride_b * es) % 16 || (cache_stride_h * es) % 16) return JK_ERR_ALIGN;
+  if (!ctx->ws) return JK_ERR_WORKSPACE;
+  int rc = jk_ensure_device_info(ctx);
+  if (rc != JK_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const jk_ws_layout& L = ctx->lay;
+  const int R = batch * tree_size, H = c.hidden, Hq = c.n_q_heads, Hkv = c.n_kv_heads, D = c.head_dim;
+  const int qkvd = (Hq + 2 * Hkv) * D;
+  float* qkv = (float*)(ctx->ws + L.pre_qkv);
+  int32_t* status = (int32_t*)(ctx->ws + L.status);
+  const bool tc = ctx->tensor_path && c.dtype == JK_BF16 && jk_tc_available(ctx);
+  // the streaming GEMM takes at most 256 activation rows: larger batches of tree tokens go
+  // through it in row chunks (each chunk streams W_qkv once)
+  for (int r0 = 0; r0 < R; r0 += 256) {
+    const int nr = R - r0 < 256 ? R - r0 : 256;
+    const char* xr = (const char*)x + (size_t)r0 * H * es;
+    if (c.dtype == JK_BF16)
+      rc = linear<__nv_bfloat16>(ctx, st, tc, w_qkv, qkvd, H, xr, nr, nr, nullptr, nullptr, 0, nullptr,
+                                 qkv + (size_t)r0 * qkvd, qkvd);
+    else
+      rc = linear<float>(ctx, st, false, w_qkv, qkvd, H, xr, nr, nr, nullptr, nullptr, 0, nullptr,
+                         qkv + (size_t)r0 * qkvd, qkvd);
+    if (rc != JK_OK) return rc;
+  }
+  JK_PROF(ctx, st, JK_ST_PRE_ROPE);
+  if (c.dtype == JK_BF16)
+    jk_launch_pdl(k_pre_rope_scatter<__nv_bfloat16>, dim3(R), dim3(256), 0, st, (const float*)qkv,
+                  tree_size, Hq, Hkv, D, rope_theta, kv_len, depth, 0, (long long)tree_size,
+                  (__nv_bfloat16*)q_out, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache,
+                  (long long)cache_stride_b, (long long)cache_stride_h, cache_rows, status);
+  else
+    jk_launch_pdl(k_pre_rope_scatter<float>, dim3(R), dim3(256), 0, st, (const float*)qkv, tree_size,
+                  Hq, Hkv, D, rope_theta, kv_len, depth, 0, (long long)tree_size, (float*)q_out,
+                  (float*)k_cache, (float*)v_cache, (long long)cache_stride_b,
+                  (long long)cache_stride_h, cache_rows, status);
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}
+
+// out[b, 0] = hidden[b, 0]; out[b, 1 + j] = hidden[b, acc_idx[b, j]] for j < n_acc[b]; zero after.
+__global__ void __launch_bounds__(256) k_gather_accepted(
+    const uint4* __restrict__ hidden, const int32_t* __restrict__ n_acc,
+    const int32_t* __restrict__ acc_idx, int M, int max_depth, int row16, int rows_out,
+    uint4* __restrict__ out, int32_t* status) {
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  const int b = blockIdx.y, j = blockIdx.x;                 // output row j of sequence b
+  const int n = n_acc[b];
+  int src = -1;
+  if (j == 0) src = 0;
+  else if (j - 1 < n && j - 1 < max_depth) src = acc_idx[(size_t)b * max_depth + j - 1];
+  if (src >= M) {
+    if (threadIdx.x == 0) jk_set_status(status, JK_ERR_BOUNDS);
+    src = -1;
+  }
+  uint4* o = out + ((size_t)b * rows_out + j) * row16;
+  const uint4* h = hidden + ((size_t)b * M + (src < 0 ? 0 : src)) * row16;
+  for (int i = threadIdx.x; i < row16; i += blockDim.x)
+    o[i] = src < 0 ? make_uint4(0u, 0u, 0u, 0u) : h[i];
+}
+
+extern "C" int jk_gather_accepted(jk_ctx* ctx, void* stream, int32_t batch, int32_t tree_size,
+                                  const void* hidden, const int32_t* n_acc, const int32_t* acc_idx,
+                                  int32_t rows_out, void* out) {
+  if (!ctx || !hidden || !n_acc || !acc_idx || !out) return JK_ERR_NULL;
+  const jk_config& c = ctx->cfg;
+  if (batch < 1 || tree_size < 1 || rows_out < 1 || rows_out > c.max_depth + 1) return JK_ERR_SHAPE;
+  if (batch > c.max_batch || tree_size > c.max_tree) return JK_ERR_CAPACITY;
+  if (!jk_aligned16(hidden) || !jk_aligned16(out)) return JK_ERR_ALIGN;
+  if (!ctx->ws) return JK_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int row16 = c.hidden * jk_elem_size(c.dtype) / 16;
+  JK_PROF(ctx, st, JK_ST_COMPACT);
+  jk_launch_pdl(k_gather_accepted, dim3(rows_out, batch), dim3(256), 0, st, (const uint4*)hidden,
+                n_acc, acc_idx, tree_size, c.max_depth, row16, rows_out, (uint4*)out,
+                (int32_t*)(ctx->ws + ctx->lay.status));
+  JK_LAUNCH_CHECK(ctx);
+  return JK_OK;
+}

@@ -76,9 +76,11 @@ def guarded_context(w, **kw):
     n = ctx.workspace_bytes
     pad = 512
     raw = torch.full((pad + n + pad + 256,), Guard.CANARY, dtype=torch.uint8, device="cuda")
-    off = ctx.set_workspace(raw, pad)             # also clears the status word
-    torch.cuda.synchronize()
-    raw[off + 256:off + n] = Guard.POISON         # everything but the status section
+    first = (raw.data_ptr() + pad + 255) // 256 * 256 - raw.data_ptr()
+    raw[first:first + n] = Guard.POISON           # poison first: jk_set_workspace then clears
+    torch.cuda.synchronize()                      # the part that has to start at zero
+    off = ctx.set_workspace(raw, pad)
+    assert off == first
 
     def check():
         torch.cuda.synchronize()

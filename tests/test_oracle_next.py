@@ -320,3 +320,46 @@ def test_pre_block_uniform_attention_closed_form():
     mean_v = vc2[:, cols].mean(axis=1)                                     # [Hkv, d]
     o = np.stack([mean_v[hh // (Hq // Hkv)] for hh in range(Hq)]).reshape(-1)
     assert np.allclose(us[4][0], pw["w_o"] @ o + us[4][1], atol=1e-10)
+
+
+# ----------------------------------------------------------------- verification-side glue
+def test_verify_qkv_append_against_loops_and_the_attention_it_feeds():
+    rng = np.random.default_rng(20)
+    M, H, Hq, Hkv, d, P, cap = 5, 6, 4, 2, 4, 3, 12
+    x = rng.standard_normal((M, H))
+    wq, wk, wv = (rng.standard_normal((Hq * d, H)), rng.standard_normal((Hkv * d, H)),
+                  rng.standard_normal((Hkv * d, H)))
+    parent = np.array([-1, 0, 0, 1, 3])
+    depth = np.array([0, 1, 1, 2, 3])
+    kc, vc = rng.standard_normal((Hkv, cap, d)), rng.standard_normal((Hkv, cap, d))
+    q, kc2, vc2 = orc.verify_qkv_append(x, wq, wk, wv, depth, kc, vc, P, Hq, Hkv, 77.0)
+    for i in range(M):
+        for hh in range(Hq):
+            raw = [sum(wq[hh * d + c, j] * x[i, j] for j in range(H)) for c in range(d)]
+            assert np.allclose(q[i, hh], orc.rope(np.array(raw), P + depth[i], 77.0), atol=1e-12)
+        for hh in range(Hkv):
+            raw = [sum(wk[hh * d + c, j] * x[i, j] for j in range(H)) for c in range(d)]
+            assert np.allclose(kc2[hh, P + i], orc.rope(np.array(raw), P + depth[i], 77.0), atol=1e-12)
+            raw = [sum(wv[hh * d + c, j] * x[i, j] for j in range(H)) for c in range(d)]
+            assert np.allclose(vc2[hh, P + i], raw, atol=1e-12)        # V is not rotated
+    untouched = [r for r in range(cap) if not P <= r < P + M]
+    assert np.array_equal(kc2[:, untouched], kc[:, untouched])
+    # siblings (nodes 1 and 2, both depth 1) share a position: equal inputs give equal q and k
+    x2 = x.copy()
+    x2[2] = x2[1]
+    q2, k2, _ = orc.verify_qkv_append(x2, wq, wk, wv, depth, kc, vc, P, Hq, Hkv, 77.0)
+    assert np.array_equal(q2[1], q2[2]) and np.array_equal(k2[:, P + 1], k2[:, P + 2])
+    # chain tree: the rows it writes are those of a plain causal decode at positions P, P+1, ...
+    chain_depth = np.arange(M)
+    qc, kcc, _ = orc.verify_qkv_append(x, wq, wk, wv, chain_depth, kc, vc, P, Hq, Hkv, 77.0)
+    for i in range(M):
+        raw = (wk @ x[i]).reshape(Hkv, d)
+        assert np.allclose(kcc[0, P + i], orc.rope(raw[0], P + i, 77.0), atol=1e-12)
+
+
+def test_gather_accepted_rows():
+    hidden = np.arange(24.0).reshape(6, 4)
+    out = orc.gather_accepted(hidden, [2, 5], rows=5)
+    assert np.array_equal(out[0], hidden[0]) and np.array_equal(out[1], hidden[2])
+    assert np.array_equal(out[2], hidden[5]) and np.all(out[3:] == 0)
+    assert np.array_equal(orc.gather_accepted(hidden, [], rows=3)[1:], np.zeros((2, 4)))
