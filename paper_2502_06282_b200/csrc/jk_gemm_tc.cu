@@ -545,7 +545,10 @@ size_t jk_tc_partial_bytes(const jk_config& c) {
   const int kt_2h = (2 * c.hidden + TC_TILE_K - 1) / TC_TILE_K, kt_q = (qd + TC_TILE_K - 1) / TC_TILE_K;
   const long long t_qkv = (qkvd + TC_TILE_M - 1) / TC_TILE_M;
   size_t e1 = tc_partial_for(t_h * kt_2h, kt_2h, np1);
-  size_t e2 = tc_partial_for(t_qkv * kt_h, kt_h, np1);
+  // (jk_verify_qkv sends up to 256 tree tokens at a time through the QKV projection)
+  int np_v = (int)jk_align_up((size_t)c.max_batch * c.max_tree, 16);
+  if (np_v > 256) np_v = 256;
+  size_t e2 = tc_partial_for(t_qkv * kt_h, kt_h, np_v > np1 ? np_v : np1);
   size_t e3 = tc_partial_for(t_h * kt_q, kt_q, np1);
   size_t m = a > b ? a : b;
   m = m > d ? m : d;
