@@ -560,6 +560,59 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
             "call_frac_tensor": round(tf / peaks["bf16_tflops"], 4),
             "flop_per_byte": round(intensity, 1), "ridge_flop_per_byte": round(ridge, 1),
             "bound": "tensor" if intensity > ridge else "hbm"})
+    # The three phases of a step, each replayed as a CUDA graph of its own (no event nodes: the
+    # kernels of a phase overlap their neighbours' tails as they do in the whole step)
+    def phase_ms(fn):
+        cs = torch.cuda.Stream()
+        cs.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cs):
+            fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cs):
+            fn()
+        g.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(5):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(10):
+                g.replay()
+            b_.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b_) / 10)
+        return float(np.median(ts))
+
+    def attn_phase():
+        for l in range(L):
+            ctx.tree_verify_attn(w.batch, w.tree_size, inA["q_all"][l], ks[l], vs[l], kv_len,
+                                 bufs.tree["parent"], scale, outs[l])
+
+    def accept_phase():
+        kv_len.copy_(kv_len0)
+        ctx.accept_and_compact(w.batch, w.tree_size, mode, 1.0, inA["tl"], bufs.tree,
+                               bufs.logits if mode else None, bufs.n_slots,
+                               inA["ua"] if mode else None, inA["ub"] if mode else None, L, kp, vp,
+                               ks[0].stride(0), ks[0].stride(1), ks[0].shape[2], kv_len,
+                               bufs.n_acc, bufs.acc_idx, bufs.acc_tok, bufs.bonus)
+
+    phases = None
+    if graph is not None:
+        try:
+            phases = {"draft_ms": round(phase_ms(lambda: draft(inA)), 4),
+                      "verify_attn_ms": round(phase_ms(attn_phase), 4),
+                      "accept_ms": round(phase_ms(accept_phase), 4)}
+            phases["attn_call_us"] = round(1000.0 * phases["verify_attn_ms"] / L, 2)
+            a_gb = L * attn_bytes / (phases["verify_attn_ms"] * 1e-3) / 1e9
+            a_tf = L * attn_flops / (phases["verify_attn_ms"] * 1e-3) / 1e12
+            phases["attn_frac_hbm"] = round(a_gb / peak, 4)
+            phases["attn_frac_hbm_nominal_8000"] = round(a_gb / NOMINAL_HBM_GBS, 4)
+            phases["attn_frac_tensor"] = round(a_tf / peaks["bf16_tflops"], 4)
+            phases["attn_bound"] = ("tensor" if attn_flops / attn_bytes > peaks["bf16_tflops"] * 1e3 / peak
+                                    else "hbm")
+        except Exception as exc:
+            phases = {"unavailable": str(exc)}
     groups = {}
     def gsum(names):
         return round(sum(kernels[n]["ms_per_step"] for n in names if n in kernels), 4)
@@ -577,6 +630,11 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     step_bytes = draft_bytes + algo_bytes_per_step["tree_attn"] + w.batch * w.tree_size * V * 4
     groups["step_algo_GB"] = round(step_bytes / 1e9, 3)
     groups["step_frac_of_peak"] = round(step_bytes / (ms_per_step * 1e-3) / 1e9 / peak, 4)
+    groups["note"] = "sums of the event-bracketed kernel times below (serialised: they exceed the step)"
+    if phases and "draft_ms" in phases:
+        phases["draft_frac_of_peak"] = round(draft_bytes / (phases["draft_ms"] * 1e-3) / 1e9 / peak, 4)
+        phases["draft_frac_of_nominal_8000"] = round(draft_bytes / (phases["draft_ms"] * 1e-3) / 1e9
+                                                     / NOMINAL_HBM_GBS, 4)
     dom = max((k for k in kernels if "GBps" in kernels[k]), key=lambda k: kernels[k]["ms_per_step"])
     ratio, ratio_src = captured_gate_up_traffic_ratio()
     per_launch_bytes = algo_bytes_per_step[dom] / kernels[dom]["launches_per_step"]
@@ -677,7 +735,7 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
                    [round(min(pass_ms), 3), round(ms, 3), round(max(pass_ms), 3)],
                "tree_tokens_per_s": value * w.batch * w.tree_size,
                "accepted_per_step": n_acc, "clocks": clocks, "e2e": e2e,
-               "gpu_launches": gpu_launches, "roofline": roofline, "groups": groups,
+               "gpu_launches": gpu_launches, "roofline": roofline, "phases": phases, "groups": groups,
                "kernels": kernels, "cpu_baseline": cpu_baseline}
     del graph
     return out
