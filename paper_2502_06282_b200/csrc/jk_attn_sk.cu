@@ -11,13 +11,16 @@
 // Inside the CTA the roles are split across warps and every stage is double-buffered, so that the
 // copy of tile i+1, the S product of tile i+1 and the softmax of tile i run at the same time:
 //   warp 0      TMA producer (K and V tiles, two buffers each)
-//   warp 1      MMA issuer (S = Q K^T into one of two tensor-memory buffers, then O += P V with V
-//               taken MN-major straight from its row-major tile)
-//   warps 2-9   softmax: two threads per query row, each owning 64 of the tile's 128 keys; they
-//               apply the tree mask (a visibility word built from the node's ancestor set and the
-//               prefix length), keep a running max and sum, rescale O in tensor memory when the
-//               max moved and write P = exp(S - max) as bf16 for the second product.
-// 192 KB of shared memory and 512 tensor-memory columns per CTA.  All waits are bounded mbarrier
+//   warp 1      MMA issuer (S = Q K^T into one of two tensor-memory buffers, then O += P V with P
+//               taken from tensor memory as the A operand and V MN-major straight from its
+//               row-major tile)
+//   warps 2-9   softmax: two threads per query row, each owning 64 of the tile's 128 keys; one
+//               read of S into registers, the tree mask (a visibility word built from the node's
+//               ancestor set and the prefix length), the halves' maxima exchanged through shared
+//               memory, P = exp(S - max) packed to bf16 and stored over S in tensor memory.  The
+//               reference maximum only moves when it is outgrown by more than 2^8, so O is rarely
+//               rescaled and the softmax of a tile seldom has to wait for the tile before it.
+// 160 KB of shared memory and 512 tensor-memory columns per CTA.  All waits are bounded mbarrier
 // waits (no named barriers), so a role that gives up cannot leave another one waiting for ever.
 #include <math.h>
 #include <stdlib.h>
@@ -32,8 +35,8 @@
 #define ASK_MAX_UNITS_X_CTAS 0x7fffffffu   // unit index * CTA count stays in 32 bits
 
 struct ask_tail {
-  uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2], s_empty[2];
-  uint64_t p_full, pv_done, q_full, par_full, o_ready;
+  uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2];
+  uint64_t p_full[2], pv_done, q_full, par_full, o_ready;
   uint64_t pair[4];                  // the two threads of a row meet here (64 arrivals)
   uint32_t tmem_base;
   int abort_flag;
@@ -118,7 +121,6 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
   constexpr int KB = D / 64;
   constexpr int Q_BYTES = ASK_ROWS * D * 2;
   constexpr int KV_BYTES = ASK_KEYS * D * 2;
-  constexpr int P_BYTES = ASK_ROWS * ASK_KEYS * 2;
   constexpr uint32_t TMEM_COLS = 512;
   constexpr uint32_t O_COL = 256;
   extern __shared__ unsigned char smem_raw[];
@@ -126,8 +128,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
   unsigned char* sq = smem;
   unsigned char* sk = sq + Q_BYTES;
   unsigned char* sv = sk + 2 * KV_BYTES;
-  unsigned char* sp = sv + 2 * KV_BYTES;
-  ask_tail& T = *reinterpret_cast<ask_tail*>(sp + P_BYTES);
+  ask_tail& T = *reinterpret_cast<ask_tail*>(sv + 2 * KV_BYTES);
   volatile int* abort_flag = &T.abort_flag;
 
   const int G = Hq / Hkv;
@@ -140,9 +141,9 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
     for (int i = 0; i < 2; ++i) {
       mbar_init(&T.k_full[i], 1); mbar_init(&T.v_full[i], 1);
       mbar_init(&T.k_empty[i], 1); mbar_init(&T.v_empty[i], 1);
-      mbar_init(&T.s_full[i], 1); mbar_init(&T.s_empty[i], ASK_SM_THREADS);
+      mbar_init(&T.s_full[i], 1);
     }
-    mbar_init(&T.p_full, ASK_SM_THREADS);
+    mbar_init(&T.p_full[0], ASK_SM_THREADS); mbar_init(&T.p_full[1], ASK_SM_THREADS);
     mbar_init(&T.pv_done, 1);
     mbar_init(&T.o_ready, 1);
     mbar_init(&T.q_full, ASK_SM_THREADS);
@@ -226,17 +227,21 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
     if (lane == 0) {
       const uint32_t idesc_s = instr_desc_bf16_ex(ASK_KEYS, 0);
       const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
-      const uint32_t qa = smem_u32(sq), pa = smem_u32(sp);
+      const uint32_t qa = smem_u32(sq);
+      // The S buffer of tile g holds P of tile g until the P V product of tile g has read it, so
+      // S of tile g+2 (same buffer) is issued only once that product has completed.  Its
+      // completion is what v_empty of the same parity signals (the tensor core gives no ordering
+      // between a product's operand reads from tensor memory and a later product's writes there).
       auto s_ready = [&](int g) -> bool {
         const int bf = g & 1;
         const uint32_t ph = (uint32_t)(g >> 1) & 1u;
-        return mbar_try_wait(&T.k_full[bf], ph) && (g < 2 || mbar_try_wait(&T.s_empty[bf], ph ^ 1u));
+        return mbar_try_wait(&T.k_full[bf], ph) && (g < 2 || mbar_try_wait(&T.v_empty[bf], ph ^ 1u));
       };
       auto issue_s = [&](int g) -> bool {
         const int bf = g & 1;
         const uint32_t ph = (uint32_t)(g >> 1) & 1u;
         if (!mbar_wait(&T.k_full[bf], ph, abort_flag, status)) return false;
-        if (g >= 2 && !mbar_wait(&T.s_empty[bf], ph ^ 1u, abort_flag, status)) return false;
+        if (g >= 2 && !mbar_wait(&T.v_empty[bf], ph ^ 1u, abort_flag, status)) return false;
         tc_fence_after();
         const uint32_t ka = smem_u32(sk + bf * KV_BYTES);
 #pragma unroll
@@ -259,16 +264,16 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
           // S of the next tile goes first if its K tile is already there, else after P V
           bool ahead = false;
           if (t + 1 < s.tile_hi && s_ready(g + 1)) { ok = issue_s(g + 1); ahead = true; }
-          ok = ok && mbar_wait(&T.p_full, (uint32_t)g & 1u, abort_flag, status);
+          ok = ok && mbar_wait(&T.p_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
           ok = ok && mbar_wait(&T.v_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t va = smem_u32(sv + bf * KV_BYTES);
 #pragma unroll
           for (int j = 0; j < ASK_KEYS / 16; ++j)
-            tc_mma_bf16(tmem_base + O_COL, smem_desc_sw128(pa + (j >> 2) * 16384 + (j & 3) * 32),
-                        smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
-                        (t > s.tile_lo || j > 0) ? 1u : 0u);
+            tc_mma_bf16_ts(tmem_base + O_COL, tmem_base + (uint32_t)bf * 128u + (uint32_t)(j * 8),
+                           smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
+                           (t > s.tile_lo || j > 0) ? 1u : 0u);
           tc_commit(&T.v_empty[bf]);
           tc_commit(&T.pv_done);
           if (t + 1 < s.tile_hi && !ahead) ok = issue_s(g + 1);
@@ -287,7 +292,6 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
     const int sm_tid = tid - 64;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const float sl2 = scale * 1.4426950408889634f;
-    unsigned char* prow = sp + half * 16384 + row * 128;
     constexpr int QV = D / 16;                       // 16-byte vectors of half a query row
     int g = 0, seg = 0;
     uint32_t pair_uses = 0;
@@ -371,10 +375,10 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = tmem_base + lane_base + (uint32_t)bf * 128u + (uint32_t)half * 64u;
-        // pass 1: maximum of the visible scores of this half; the row maximum via the partner
+        // this thread's half row of S, read once; the row maximum via the partner
+        uint32_t r0[32], r1[32];
         float mx = -INFINITY;
         if (warp_active) {
-          uint32_t r0[32], r1[32];
           tmem_ld32(sa, r0);
           tmem_ld32(sa + 32u, r1);
           tmem_ld_wait();
@@ -385,19 +389,48 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
           }
         }
         T.xmax[bf][half][row] = mx;
-        ok = pair_sync();
+        tc_fence_before();
+        ok = pair_sync();                  // both halves have S in registers: P may overwrite it
         if (!ok) break;
-        const float m_new = fmaxf(m_run, fmaxf(mx, T.xmax[bf][half ^ 1][row]));
-        const float alpha = (m_run == -INFINITY) ? ((m_new == -INFINITY) ? 1.f : 0.f)
-                                                 : fast_exp2((m_run - m_new) * sl2);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        if (tile > s.tile_lo) {
-          // P and O are free once the previous tile's P V product has completed
+        tc_fence_after();
+        mx = fmaxf(mx, T.xmax[bf][half ^ 1][row]);
+        // The reference maximum moves only when the row maximum outgrows it by more than 2^8.
+        float alpha = 1.f;
+        if (mx != -INFINITY && (m_run == -INFINITY || (mx - m_run) * sl2 > 8.f)) {
+          alpha = (m_run == -INFINITY) ? 0.f : fast_exp2((m_run - mx) * sl2);
+          m_run = mx;
+        }
+        const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+        // P = exp(S - max) as bf16, two keys per 32-bit column, back into tensor memory over S
+        float lsum = 0.f;
+        if (warp_active) {
+          uint32_t pk[32];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = ((b0 >> j) & 1u) ? fast_exp2((__uint_as_float(r0[j]) - m_use) * sl2) : 0.f;
+            const float p1 = ((b0 >> (j + 1)) & 1u)
+                                 ? fast_exp2((__uint_as_float(r0[j + 1]) - m_use) * sl2) : 0.f;
+            const float p2 = ((b1 >> j) & 1u) ? fast_exp2((__uint_as_float(r1[j]) - m_use) * sl2) : 0.f;
+            const float p3 = ((b1 >> (j + 1)) & 1u)
+                                 ? fast_exp2((__uint_as_float(r1[j + 1]) - m_use) * sl2) : 0.f;
+            const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+            const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+            // the sum runs over the rounded values the second product will use
+            lsum += (__low2float(h01) + __high2float(h01)) + (__low2float(h23) + __high2float(h23));
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+            pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+          }
+          tmem_st32(tmem_base + lane_base + (uint32_t)bf * 128u + (uint32_t)half * 32u, pk);
+        }
+        // O is rescaled only when some row of the warp moved its reference, and only then does
+        // the softmax have to wait for the previous tile's P V product (both warps of a row pair
+        // see the same rows and take the same decision)
+        if (tile > s.tile_lo && __any_sync(0xffffffffu, alpha != 1.f)) {
           const bool okp = mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
           ok = __all_sync(0xffffffffu, okp);
           if (!ok) break;
           tc_fence_after();
-          if (warp_active && __any_sync(0xffffffffu, alpha != 1.f)) {
+          if (warp_active) {
 #pragma unroll 1
             for (int c = 0; c < D / 64; ++c) {
               uint32_t r[32];
@@ -408,38 +441,10 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
               for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
               tmem_st32(oa, r);
             }
-            tmem_st_wait();
           }
         }
-        // pass 2: P = exp(S - max) as bf16, 32 keys at a time, read again from tensor memory
-        float lsum = 0.f;
-        if (warp_active) {
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            uint32_t r[32];
-            tmem_ld32(sa + (uint32_t)(hh * 32), r);
-            tmem_ld_wait();
-            const unsigned bits = hh ? b1 : b0;
-            uint32_t pk[16];
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              const float p0 = ((bits >> j) & 1u) ? fast_exp2((__uint_as_float(r[j]) - m_use) * sl2) : 0.f;
-              const float p1 = ((bits >> (j + 1)) & 1u)
-                                   ? fast_exp2((__uint_as_float(r[j + 1]) - m_use) * sl2) : 0.f;
-              lsum += p0 + p1;
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-              pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-              const int cb = hh * 4 + cc;
-              *reinterpret_cast<uint4*>(prow + ((cb ^ (row & 7)) << 4)) =
-                  make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-            }
-          }
-        }
+        if (warp_active) tmem_st_wait();
         l_run = l_run * alpha + lsum;
-        m_run = m_new;
         // Cache rows past the last live key (only a sequence's last tile has any) may hold
         // anything, NaN bit patterns included, and 0 * NaN would poison every output row: they
         // are cleared in the V tile before the second product reads it.
@@ -458,8 +463,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         }
         fence_proxy_async_smem();
         tc_fence_before();
-        mbar_arrive(&T.s_empty[bf]);
-        mbar_arrive(&T.p_full);
+        mbar_arrive(&T.p_full[bf]);
       }
       if (!ok) break;
       // ---- the segment's partial (max, sum, O) of every row
@@ -634,8 +638,7 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024));
     ctx->attn_sk_smem_set = 1;
   }
-  const size_t smem = (size_t)ASK_ROWS * D * 2 + 4 * (size_t)ASK_KEYS * D * 2 +
-                      (size_t)ASK_ROWS * ASK_KEYS * 2 + sizeof(ask_tail) + 1024;
+  const size_t smem = (size_t)ASK_ROWS * D * 2 + 4 * (size_t)ASK_KEYS * D * 2 + sizeof(ask_tail) + 1024;
   const int n_cta = ctx->sm_count;
   const int ms = L.attn_max_split;
   const int min_units = 1;
