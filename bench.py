@@ -600,9 +600,11 @@ def run_workload(args, name, rank, world, torch, dist, jk, synth, replicas):
     phases = None
     if graph is not None:
         try:
-            phases = {"draft_ms": round(phase_ms(lambda: draft(inA)), 4),
-                      "verify_attn_ms": round(phase_ms(attn_phase), 4),
-                      "accept_ms": round(phase_ms(accept_phase), 4)}
+            phases = {"draft_ms": round(phase_ms(lambda: draft(inA)), 4)}
+            kv_len.copy_(kv_len0)        # the last step's acceptance moved it; attention reads it only
+            phases["verify_attn_ms"] = round(phase_ms(attn_phase), 4)
+            phases["accept_ms"] = round(phase_ms(accept_phase), 4)
+            assert ctx.read_status() == 0, "device status word reports an error in a phase"
             phases["attn_call_us"] = round(1000.0 * phases["verify_attn_ms"] / L, 2)
             a_gb = L * attn_bytes / (phases["verify_attn_ms"] * 1e-3) / 1e9
             a_tf = L * attn_flops / (phases["verify_attn_ms"] * 1e-3) / 1e12

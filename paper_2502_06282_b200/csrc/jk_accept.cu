@@ -8,7 +8,9 @@
 
 // ------------------------------------------------------------------------------------------
 // Row statistics: top-1 token (ties: lower id), max and sum exp((x - max)/T).  One block per
-// tree node.
+// row, one pass over it: every thread keeps a running (max, argmax, sum relative to that max)
+// over batches of vectors that are all requested before the first one is used, and the block
+// brings the partial sums onto the row maximum at the end.
 // ------------------------------------------------------------------------------------------
 template <typename TL>
 __device__ __forceinline__ void row_stats_row(const TL* __restrict__ r, size_t row, int V,
@@ -17,20 +19,54 @@ __device__ __forceinline__ void row_stats_row(const TL* __restrict__ r, size_t r
                                               float* __restrict__ rs_sum, float* red, float* wv,
                                               int* wi) {
   constexpr int VN = jk_vec<TL>::N;
-  float bv = -INFINITY;
+  constexpr int U = 32 / VN;                       // vectors in flight per thread (32 values)
+  float bv = -INFINITY, s = 0.f;
   int bi = INT_MAX;
   const int vmain = V / VN * VN;
-  for (int k = threadIdx.x * VN; k < vmain; k += blockDim.x * VN) {
-    float v[VN];
-    jk_vec<TL>::load(r + k, v);
+  const int step = blockDim.x * VN;
+  for (int k0 = threadIdx.x * VN; k0 < vmain; k0 += step * U) {
+    float v[U][VN];
 #pragma unroll
-    for (int i = 0; i < VN; ++i)
-      if (jk_better(v[i], k + i, bv, bi)) { bv = v[i]; bi = k + i; }
+    for (int u = 0; u < U; ++u) {
+      const int k = k0 + u * step;
+      if (k < vmain) {
+        jk_vec<TL>::load(r + k, v[u]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < VN; ++i) v[u][i] = -INFINITY;
+      }
+    }
+    float cv = bv;
+    int ci = bi;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int k = k0 + u * step;
+      if (k < vmain) {                             // the padding takes no part in the argmax
+#pragma unroll
+        for (int i = 0; i < VN; ++i)
+          if (jk_better(v[u][i], k + i, cv, ci)) { cv = v[u][i]; ci = k + i; }
+      }
+    }
+    if (cv > bv) s *= expf((bv - cv) * inv_t);     // bv = -inf: s is 0 and stays 0
+    bv = cv;
+    bi = ci;
+    if (bv > -INFINITY) {
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int i = 0; i < VN; ++i) s += expf((v[u][i] - bv) * inv_t);
+    }
   }
   for (int k = vmain + threadIdx.x; k < V; k += blockDim.x) {
     const float v = jk_to_float(r[k]);
-    if (jk_better(v, k, bv, bi)) { bv = v; bi = k; }
+    if (jk_better(v, k, bv, bi)) {
+      if (v > bv) s *= expf((bv - v) * inv_t);
+      bv = v;
+      bi = k;
+    }
+    if (bv > -INFINITY) s += expf((v - bv) * inv_t);
   }
+  const float own = bv;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
@@ -44,15 +80,7 @@ __device__ __forceinline__ void row_stats_row(const TL* __restrict__ r, size_t r
   int am = wi[0];
   for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
     if (jk_better(wv[w], wi[w], mx, am)) { mx = wv[w]; am = wi[w]; }
-  float s = 0.f;
-  for (int k = threadIdx.x * VN; k < vmain; k += blockDim.x * VN) {
-    float v[VN];
-    jk_vec<TL>::load(r + k, v);
-#pragma unroll
-    for (int i = 0; i < VN; ++i) s += expf((v[i] - mx) * inv_t);
-  }
-  for (int k = vmain + threadIdx.x; k < V; k += blockDim.x)
-    s += expf((jk_to_float(r[k]) - mx) * inv_t);
+  s = own > -INFINITY ? s * expf((own - mx) * inv_t) : 0.f;
   s = jk_block_sum(s, red);
   if (threadIdx.x == 0) { rs_arg[row] = am; rs_max[row] = mx; rs_sum[row] = s; }
 }
@@ -158,7 +186,6 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
   __shared__ int n_kids;
   __shared__ int path[16], path_tok[16];
   __shared__ int s_decision;
-  __shared__ float scan_s[1024];
   __shared__ int s_found;
   const int b = blockIdx.x, t = threadIdx.x, nt = blockDim.x;
   const int lane = t & 31, warp = t >> 5, nw = nt >> 5;
@@ -318,22 +345,41 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
       const walk_vec4 pv = p_at4(v);
       loc += (pv.v[0] + pv.v[1]) + (pv.v[2] + pv.v[3]);
     }
-    scan_s[t] = loc;
-    if (t == 0) s_found = INT_MAX;
-    __syncthreads();
-    for (int off = 1; off < nt; off <<= 1) {
-      const float add = t >= off ? scan_s[t - off] : 0.f;
-      __syncthreads();
-      scan_s[t] += add;
-      __syncthreads();
+    // inclusive scan of the runs' sums: shuffles inside a warp, the 32 warp totals by warp 0
+    float incl = loc;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const float y = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += y;
     }
-    const float total = scan_s[nt - 1];
+    if (t == 0) s_found = INT_MAX;
+    __syncthreads();                       // red[] is free (the last block sum has been read)
+    if (lane == 31) red[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const float w = lane < nw ? red[lane] : 0.f;
+      float wi = w;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const float y = __shfl_up_sync(0xffffffffu, wi, off);
+        if (lane >= off) wi += y;
+      }
+      red[33 + lane] = wi - w;             // what lies before this warp
+      if (lane == 31) red[32] = wi;
+    }
+    __syncthreads();
+    incl += red[33 + warp];
+    const float total = red[32];
     const float thr = ub * total;
-    const float before = scan_s[t] - loc;
-    // The crossing lies in this thread's run (the scan is non-decreasing, so the test picks the
-    // first run whose end passes the threshold; several can pass it only when later runs are
-    // empty, and atomicMin keeps the first).
-    const bool mine = before <= thr && scan_s[t] > thr;
+    // `before` is exactly the previous thread's inclusive value, so the runs' intervals
+    // [before, incl) join without gaps and some run claims every threshold below the total.
+    if (lane == 31) red[warp] = incl;
+    __syncthreads();
+    const float up = __shfl_up_sync(0xffffffffu, incl, 1);
+    const float before = lane ? up : (warp ? red[warp - 1] : 0.f);
+    // The crossing lies in this thread's run; rounding can let more than one run claim the
+    // threshold (the scan need not be monotone to the last bit) and atomicMin keeps the first.
+    const bool mine = before <= thr && incl > thr;
     if (mine) {
       float run = before;
       int last_pos = -1;

@@ -61,13 +61,17 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->gemm_part = take(L->gemm_part_bytes);
   // split-KV partials, capped at 256 MiB
   const size_t pre_nodes = (size_t)c.max_batch * c.max_depth * c.max_frontier;
-  const size_t rows = (BM > pre_nodes ? BM : pre_nodes) * c.n_q_heads;
-  const size_t per_split = rows * (c.head_dim + 2) * 4;
+  size_t rows = (BM > pre_nodes ? BM : pre_nodes) * c.n_q_heads;
+  // the persistent kernel keeps its partials per 128-row query block, dead rows included
+  const size_t grp = (size_t)(c.n_q_heads / c.n_kv_heads) * c.max_tree;
+  const size_t rows_blk = (size_t)c.max_batch * c.n_kv_heads * ((grp + 127) / 128) * 128;
+  if (rows_blk > rows) rows = rows_blk;
+  const size_t per_split = rows * (c.head_dim + 4) * 4;
   int ms = JK_ATTN_MAX_SPLIT;
   while (ms > 1 && per_split * ms > ((size_t)256 << 20)) --ms;
   L->attn_max_split = ms;
   L->attn_o = take(rows * c.head_dim * 4 * ms);
-  L->attn_ml = take(rows * 2 * 4 * ms);
+  L->attn_ml = take(rows * 4 * 4 * ms);
   L->rs_arg = take(BM * 4);
   L->rs_max = take(BM * 4);
   L->rs_sum = take(BM * 4);

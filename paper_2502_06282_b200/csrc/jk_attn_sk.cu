@@ -8,20 +8,28 @@
 // spread over several CTAs gets one unnormalised partial (max, sum, O) per CTA, numbered from the
 // first CTA that touches it, and the merge kernel below combines them.
 //
-// Inside the CTA the roles are split across warps and every stage is double-buffered, so that the
-// copy of tile i+1, the S product of tile i+1 and the softmax of tile i run at the same time:
-//   warp 0      TMA producer (K and V tiles, two buffers each)
-//   warp 1      MMA issuer (S = Q K^T into one of two tensor-memory buffers, then O += P V with P
-//               taken from tensor memory as the A operand and V MN-major straight from its
-//               row-major tile)
+// Inside the CTA the roles are split across warps and every stage is buffered at least twice, so
+// that the copy of tile i+2, the S product of tile i+1 and the softmax of tile i run at the same
+// time:
+//   warp 0      TMA producer (a ring of three K tiles and one of two or three V tiles)
+//   warp 1      MMA issuer: S = Q K^T into one of three tensor-memory buffers, then O += P V with
+//               P taken from tensor memory as the A operand and V MN-major straight from its
+//               row-major tile.  It polls for whichever of "next S" and "this P V" has its inputs
+//               first, without parking on either.
 //   warps 2-9   softmax: two threads per query row, each owning 64 of the tile's 128 keys; one
 //               read of S into registers, the tree mask (a visibility word built from the node's
-//               ancestor set and the prefix length), the halves' maxima exchanged through shared
-//               memory, P = exp(S - max) packed to bf16 and stored over S in tensor memory.  The
-//               reference maximum only moves when it is outgrown by more than 2^8, so O is rarely
-//               rescaled and the softmax of a tile seldom has to wait for the tile before it.
-// 160 KB of shared memory and 512 tensor-memory columns per CTA.  All waits are bounded mbarrier
-// waits (no named barriers), so a role that gives up cannot leave another one waiting for ever.
+//               ancestor set and the prefix length; a tile inside the prefix takes a path without
+//               any masking, chosen per warp), the halves' maxima exchanged through shared
+//               memory, P = exp2(S * c - max * c) packed to bf16 and stored over S in tensor
+//               memory.  The reference maximum only moves when it is outgrown by more than 2^8, so
+//               O is rarely rescaled and the softmax of a tile seldom has to wait for the tile
+//               before it.  At a segment's end they request the next segment's query rows, stage
+//               them as soon as the last product has completed, and only then store the partial,
+//               laid out [slice][query block][16-byte piece][row] so that a warp's 32 rows write
+//               512 contiguous bytes per instruction.
+// 190 to 220 KB of shared memory and 512 tensor-memory columns per CTA.  All waits are bounded
+// mbarrier waits (no named barriers), so a role that gives up cannot leave another one waiting
+// for ever.
 #include <math.h>
 #include <stdlib.h>
 
@@ -32,11 +40,14 @@
 #define ASK_KEYS 128
 #define ASK_THREADS 320
 #define ASK_SM_THREADS 256
+#define ASK_NK 3                    // K tiles in the ring
+#define ASK_NV_MAX 3                // V tiles in the ring: 3 with a 64-row Q tile, else 2
+#define ASK_NS 3                    // S / P buffers in tensor memory (128 columns each)
 #define ASK_MAX_UNITS_X_CTAS 0x7fffffffu   // unit index * CTA count stays in 32 bits
 
 struct ask_tail {
-  uint64_t k_full[2], v_full[2], k_empty[2], v_empty[2], s_full[2];
-  uint64_t p_full[2], pv_done, q_full, par_full, o_ready;
+  uint64_t k_full[ASK_NK], v_full[ASK_NV_MAX], k_empty[ASK_NK], v_empty[ASK_NV_MAX], s_full[ASK_NS];
+  uint64_t p_full[ASK_NS], p_free[ASK_NS], q_full, par_full, o_ready;
   uint64_t pair[4];                  // the two threads of a row meet here (64 arrivals)
   uint32_t tmem_base;
   int abort_flag;
@@ -44,8 +55,7 @@ struct ask_tail {
   int parent[JK_MAX_TREE];
   int tiles[JK_MAX_ROWS];            // key tiles of every sequence
   int plen[JK_MAX_ROWS];             // prefix length of every sequence
-  float xmax[2][2][ASK_ROWS];        // [tile parity][key half][row]: tile maximum of that half
-  float xsum[2][ASK_ROWS];
+  float xmax[ASK_NS][2][ASK_ROWS];   // [S buffer][key half][row]: tile maximum of that half
 };
 
 struct ask_plan {
@@ -111,7 +121,10 @@ __device__ __forceinline__ ask_seg ask_segment(const int* tiles, int B, int item
   return s;
 }
 
-template <int D>
+// QR = rows of the Q tile kept in shared memory: 64 when a query block has at most 64 live rows
+// (the product still spans 128 rows; rows 64..127 then read whatever follows the Q tile, and their
+// results, which no one reads, stay in their own rows), which leaves room for a third V tile.
+template <int D, int QR>
 __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
     const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
     const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ kv_len,
@@ -119,16 +132,19 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
     int min_units, int cache_rows, float* __restrict__ part_o, float* __restrict__ part_ml,
     int32_t* status) {
   constexpr int KB = D / 64;
-  constexpr int Q_BYTES = ASK_ROWS * D * 2;
+  constexpr int ASK_NV = QR == 64 ? 3 : 2;
+  constexpr int Q_BYTES = QR * D * 2;
+  constexpr int Q_KB = QR * 128;                   // bytes of one 64-column block of the Q tile
   constexpr int KV_BYTES = ASK_KEYS * D * 2;
   constexpr uint32_t TMEM_COLS = 512;
-  constexpr uint32_t O_COL = 256;
+  constexpr uint32_t O_COL = ASK_NS * 128;
+  static_assert(O_COL + D <= TMEM_COLS, "S buffers and O must fit the tensor memory of an SM");
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* sq = smem;
   unsigned char* sk = sq + Q_BYTES;
-  unsigned char* sv = sk + 2 * KV_BYTES;
-  ask_tail& T = *reinterpret_cast<ask_tail*>(sv + 2 * KV_BYTES);
+  unsigned char* sv = sk + ASK_NK * KV_BYTES;
+  ask_tail& T = *reinterpret_cast<ask_tail*>(sv + ASK_NV * KV_BYTES);
   volatile int* abort_flag = &T.abort_flag;
 
   const int G = Hq / Hkv;
@@ -138,13 +154,12 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
   const int items_per_b = Hkv * n_qblk;
   const size_t n_out = (size_t)B * M * Hq;
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&T.k_full[i], 1); mbar_init(&T.v_full[i], 1);
-      mbar_init(&T.k_empty[i], 1); mbar_init(&T.v_empty[i], 1);
-      mbar_init(&T.s_full[i], 1);
+    for (int i = 0; i < ASK_NK; ++i) { mbar_init(&T.k_full[i], 1); mbar_init(&T.k_empty[i], 1); }
+    for (int i = 0; i < ASK_NV; ++i) { mbar_init(&T.v_full[i], 1); mbar_init(&T.v_empty[i], 1); }
+    for (int i = 0; i < ASK_NS; ++i) {
+      mbar_init(&T.s_full[i], 1); mbar_init(&T.p_free[i], 1);
+      mbar_init(&T.p_full[i], ASK_SM_THREADS);
     }
-    mbar_init(&T.p_full[0], ASK_SM_THREADS); mbar_init(&T.p_full[1], ASK_SM_THREADS);
-    mbar_init(&T.pv_done, 1);
     mbar_init(&T.o_ready, 1);
     mbar_init(&T.q_full, ASK_SM_THREADS);
     mbar_init(&T.par_full, ASK_SM_THREADS);
@@ -184,16 +199,16 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    // K runs one tile ahead of V: the K buffer of tile g is free as soon as S of tile g-2 has
-    // completed, the V buffer only after the second product of tile g-2.
+    // K runs one tile ahead of V: the K buffer of tile g is free as soon as S of tile g - ASK_NK
+    // has completed, the V buffer only after the second product of tile g - ASK_NV.
     if (lane == 0) {
       const uint64_t pol = l2_policy_evict_first();   // the cache is read once per call
       int g = 0;
       int pt = 0, pkvh = 0, pb = 0;                 // coordinates of tile g-1 (its V is still due)
       auto load_v = [&](int gv, int t, int kvh, int b) -> bool {
-        const int bf = gv & 1;
-        if (gv >= 2 &&
-            !mbar_wait(&T.v_empty[bf], (uint32_t)((gv >> 1) - 1) & 1u, abort_flag, status))
+        const int bf = gv % ASK_NV;
+        if (gv >= ASK_NV &&
+            !mbar_wait(&T.v_empty[bf], (uint32_t)(gv / ASK_NV - 1) & 1u, abort_flag, status))
           return false;
         mbar_expect_tx(&T.v_full[bf], KV_BYTES);
 #pragma unroll
@@ -205,9 +220,9 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
       for (uint32_t x = x0; x < x1 && ok;) {
         const ask_seg s = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
         for (int t = s.tile_lo; t < s.tile_hi; ++t, ++g) {
-          const int bf = g & 1;
-          if (g >= 2)
-            ok = mbar_wait(&T.k_empty[bf], (uint32_t)((g >> 1) - 1) & 1u, abort_flag, status);
+          const int bf = g % ASK_NK;
+          if (g >= ASK_NK)
+            ok = mbar_wait(&T.k_empty[bf], (uint32_t)(g / ASK_NK - 1) & 1u, abort_flag, status);
           if (!ok) break;
           mbar_expect_tx(&T.k_full[bf], KV_BYTES);
 #pragma unroll
@@ -229,29 +244,30 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
       const uint32_t idesc_pv = instr_desc_bf16_ex(D, 1);
       const uint32_t qa = smem_u32(sq);
       // The S buffer of tile g holds P of tile g until the P V product of tile g has read it, so
-      // S of tile g+2 (same buffer) is issued only once that product has completed.  Its
-      // completion is what v_empty of the same parity signals (the tensor core gives no ordering
-      // between a product's operand reads from tensor memory and a later product's writes there).
+      // S of tile g + ASK_NS (same buffer) is issued only once that product has completed, which
+      // is what p_free signals (the tensor core gives no ordering between a product's operand
+      // reads from tensor memory and a later product's writes there).
       auto s_ready = [&](int g) -> bool {
-        const int bf = g & 1;
-        const uint32_t ph = (uint32_t)(g >> 1) & 1u;
-        return mbar_try_wait(&T.k_full[bf], ph) && (g < 2 || mbar_try_wait(&T.v_empty[bf], ph ^ 1u));
+        const int bf = g % ASK_NS;
+        const uint32_t ph = (uint32_t)(g / ASK_NS) & 1u;
+        return mbar_test(&T.k_full[g % ASK_NK], (uint32_t)(g / ASK_NK) & 1u) &&
+               (g < ASK_NS || mbar_test(&T.p_free[bf], ph ^ 1u));
       };
       auto issue_s = [&](int g) -> bool {
-        const int bf = g & 1;
-        const uint32_t ph = (uint32_t)(g >> 1) & 1u;
-        if (!mbar_wait(&T.k_full[bf], ph, abort_flag, status)) return false;
-        if (g >= 2 && !mbar_wait(&T.v_empty[bf], ph ^ 1u, abort_flag, status)) return false;
+        const int bf = g % ASK_NS, kbf = g % ASK_NK;
+        const uint32_t ph = (uint32_t)(g / ASK_NS) & 1u;
+        if (!mbar_wait(&T.k_full[kbf], (uint32_t)(g / ASK_NK) & 1u, abort_flag, status)) return false;
+        if (g >= ASK_NS && !mbar_wait(&T.p_free[bf], ph ^ 1u, abort_flag, status)) return false;
         tc_fence_after();
-        const uint32_t ka = smem_u32(sk + bf * KV_BYTES);
+        const uint32_t ka = smem_u32(sk + kbf * KV_BYTES);
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            tc_mma_bf16(tmem_base + (uint32_t)bf * 128u, smem_desc_sw128(qa + kb * 16384 + k * 32),
+            tc_mma_bf16(tmem_base + (uint32_t)bf * 128u, smem_desc_sw128(qa + kb * Q_KB + k * 32),
                         smem_desc_sw128(ka + kb * 16384 + k * 32), idesc_s, (kb | k) ? 1u : 0u);
         tc_commit(&T.s_full[bf]);
-        tc_commit(&T.k_empty[bf]);
+        tc_commit(&T.k_empty[kbf]);
         return true;
       };
       int g = 0, seg = 0;
@@ -260,26 +276,52 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         ok = mbar_wait(&T.q_full, (uint32_t)seg & 1u, abort_flag, status);
         ok = ok && issue_s(g);
         for (int t = s.tile_lo; t < s.tile_hi && ok; ++t, ++g) {
-          const int bf = g & 1;
-          // S of the next tile goes first if its K tile is already there, else after P V
-          bool ahead = false;
-          if (t + 1 < s.tile_hi && s_ready(g + 1)) { ok = issue_s(g + 1); ahead = true; }
-          ok = ok && mbar_wait(&T.p_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
-          ok = ok && mbar_wait(&T.v_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t va = smem_u32(sv + bf * KV_BYTES);
+          const int bf = g % ASK_NS;
+          const int vbf = g % ASK_NV;
+          // The next kernel of the stream (the merge) may be scheduled once every CTA has reached
+          // its last tile: its launch and its prologue then pass under the tail of this kernel,
+          // while its CTAs do not sit on the SMs for long (they were measured to slow this kernel's
+          // warps when they arrive early).
+          // Two things are due, in whichever order their inputs arrive: S of the next tile (its K
+          // tile has landed and its buffer is free) and P V of this tile (P written, V landed).
+          bool s_due = t + 1 < s.tile_hi, pv_due = true;
+          const long long w0 = clock64();
+          for (unsigned it = 1; ok && (s_due || pv_due); ++it) {
+            if (s_due && s_ready(g + 1)) {
+              ok = issue_s(g + 1);
+              s_due = false;
+              continue;
+            }
+            if (pv_due && mbar_test(&T.p_full[bf], (uint32_t)(g / ASK_NS) & 1u) &&
+                mbar_test(&T.v_full[vbf], (uint32_t)(g / ASK_NV) & 1u)) {
+              tc_fence_after();
+              const uint32_t va = smem_u32(sv + vbf * KV_BYTES);
 #pragma unroll
-          for (int j = 0; j < ASK_KEYS / 16; ++j)
-            tc_mma_bf16_ts(tmem_base + O_COL, tmem_base + (uint32_t)bf * 128u + (uint32_t)(j * 8),
-                           smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
-                           (t > s.tile_lo || j > 0) ? 1u : 0u);
-          tc_commit(&T.v_empty[bf]);
-          tc_commit(&T.pv_done);
-          if (t + 1 < s.tile_hi && !ahead) ok = issue_s(g + 1);
+              for (int j = 0; j < ASK_KEYS / 16; ++j)
+                tc_mma_bf16_ts(tmem_base + O_COL, tmem_base + (uint32_t)bf * 128u + (uint32_t)(j * 8),
+                               smem_desc_mn_sw128(va + j * 2048, 16384), idesc_pv,
+                               (t > s.tile_lo || j > 0) ? 1u : 0u);
+              tc_commit(&T.v_empty[vbf]);
+              tc_commit(&T.p_free[bf]);
+              pv_due = false;
+              continue;
+            }
+            __nanosleep(40);               // leave the issue slots to the softmax warps of this quarter
+            if ((it & 255u) == 0) {
+              if (*abort_flag) ok = false;
+              else if (clock64() - w0 > TC_WAIT_CYCLES) {
+                *abort_flag = 1;
+                jk_set_status(status, JK_ERR_TIMEOUT);
+                ok = false;
+              }
+            }
+          }
         }
         // the segment's O is complete: pass that on through a barrier this thread arrives on
-        ok = ok && mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
+        // (p_free of the last tile's buffer: the phase before it completed before that tile's S
+        // was issued, so the parity cannot be mistaken for an older one)
+        ok = ok && mbar_wait(&T.p_free[(g - 1) % ASK_NS], (uint32_t)((g - 1) / ASK_NS) & 1u, abort_flag,
+                             status);
         if (ok) mbar_arrive(&T.o_ready);
         x += (uint32_t)(s.tile_hi - s.tile_lo);
       }
@@ -301,34 +343,58 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
       ++pair_uses;
       return __all_sync(0xffffffffu, o);
     };
-    for (uint32_t x = x0; x < x1; ++seg) {
-      const ask_seg s = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
-      x += (uint32_t)(s.tile_hi - s.tile_lo);
-      const int P = T.plen[s.b];
-      const int row0 = s.qblk * ASK_ROWS;
-      const bool row_valid = row0 + row < n_rows;
-      const bool warp_active = row0 + quarter * 32 < n_rows;
-      const int g_idx = row_valid ? (row0 + row) / M : 0;
-      const int node = row_valid ? (row0 + row) % M : 0;
-      const size_t orow = ((size_t)s.b * M + node) * Hq + s.kvh * G + g_idx;
-      // this segment's tree and query rows (every MMA of the previous segment has completed)
-      uint4 qv[QV];
+    // Per segment: where this thread's row lives.  The query rows and the tree of the NEXT segment
+    // are fetched while the last product of the current one drains, and staged as soon as that
+    // product has completed, so that the next segment's first S runs under this one's epilogue.
+    struct seg_row { bool row_valid, warp_active; int node; size_t orow; };
+    auto row_of = [&](const ask_seg& sg) -> seg_row {
+      seg_row r;
+      const int row0 = sg.qblk * ASK_ROWS;
+      r.row_valid = row0 + row < n_rows;
+      r.warp_active = row0 + quarter * 32 < n_rows;
+      const int g_idx = r.row_valid ? (row0 + row) / M : 0;
+      r.node = r.row_valid ? (row0 + row) % M : 0;
+      r.orow = ((size_t)sg.b * M + r.node) * Hq + sg.kvh * G + g_idx;
+      return r;
+    };
+    uint4 qv[QV];
+    auto fetch_q = [&](const seg_row& r) {
 #pragma unroll
       for (int c = 0; c < QV; ++c) {
         qv[c] = make_uint4(0u, 0u, 0u, 0u);
-        if (row_valid)
-          qv[c] = __ldg(reinterpret_cast<const uint4*>(q + orow * D + half * (D / 2) + c * 8));
+        if (r.row_valid)
+          qv[c] = __ldg(reinterpret_cast<const uint4*>(q + r.orow * D + half * (D / 2) + c * 8));
       }
-      if (sm_tid < M) T.parent[sm_tid] = __ldg(parent + (size_t)s.b * M + sm_tid);
+    };
+    // (every MMA that read the Q tile has completed when this runs)
+    auto stage = [&](const ask_seg& sg) {
+      if (sm_tid < M) T.parent[sm_tid] = __ldg(parent + (size_t)sg.b * M + sm_tid);
       mbar_arrive(&T.par_full);
 #pragma unroll
       for (int c = 0; c < QV; ++c) {
         const int ch = half * QV + c;
-        *reinterpret_cast<uint4*>(sq + (ch >> 3) * 16384 + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
-            qv[c];
+        if (row < QR)
+          *reinterpret_cast<uint4*>(sq + (ch >> 3) * Q_KB + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
+              qv[c];
       }
       fence_proxy_async_smem();
       mbar_arrive(&T.q_full);
+    };
+    uint32_t x = x0;
+    bool have = x < x1;
+    ask_seg s{};
+    if (have) {
+      s = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
+      fetch_q(row_of(s));
+      stage(s);
+    }
+    for (; have; ++seg) {
+      x += (uint32_t)(s.tile_hi - s.tile_lo);
+      const int P = T.plen[s.b];
+      const seg_row sr = row_of(s);
+      const bool row_valid = sr.row_valid, warp_active = sr.warp_active;
+      const int node = sr.node;
+      const size_t orow = sr.orow;
       {
         const bool okp = mbar_wait(&T.par_full, (uint32_t)seg & 1u, abort_flag, status);
         ok = __all_sync(0xffffffffu, okp);
@@ -345,7 +411,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
       }
       float m_run = -INFINITY, l_run = 0.f;
       for (int tile = s.tile_lo; tile < s.tile_hi; ++tile, ++g) {
-        const int bf = g & 1;
+        const int bf = g % ASK_NS;
         // visibility of this thread's 64 keys (Fig. 4): prefix keys, then the ancestor set
         unsigned long long vis_lo = 0ull, vis_hi = 0ull;
         if (row_valid) {
@@ -369,7 +435,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         const unsigned long long vis = half ? vis_hi : vis_lo;
         const unsigned b0 = (unsigned)vis, b1 = (unsigned)(vis >> 32);
         {
-          const bool okw = mbar_wait(&T.s_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
+          const bool okw = mbar_wait(&T.s_full[bf], (uint32_t)(g / ASK_NS) & 1u, abort_flag, status);
           ok = __all_sync(0xffffffffu, okw);
         }
         if (!ok) break;
@@ -378,14 +444,28 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         // this thread's half row of S, read once; the row maximum via the partner
         uint32_t r0[32], r1[32];
         float mx = -INFINITY;
+        // A tile inside the prefix needs no masking at all.  The choice is made per warp (a warp
+        // that ran both paths would pay for both): rows past the last live one count as fully
+        // visible there, their values are finite and nobody reads them.
+        const bool all_vis = __all_sync(0xffffffffu, vis == ~0ull || !row_valid);
         if (warp_active) {
           tmem_ld32(sa, r0);
           tmem_ld32(sa + 32u, r1);
           tmem_ld_wait();
+          if (all_vis) {
+            float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
-            if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r1[j]));
+            for (int j = 0; j < 32; j += 2) {
+              m0 = fmaxf(m0, fmaxf(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1])));
+              m1 = fmaxf(m1, fmaxf(__uint_as_float(r1[j]), __uint_as_float(r1[j + 1])));
+            }
+            mx = fmaxf(m0, m1);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
+              if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r1[j]));
+            }
           }
         }
         T.xmax[bf][half][row] = mx;
@@ -400,33 +480,53 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
           alpha = (m_run == -INFINITY) ? 0.f : fast_exp2((m_run - mx) * sl2);
           m_run = mx;
         }
-        const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-        // P = exp(S - max) as bf16, two keys per 32-bit column, back into tensor memory over S
+        const float m_sl2 = (m_run == -INFINITY) ? 0.f : m_run * sl2;
+        // P = exp2(S * scale * log2 e - max * scale * log2 e) as bf16, two keys per 32-bit column,
+        // back into tensor memory over S; the row sum adds the values before their rounding
         float lsum = 0.f;
         if (warp_active) {
           uint32_t pk[32];
+          float l0 = 0.f, l1 = 0.f;
+          if (all_vis) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = ((b0 >> j) & 1u) ? fast_exp2((__uint_as_float(r0[j]) - m_use) * sl2) : 0.f;
-            const float p1 = ((b0 >> (j + 1)) & 1u)
-                                 ? fast_exp2((__uint_as_float(r0[j + 1]) - m_use) * sl2) : 0.f;
-            const float p2 = ((b1 >> j) & 1u) ? fast_exp2((__uint_as_float(r1[j]) - m_use) * sl2) : 0.f;
-            const float p3 = ((b1 >> (j + 1)) & 1u)
-                                 ? fast_exp2((__uint_as_float(r1[j + 1]) - m_use) * sl2) : 0.f;
-            const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
-            const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
-            // the sum runs over the rounded values the second product will use
-            lsum += (__low2float(h01) + __high2float(h01)) + (__low2float(h23) + __high2float(h23));
-            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
-            pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+            for (int j = 0; j < 32; j += 2) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(r0[j]), sl2, -m_sl2));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(r0[j + 1]), sl2, -m_sl2));
+              const float p2 = fast_exp2(fmaf(__uint_as_float(r1[j]), sl2, -m_sl2));
+              const float p3 = fast_exp2(fmaf(__uint_as_float(r1[j + 1]), sl2, -m_sl2));
+              const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+              const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+              l0 += p0 + p1;
+              l1 += p2 + p3;
+              pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+              pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              const float p0 = ((b0 >> j) & 1u) ? fast_exp2(fmaf(__uint_as_float(r0[j]), sl2, -m_sl2)) : 0.f;
+              const float p1 = ((b0 >> (j + 1)) & 1u)
+                                   ? fast_exp2(fmaf(__uint_as_float(r0[j + 1]), sl2, -m_sl2)) : 0.f;
+              const float p2 = ((b1 >> j) & 1u) ? fast_exp2(fmaf(__uint_as_float(r1[j]), sl2, -m_sl2)) : 0.f;
+              const float p3 = ((b1 >> (j + 1)) & 1u)
+                                   ? fast_exp2(fmaf(__uint_as_float(r1[j + 1]), sl2, -m_sl2)) : 0.f;
+              const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+              const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+              l0 += p0 + p1;
+              l1 += p2 + p3;
+              pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+              pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+            }
           }
+          lsum = l0 + l1;
           tmem_st32(tmem_base + lane_base + (uint32_t)bf * 128u + (uint32_t)half * 32u, pk);
         }
         // O is rescaled only when some row of the warp moved its reference, and only then does
         // the softmax have to wait for the previous tile's P V product (both warps of a row pair
         // see the same rows and take the same decision)
         if (tile > s.tile_lo && __any_sync(0xffffffffu, alpha != 1.f)) {
-          const bool okp = mbar_wait(&T.pv_done, (uint32_t)(g - 1) & 1u, abort_flag, status);
+          const bool okp = mbar_wait(&T.p_free[(g - 1) % ASK_NS], (uint32_t)((g - 1) / ASK_NS) & 1u,
+                                     abort_flag, status);
           ok = __all_sync(0xffffffffu, okp);
           if (!ok) break;
           tc_fence_after();
@@ -450,11 +550,11 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         // are cleared in the V tile before the second product reads it.
         const int live = P + M - tile * ASK_KEYS;
         if (live < ASK_KEYS) {
-          const bool okv = mbar_wait(&T.v_full[bf], (uint32_t)(g >> 1) & 1u, abort_flag, status);
+          const bool okv = mbar_wait(&T.v_full[g % ASK_NV], (uint32_t)(g / ASK_NV) & 1u, abort_flag, status);
           ok = __all_sync(0xffffffffu, okv);
           if (!ok) break;
           const int n16 = (ASK_KEYS - live) * 8;               // 16-byte pieces per 64-wide block
-          unsigned char* vt = sv + bf * KV_BYTES;
+          unsigned char* vt = sv + (g % ASK_NV) * KV_BYTES;
           for (int idx = sm_tid; idx < n16 * KB; idx += ASK_SM_THREADS) {
             const int kb = idx / n16, rem = idx % n16;
             *reinterpret_cast<uint4*>(vt + kb * 16384 + (live + (rem >> 3)) * 128 + ((rem & 7) << 4)) =
@@ -466,18 +566,28 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
         mbar_arrive(&T.p_full[bf]);
       }
       if (!ok) break;
-      // ---- the segment's partial (max, sum, O) of every row
+      // ---- the next segment's rows are requested now and staged once this segment's products
+      //      have completed; then the segment's partial (max, sum, O) of every row
+      const bool have_next = x < x1;
+      ask_seg sn{};
+      if (have_next) {
+        sn = ask_segment(T.tiles, B, items_per_b, n_qblk, x, x1, pl, cta);
+        fetch_q(row_of(sn));
+      }
       {
         const bool okd = mbar_wait(&T.o_ready, (uint32_t)seg & 1u, abort_flag, status);
         ok = __all_sync(0xffffffffu, okd);
       }
       if (!ok) break;
       tc_fence_after();
-      T.xsum[half][row] = l_run;
-      ok = pair_sync();
-      if (!ok) break;
+      if (have_next) stage(sn);
+      // The partials are laid out for this store: [slice][item][16-byte piece][row of the block],
+      // so that the 32 rows of a warp write 512 contiguous bytes per instruction.  Each half row
+      // stores its own sum; the merge adds the two.
       if (warp_active) {
-        float* po = part_o + ((size_t)s.slice * n_out + orow) * D + half * (D / 2);
+        const size_t item = ((size_t)s.b * Hkv + s.kvh) * n_qblk + s.qblk;
+        const size_t blk = (size_t)s.slice * ((size_t)B * items_per_b) + item;
+        float* po = part_o + blk * ((size_t)ASK_ROWS * D) + (size_t)row * 4;
 #pragma unroll 1
         for (int c = 0; c < D / 64; ++c) {
           uint32_t r[32];
@@ -485,19 +595,23 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
           tmem_ld_wait();
           if (row_valid) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(po + c * 32 + j) =
+            for (int j = 0; j < 32; j += 4) {
+              const int piece = (half * (D / 2) + c * 32 + j) >> 2;
+              *reinterpret_cast<float4*>(po + (size_t)piece * (ASK_ROWS * 4)) =
                   make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
                               __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            }
           }
         }
-        if (row_valid && half == 0) {
-          part_ml[((size_t)s.slice * n_out + orow) * 2] =
-              (m_run == -INFINITY) ? -INFINITY : m_run * scale;
-          part_ml[((size_t)s.slice * n_out + orow) * 2 + 1] = l_run + T.xsum[1][row];
+        if (row_valid) {
+          float* pm = part_ml + (blk * ASK_ROWS + row) * 4;
+          if (half == 0) pm[0] = (m_run == -INFINITY) ? -INFINITY : m_run * scale;
+          pm[1 + half] = l_run;
         }
       }
       tc_fence_before();
+      s = sn;
+      have = have_next;
     }
   }
   if (tid == 0 && *abort_flag) {
@@ -507,9 +621,7 @@ __global__ void __launch_bounds__(ASK_THREADS, 1) k_tree_attn_sk(
   }
   tc_fence_before();
   __syncthreads();
-  // Only now may the next kernel of the stream be scheduled: CTAs of a dependent grid that sit
-  // on this SM in their grid-dependency wait were measured to slow this kernel's own warps.
-  jk_pdl_trigger();
+  jk_pdl_trigger();                  // (CTAs without work, and the ones that gave up)
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
@@ -555,8 +667,13 @@ __global__ void __launch_bounds__(256) k_attn_combine_sk(
   const uint32_t item = (uint32_t)((head / G) * n_qblk + ((head % G) * M + node) / ASK_ROWS);
   const uint32_t start = base + item * Tb;
   const int n_split = (int)(ask_owner(start + Tb - 1u, pl) - ask_owner(start, pl)) + 1;
-  const float* po = part_o + row * D + lane * DPL;      // partial s is s * n_out * D further
-  const size_t sstride = n_out * D;
+  // [slice][item][16-byte piece][row of the block][4]: see the attention kernel's epilogue
+  const size_t gitem = (size_t)b * items_per_b + item;
+  const int lrow = ((head % G) * M + node) % ASK_ROWS;
+  const size_t n_items = (size_t)B * items_per_b;
+  const float* po = part_o + gitem * ((size_t)ASK_ROWS * D) +
+                    ((size_t)((lane * DPL) >> 2) * ASK_ROWS + lrow) * 4 + ((lane * DPL) & 3);
+  const size_t sstride = n_items * ((size_t)ASK_ROWS * D);
   auto load_batch = [&](int s0, float (&v)[4][DPL]) {   // four independent vector loads in flight
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -576,9 +693,10 @@ __global__ void __launch_bounds__(256) k_attn_combine_sk(
   // lane s holds (max, sum) of partial s (n_split < 32); one load round for all partials
   float ms = -INFINITY, ls = 0.f;
   if (lane < n_split) {
-    const float2 x = *reinterpret_cast<const float2*>(part_ml + ((size_t)lane * n_out + row) * 2);
+    const float4 x = *reinterpret_cast<const float4*>(
+        part_ml + (((size_t)lane * n_items + gitem) * ASK_ROWS + lrow) * 4);
     ms = x.x;
-    ls = x.y;
+    ls = x.y + x.z;
   }
   const float m = jk_warp_max(ms);
   const float w_lane = (ms == -INFINITY) ? 0.f : __expf(ms - m);
@@ -632,25 +750,37 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   float* part_ml = (float*)(ctx->ws + L.attn_ml);
   int32_t* status = (int32_t*)(ctx->ws + L.status);
   if (!ctx->attn_sk_smem_set) {
-    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<128>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024));
-    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<64>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 210 * 1024));
+    const int cap = 227 * 1024;
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<128, 128>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, cap));
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<128, 64>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, cap));
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<64, 128>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, cap));
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tree_attn_sk<64, 64>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, cap));
     ctx->attn_sk_smem_set = 1;
   }
-  const size_t smem = (size_t)ASK_ROWS * D * 2 + 4 * (size_t)ASK_KEYS * D * 2 + sizeof(ask_tail) + 1024;
+  // a query block of at most 64 live rows keeps a 64-row Q tile and a third V tile instead
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int qr = (G * M <= 64) ? 64 : ASK_ROWS;
+  const int nv = qr == 64 ? 3 : 2;
+  const size_t smem = (size_t)qr * D * 2 + (size_t)(ASK_NK + nv) * ASK_KEYS * D * 2 +
+                      sizeof(ask_tail) + 1024;
   const int n_cta = ctx->sm_count;
   const int ms = L.attn_max_split;
   const int min_units = 1;
   JK_PROF(ctx, st, ctx->st_attn);
-  if (D == 128)
-    jk_launch_pdl(k_tree_attn_sk<128>, dim3(n_cta), dim3(ASK_THREADS), smem, st, mk, mv,
-                  (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
-                  ms, min_units, cache_rows, part_o, part_ml, status);
-  else
-    jk_launch_pdl(k_tree_attn_sk<64>, dim3(n_cta), dim3(ASK_THREADS), smem, st, mk, mv,
-                  (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,
-                  ms, min_units, cache_rows, part_o, part_ml, status);
+#define ASK_LAUNCH(DD, QQ)                                                                        \
+  jk_launch_pdl(k_tree_attn_sk<DD, QQ>, dim3(n_cta), dim3(ASK_THREADS), smem, st, mk, mv,         \
+                (const __nv_bfloat16*)q, kv_len, parent, scale, B, M, c.n_q_heads, c.n_kv_heads,  \
+                ms, min_units, cache_rows, part_o, part_ml, status)
+  if (D == 128) {
+    if (qr == 64) ASK_LAUNCH(128, 64); else ASK_LAUNCH(128, 128);
+  } else {
+    if (qr == 64) ASK_LAUNCH(64, 64); else ASK_LAUNCH(64, 128);
+  }
+#undef ASK_LAUNCH
   JK_LAUNCH_CHECK(ctx);
   const size_t n_out = (size_t)B * M * c.n_q_heads;
   JK_PROF(ctx, st, ctx->st_combine);
