@@ -213,14 +213,28 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       const uint32_t sa = tmem_base + lane_base + (uint32_t)half * 64u;
       uint32_t r0[32], r1[32];
       float mx = -INFINITY;
+      // A tile inside the prefix needs no masking at all.  The choice is made per warp (a warp
+      // that ran both paths would pay for both): rows past the last live one count as fully
+      // visible there, their values are finite and nobody reads them.
+      const bool all_vis = __all_sync(0xffffffffu, vis == ~0ull || !row_valid);
       if (warp_has_rows) {
         tmem_ld32(sa, r0);
         tmem_ld32(sa + 32u, r1);
         tmem_ld_wait();
+        if (all_vis) {
+          float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
-          if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r1[j]));
+          for (int j = 0; j < 32; j += 2) {
+            m0 = fmaxf(m0, fmaxf(__uint_as_float(r0[j]), __uint_as_float(r0[j + 1])));
+            m1 = fmaxf(m1, fmaxf(__uint_as_float(r1[j]), __uint_as_float(r1[j + 1])));
+          }
+          mx = fmaxf(m0, m1);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if ((b0 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r0[j]));
+            if ((b1 >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r1[j]));
+          }
         }
       }
       T.xmax[half][row] = mx;
@@ -236,27 +250,46 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
         alpha = (m_run == -INFINITY) ? 0.f : fast_exp2((m_run - mx) * sl2);
         m_run = mx;
       }
-      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      // ---- P = exp(S - max) as bf16, two keys per 32-bit column, back into tensor memory over
-      // S (its only reader, this thread pair, is done with it)
+      const float m_sl2 = (m_run == -INFINITY) ? 0.f : m_run * sl2;
+      // ---- P = exp2(S * c - max * c) as bf16, two keys per 32-bit column, back into tensor
+      // memory over S (its only reader, this thread pair, is done with it); the row sum adds the
+      // values before their rounding
       float lsum = 0.f;
       if (warp_has_rows) {
         uint32_t pk[32];
+        float l0 = 0.f, l1 = 0.f;
+        if (all_vis) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const float p0 = ((b0 >> j) & 1u) ? fast_exp2((__uint_as_float(r0[j]) - m_use) * sl2) : 0.f;
-          const float p1 = ((b0 >> (j + 1)) & 1u)
-                               ? fast_exp2((__uint_as_float(r0[j + 1]) - m_use) * sl2) : 0.f;
-          const float p2 = ((b1 >> j) & 1u) ? fast_exp2((__uint_as_float(r1[j]) - m_use) * sl2) : 0.f;
-          const float p3 = ((b1 >> (j + 1)) & 1u)
-                               ? fast_exp2((__uint_as_float(r1[j + 1]) - m_use) * sl2) : 0.f;
-          const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
-          const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
-          // the sum runs over the rounded values the second product will use
-          lsum += (__low2float(h01) + __high2float(h01)) + (__low2float(h23) + __high2float(h23));
-          pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
-          pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(r0[j]), sl2, -m_sl2));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(r0[j + 1]), sl2, -m_sl2));
+            const float p2 = fast_exp2(fmaf(__uint_as_float(r1[j]), sl2, -m_sl2));
+            const float p3 = fast_exp2(fmaf(__uint_as_float(r1[j + 1]), sl2, -m_sl2));
+            const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+            const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+            l0 += p0 + p1;
+            l1 += p2 + p3;
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+            pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = ((b0 >> j) & 1u) ? fast_exp2(fmaf(__uint_as_float(r0[j]), sl2, -m_sl2)) : 0.f;
+            const float p1 = ((b0 >> (j + 1)) & 1u)
+                                 ? fast_exp2(fmaf(__uint_as_float(r0[j + 1]), sl2, -m_sl2)) : 0.f;
+            const float p2 = ((b1 >> j) & 1u) ? fast_exp2(fmaf(__uint_as_float(r1[j]), sl2, -m_sl2)) : 0.f;
+            const float p3 = ((b1 >> (j + 1)) & 1u)
+                                 ? fast_exp2(fmaf(__uint_as_float(r1[j + 1]), sl2, -m_sl2)) : 0.f;
+            const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+            const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+            l0 += p0 + p1;
+            l1 += p2 + p3;
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&h01);
+            pk[16 + (j >> 1)] = *reinterpret_cast<const uint32_t*>(&h23);
+          }
         }
+        lsum = l0 + l1;
         tmem_st32(tmem_base + lane_base + (uint32_t)half * 32u, pk);
         // rescale this thread's half of the running output when some row of the warp moved its
         // reference (the previous tile's P V product has completed: the loop waits for it)
