@@ -6,7 +6,7 @@
 // persistent kernel serves them:
 //   - the weight matrix sits on the 128-row M side of tcgen05.mma, the activation rows on N
 //     (padded to a multiple of 16), accumulators in tensor memory;
-//   - work is cut into units of one 128 x 64 weight tile; the units of all (group, tile) pairs are
+//   - work is cut into units of one 128 x 128 (or 128 x 64) weight tile; the units of all (group, tile) pairs are
 //     laid end to end and every CTA takes an equal contiguous span (stream-K), so all SMs stream
 //     the same number of bytes whatever the tile count is;
 //   - a producer thread feeds a ring of shared-memory stages with TMA (128B swizzle), one thread
@@ -24,7 +24,11 @@
 #include "jk_topk.cuh"
 
 #define TC_TILE_M 128
-#define TC_TILE_K 64
+#define TC_BOX_K 64                  // one TMA box: 64 bf16 = the 128-byte swizzle span
+// A stage holds KB boxes side by side along K.  Two (256 contiguous bytes of every weight row per
+// stage) stream measurably faster than one; with many activation rows a two-box stage would leave
+// too few stages in the ring, and one box is used.
+#define TC_KB_WIDE_MIN_STAGES 4
 #define TC_THREADS 192               // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
 #define TC_MAX_GROUPS 16
 #define TC_MAX_STAGES 12
@@ -37,7 +41,9 @@ struct tc_params {
   int group_arow0[TC_MAX_GROUPS];    // first row of the group in its A tensor map
   int group_brow0[TC_MAX_GROUPS];    // first row of the group's activations in the B tensor map
   int tiles_per_group;               // ceil(M_rows / 128)
-  int kt;                            // ceil(K / 64)
+  int kdim;                          // K
+  int kb;                            // TMA boxes per stage along K (1 or 2)
+  int kt;                            // ceil(K / (64 * kb))
   int n_pad;                         // activation rows, multiple of 16
   int stages;
   int max_seg;                       // partial slots per CTA
@@ -98,12 +104,14 @@ struct __align__(1024) tc_smem_tail {
   tc_plan plan;
 };
 
+template <int TC_KB>
 __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
     const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
     const __grid_constant__ CUtensorMap map_b, const tc_params p, const int32_t* __restrict__ expert,
     float* __restrict__ partial, int32_t* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int TC_TILE_K = TC_KB * TC_BOX_K;
   const int stage_bytes = TC_TILE_M * TC_TILE_K * 2 + p.n_pad * TC_TILE_K * 2;
   tc_smem_tail& T = *reinterpret_cast<tc_smem_tail*>(smem + (size_t)p.stages * stage_bytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -186,15 +194,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       cursor cb = ca;
       for (int i = 0; i < npre; ++i) {
         mbar_expect_tx(&T.full[i], (uint32_t)stage_bytes);
-        tma_load_2d_hint(smem + (size_t)i * stage_bytes, ca.ma, ca.kt * TC_TILE_K, ca.arow,
-                         &T.full[i], pol);
+#pragma unroll
+        for (int kb = 0; kb < TC_KB; ++kb)
+          tma_load_2d_hint(smem + (size_t)i * stage_bytes + kb * (TC_TILE_M * TC_BOX_K * 2), ca.ma,
+                           ca.kt * TC_TILE_K + kb * TC_BOX_K, ca.arow, &T.full[i], pol);
         cur_next(ca, i + 1 < n_units);
       }
       jk_pdl_wait();
       jk_pdl_trigger();
       for (int i = 0; i < npre; ++i) {
-        tma_load_2d(smem + (size_t)i * stage_bytes + TC_TILE_M * TC_TILE_K * 2, &map_b,
-                    cb.kt * TC_TILE_K, cb.brow, &T.full[i]);
+#pragma unroll
+        for (int kb = 0; kb < TC_KB; ++kb)
+          tma_load_2d(smem + (size_t)i * stage_bytes + TC_TILE_M * TC_TILE_K * 2 +
+                          kb * (p.n_pad * TC_BOX_K * 2),
+                      &map_b, cb.kt * TC_TILE_K + kb * TC_BOX_K, cb.brow, &T.full[i]);
         cur_next(cb, i + 1 < n_units);
       }
       issued = npre;
@@ -206,8 +219,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       unsigned char* sa = smem + (size_t)s * stage_bytes;
       unsigned char* sb = sa + TC_TILE_M * TC_TILE_K * 2;
       mbar_expect_tx(&T.full[s], (uint32_t)stage_bytes);
-      tma_load_2d_hint(sa, ca.ma, ca.kt * TC_TILE_K, ca.arow, &T.full[s], pol);
-      tma_load_2d(sb, &map_b, ca.kt * TC_TILE_K, ca.brow, &T.full[s]);
+#pragma unroll
+      for (int kb = 0; kb < TC_KB; ++kb)
+        tma_load_2d_hint(sa + kb * (TC_TILE_M * TC_BOX_K * 2), ca.ma,
+                         ca.kt * TC_TILE_K + kb * TC_BOX_K, ca.arow, &T.full[s], pol);
+#pragma unroll
+      for (int kb = 0; kb < TC_KB; ++kb)
+        tma_load_2d(sb + kb * (p.n_pad * TC_BOX_K * 2), &map_b, ca.kt * TC_TILE_K + kb * TC_BOX_K,
+                    ca.brow, &T.full[s]);
       if (++s == p.stages) { s = 0; ph ^= 1u; }
       cur_next(ca, issued + 1 < n_units);
     }
@@ -241,12 +260,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
         const uint32_t b_addr = a_addr + TC_TILE_M * TC_TILE_K * 2;
-        const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
 #pragma unroll
-        for (int k = 0; k < TC_TILE_K / 16; ++k) {
-          // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in the address field
-          tc_mma_bf16(d_addr, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
-                      (first && k == 0) ? 0u : 1u);
+        for (int kb = 0; kb < TC_KB; ++kb) {
+          const uint64_t da = smem_desc_sw128(a_addr + kb * (TC_TILE_M * TC_BOX_K * 2));
+          const uint64_t db = smem_desc_sw128(b_addr + kb * (p.n_pad * TC_BOX_K * 2));
+#pragma unroll
+          for (int k = 0; k < TC_BOX_K / 16; ++k) {
+            // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in the address field
+            tc_mma_bf16(d_addr, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
+                        (first && kb == 0 && k == 0) ? 0u : 1u);
+          }
         }
         first = false;
         tc_commit(&T.empty[s]);          // the stage is free once these MMAs have read it
@@ -512,10 +535,10 @@ static int tc_grid(const jk_ctx* ctx) {
   return n > TC_MAX_GRID ? TC_MAX_GRID : n;
 }
 
-static int tc_stage_bytes(int n_pad) { return TC_TILE_M * TC_TILE_K * 2 + n_pad * TC_TILE_K * 2; }
+static int tc_stage_bytes(int n_pad, int kb) { return (TC_TILE_M + n_pad) * kb * TC_BOX_K * 2; }
 
-static int tc_stages(int n_pad) {
-  int s = (TC_SMEM_BUDGET - (int)sizeof(tc_smem_tail) - 1024) / tc_stage_bytes(n_pad);
+static int tc_stages(int n_pad, int kb) {
+  int s = (TC_SMEM_BUDGET - (int)sizeof(tc_smem_tail) - 1024) / tc_stage_bytes(n_pad, kb);
   if (s > TC_MAX_STAGES) s = TC_MAX_STAGES;
   return s;
 }
@@ -534,7 +557,7 @@ static size_t tc_partial_for(long long units, int kt, int n_pad) {
 size_t jk_tc_partial_bytes(const jk_config& c) {
   const int R = c.max_batch * c.max_frontier;
   const int np1 = (int)jk_align_up(R, 16), np2 = (int)jk_align_up((size_t)R * c.top_k, 16);
-  const int kt_h = (c.hidden + TC_TILE_K - 1) / TC_TILE_K, kt_i = (c.inter + TC_TILE_K - 1) / TC_TILE_K;
+  const int kt_h = (c.hidden + TC_BOX_K - 1) / TC_BOX_K, kt_i = (c.inter + TC_BOX_K - 1) / TC_BOX_K;
   const long long t_i = (c.inter + TC_TILE_M - 1) / TC_TILE_M, t_h = (c.hidden + TC_TILE_M - 1) / TC_TILE_M,
                   t_v = (c.vocab + TC_TILE_M - 1) / TC_TILE_M;
   size_t a = tc_partial_for(2ll * c.n_experts * t_i * kt_h, kt_h, np1);
@@ -542,7 +565,7 @@ size_t jk_tc_partial_bytes(const jk_config& c) {
   size_t d = tc_partial_for(t_v * kt_h, kt_h, np2);
   // the draft layer's reduction, QKV and output projections (one group each)
   const int qd = c.n_q_heads * c.head_dim, qkvd = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
-  const int kt_2h = (2 * c.hidden + TC_TILE_K - 1) / TC_TILE_K, kt_q = (qd + TC_TILE_K - 1) / TC_TILE_K;
+  const int kt_2h = (2 * c.hidden + TC_BOX_K - 1) / TC_BOX_K, kt_q = (qd + TC_BOX_K - 1) / TC_BOX_K;
   const long long t_qkv = (qkvd + TC_TILE_M - 1) / TC_TILE_M;
   size_t e1 = tc_partial_for(t_h * kt_2h, kt_2h, np1);
   // (jk_verify_qkv sends up to 256 tree tokens at a time through the QKV projection)
@@ -584,7 +607,7 @@ int jk_tc_available(const jk_ctx* ctx) {
   if (c.dtype != JK_BF16) return 0;
   const int np2 = (int)jk_align_up((size_t)c.max_batch * c.max_frontier * c.top_k, 16);
   if (np2 > 256) return 0;                       // two accumulators must fit the 512 TMEM columns
-  if (tc_stages(np2) < 2) return 0;
+  if (tc_stages(np2, 1) < 2) return 0;
   tc_state* s = tc_get_state(const_cast<jk_ctx*>(ctx));
   return s && !s->failed;
 }
@@ -604,7 +627,7 @@ static const CUtensorMap* tc_map_lookup(jk_ctx* ctx, tc_state* s, const void* pt
   tc_map_entry& e = s->maps[s->n_maps];
   const cuuint64_t gdim[2] = {cols, rows};
   const cuuint64_t gstride[1] = {cols * 2};
-  const cuuint32_t box[2] = {TC_TILE_K, box_rows};
+  const cuuint32_t box[2] = {TC_BOX_K, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   CUresult r = s->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim,
                          gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -634,7 +657,9 @@ static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUten
                           const int32_t* expert, int stage_id, int* n_cta_out) {
   const jk_ws_layout& L = ctx->lay;
   const int n_cta = tc_grid(ctx);
-  p.stages = tc_stages(p.n_pad);
+  p.kb = tc_stages(p.n_pad, 2) >= TC_KB_WIDE_MIN_STAGES ? 2 : 1;
+  p.kt = (p.kdim + p.kb * TC_BOX_K - 1) / (p.kb * TC_BOX_K);
+  p.stages = tc_stages(p.n_pad, p.kb);
   const long long max_units = (long long)p.n_groups_max * p.tiles_per_group * p.kt;
   p.max_seg = tc_max_seg(max_units, n_cta, p.kt);
   if (max_units * TC_MAX_GRID >= (1ll << 31)) return JK_ERR_SHAPE;   // 32-bit span arithmetic
@@ -643,16 +668,21 @@ static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUten
   p.tmem_cols = cols;
   if ((size_t)n_cta * p.max_seg * p.n_pad * TC_TILE_M * sizeof(float) > L.gemm_part_bytes)
     return JK_ERR_WORKSPACE;
-  const size_t smem = (size_t)p.stages * tc_stage_bytes(p.n_pad) + sizeof(tc_smem_tail) + 1024;
+  const size_t smem = (size_t)p.stages * tc_stage_bytes(p.n_pad, p.kb) + sizeof(tc_smem_tail) + 1024;
   if (!s->smem_set) {
-    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tc_gemm<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            TC_SMEM_BUDGET));
+    JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tc_gemm<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             TC_SMEM_BUDGET));
     s->smem_set = 1;
   }
   JK_PROF(ctx, st, stage_id);
-  jk_launch_pdl(k_tc_gemm, dim3(n_cta), dim3(TC_THREADS), smem, st, *a0, *a1, *b, p, expert,
-                                             (float*)(ctx->ws + L.gemm_part),
-                                             (int32_t*)(ctx->ws + L.status));
+  if (p.kb == 2)
+    jk_launch_pdl(k_tc_gemm<2>, dim3(n_cta), dim3(TC_THREADS), smem, st, *a0, *a1, *b, p, expert,
+                  (float*)(ctx->ws + L.gemm_part), (int32_t*)(ctx->ws + L.status));
+  else
+    jk_launch_pdl(k_tc_gemm<1>, dim3(n_cta), dim3(TC_THREADS), smem, st, *a0, *a1, *b, p, expert,
+                  (float*)(ctx->ws + L.gemm_part), (int32_t*)(ctx->ws + L.status));
   JK_LAUNCH_CHECK(ctx);
   *n_cta_out = n_cta;
   return JK_OK;
@@ -686,7 +716,7 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
       p.group_expert[g] = e; p.group_amap[g] = h; p.group_arow0[g] = e * I; p.group_brow0[g] = 0;
     }
   p.tiles_per_group = (I + TC_TILE_M - 1) / TC_TILE_M;
-  p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
+  p.kdim = H;
   p.n_pad = n_pad;
   int rc = tc_launch_gemm(ctx, st, s, &ag, &au, &bx, p, expert, JK_ST_GATEUP, &n_cta);
   if (rc != JK_OK) return rc;
@@ -704,7 +734,7 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
     p.group_expert[e] = e; p.group_amap[e] = 0; p.group_arow0[e] = e * H; p.group_brow0[e] = e * Rp;
   }
   p.tiles_per_group = (H + TC_TILE_M - 1) / TC_TILE_M;
-  p.kt = (I + TC_TILE_K - 1) / TC_TILE_K;
+  p.kdim = I;
   p.prefetch = 1;
   rc = tc_launch_gemm(ctx, st, s, &ad, &ad, &bh, p, expert, JK_ST_DOWN, &n_cta);
   if (rc != JK_OK) return rc;
@@ -737,7 +767,7 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
   p.n_groups_max = 1;
   p.group_expert[0] = -1; p.group_amap[0] = 0; p.group_arow0[0] = 0; p.group_brow0[0] = 0;
   p.tiles_per_group = (V + TC_TILE_M - 1) / TC_TILE_M;
-  p.kt = (H + TC_TILE_K - 1) / TC_TILE_K;
+  p.kdim = H;
   p.n_pad = n_pad;
   int n_cta = 0;
   p.prefetch = 1;
@@ -797,7 +827,7 @@ int jk_tc_linear(jk_ctx* ctx, cudaStream_t st, const void* W, int Mrows, int Kdi
   p.n_groups_max = 1;
   p.group_expert[0] = -1; p.group_amap[0] = 0; p.group_arow0[0] = 0; p.group_brow0[0] = 0;
   p.tiles_per_group = (Mrows + TC_TILE_M - 1) / TC_TILE_M;
-  p.kt = (Kdim + TC_TILE_K - 1) / TC_TILE_K;
+  p.kdim = Kdim;
   p.n_pad = n_pad;
   p.prefetch = 1;
   int n_cta = 0;
