@@ -101,17 +101,21 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
   uint32_t tmem_base = 0;
   float m_run = -INFINITY, l_run = 0.f;
 
-  auto issue_kv = [&](int tile) {
+  auto issue_k = [&](int tile) {
     const uint64_t pol = l2_policy_evict_first();   // the cache is read once per call
     mbar_expect_tx(&T.bar_k, ATC_KEYS * D * 2);
 #pragma unroll
     for (int kb = 0; kb < KB; ++kb)
       tma_load_4d_hint(skp + kb * 16384, &map_k, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_k, pol);
+  };
+  auto issue_v = [&](int tile) {
+    const uint64_t pol = l2_policy_evict_first();
     mbar_expect_tx(&T.bar_v, ATC_KEYS * D * 2);
 #pragma unroll
     for (int kb = 0; kb < KB; ++kb)
       tma_load_4d_hint(sv + kb * 16384, &map_v, kb * 64, tile * ATC_KEYS, kvh, b, &T.bar_v, pol);
   };
+  auto issue_kv = [&](int tile) { issue_k(tile); issue_v(tile); };
   const bool early = have_keys && (t0 + 1) * ATC_KEYS <= P;
   if (early && tid == 0) issue_kv(t0);
   jk_pdl_wait();
@@ -207,6 +211,8 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       ok = ok && mbar_wait(&T.bar_s, ph, abort_flag, status);
       if (!__syncthreads_and(ok)) { ok = false; break; }
       tc_fence_after();
+      // S is complete, so the K tile is free: the next one travels under this tile's softmax
+      if (tid == 0 && tile + 1 < t1) issue_k(tile + 1);
 
       // ---- this thread's half row of S, read once.  (Warps whose 32 rows all lie past the last
       // query row skip the row work: their rows of P and O are never stored.)
@@ -342,7 +348,7 @@ __global__ void __launch_bounds__(ATC_THREADS, 2) k_tree_attn_tc(
       ok = ok && mbar_wait(&T.bar_o, ph, abort_flag, status);
       if (!__syncthreads_and(ok)) { ok = false; break; }
       tc_fence_after();
-      if (tid == 0 && tile + 1 < t1) issue_kv(tile + 1);
+      if (tid == 0 && tile + 1 < t1) issue_v(tile + 1);
     }
     if (ok) {
       // The partial O goes through shared memory (over the K and V tiles: every MMA has
@@ -477,15 +483,20 @@ int jk_attn_tc(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
                const int32_t* parent, float scale, void* out) {
   const jk_config& c = ctx->cfg;
   const jk_ws_layout& L = ctx->lay;
-  // The persistent kernel wins once every SM has many key tiles to walk (measured: 56 against 79 us
-  // at 18 tiles per SM, 37 against 33 us at 7); below that its longer set-up costs more than its
-  // pipelining saves.
+  // The persistent kernel wins where the call is bound by streaming K and V and every SM has
+  // many key tiles to walk: one query block per kv head (at most 128 (q head, node) rows share a
+  // K/V tile) and at least 16 tiles per SM.  Measured, persistent against per-slice: 50 against
+  // 65 us (40 heads, batch 4, prefix 2048), 261 against 410 us (batch 8, prefix 8192), but 32
+  // against 30 us at 9 tiles per SM.  With several query blocks per kv head the call is bound by
+  // the tensor pipe and the exponentials, and two per-slice CTAs per SM overlap those better
+  // than one persistent CTA does (64 q / 8 kv heads, batch 8, prefix 8192: 218 against 228 us).
   {
     const int Gq = c.n_q_heads / c.n_kv_heads;
-    const long long units = (long long)B * c.n_kv_heads * ((Gq * M + ATC_ROWS - 1) / ATC_ROWS) *
+    const int n_qblk = (Gq * M + ATC_ROWS - 1) / ATC_ROWS;
+    const long long units = (long long)B * c.n_kv_heads * n_qblk *
                             ((cache_rows + ATC_KEYS - 1) / ATC_KEYS);
     const bool want = ctx->attn_kernel == 2 ||
-                      (ctx->attn_kernel == 0 && units >= 8ll * ctx->sm_count);
+                      (ctx->attn_kernel == 0 && n_qblk == 1 && units >= 16ll * ctx->sm_count);
     if (want && jk_attn_sk_usable(ctx, B, M, cache_rows))
       return jk_attn_sk(ctx, st, B, M, q, kc, vc, sb, sh, cache_rows, kv_len, parent, scale, out);
   }
