@@ -59,6 +59,7 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->tk_ms = take(RK * L->topk_chunks * 2 * 4);
   L->gemm_part_bytes = c.dtype == JK_BF16 ? jk_tc_partial_bytes(c) : 0;
   L->gemm_part = take(L->gemm_part_bytes);
+  L->gemm_cnt = take(16);
   // split-KV partials, capped at 256 MiB
   const size_t pre_nodes = (size_t)c.max_batch * c.max_depth * c.max_frontier;
   size_t rows = (BM > pre_nodes ? BM : pre_nodes) * c.n_q_heads;
@@ -131,6 +132,7 @@ extern "C" int jk_set_workspace(jk_ctx* ctx, void* stream, void* dev_ptr, size_t
   ctx->ws_bytes = bytes;
   jk_tc_destroy(ctx);   // tensor maps over an earlier workspace are stale
   JK_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.status, 0, 16, (cudaStream_t)stream));
+  JK_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->ws + ctx->lay.gemm_cnt, 0, 16, (cudaStream_t)stream));
   return JK_OK;
 }
 

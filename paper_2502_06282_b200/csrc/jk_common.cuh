@@ -53,6 +53,7 @@ struct jk_ws_layout {
   size_t pre_ao;        // T   [Rp, Hq d]    attention outputs of this pass's nodes (O-proj input)
   size_t total;
   int attn_max_split;
+  size_t gemm_cnt;       // four item counters of the streaming GEMM (zero between launches)
   int topk_chunks;
   int rows_pad;         // Rp
   int rk_pad;           // RKp
@@ -82,6 +83,7 @@ struct jk_ctx {
   int sm_count;           // filled at the first launch
   int attn_smem_set;
   int attn_sk_smem_set;
+  unsigned gemm_seq;     // GEMM launches so far: picks the item counter
   int st_attn, st_combine;  // profiling stages the attention kernels are booked under
   int attn_kernel;        // 0 = by size, 1 = CTA per (query block, key slice), 2 = persistent,
                           // 3 = cluster-merged

@@ -6,14 +6,15 @@
 // persistent kernel serves them:
 //   - the weight matrix sits on the 128-row M side of tcgen05.mma, the activation rows on N
 //     (padded to a multiple of 16), accumulators in tensor memory;
-//   - work is cut into units of one 128 x 128 (or 128 x 64) weight tile; the units of all (group, tile) pairs are
-//     laid end to end and every CTA takes an equal contiguous span (stream-K), so all SMs stream
-//     the same number of bytes whatever the tile count is;
+//   - work is cut into items: a run of k steps (a chunk, at least 128 KB of weights) of one 128-row
+//     weight tile; the CTAs take items from a global counter one after the other, so an SM that
+//     gets less of the memory bandwidth at some moment simply ends up with fewer items;
 //   - a producer thread feeds a ring of shared-memory stages with TMA (128B swizzle), one thread
 //     issues the MMAs, four warps drain finished accumulators to fp32 partial tiles in global
-//     memory; a small second kernel adds the partials of each tile in a fixed order (no atomics,
-//     bitwise reproducible) and applies the epilogue: SiLU * up; residual, gates and branch
-//     features; or the LM head's per-chunk top-k statistics.
+//     memory, one per item at a place that depends on the item alone; a small second kernel adds
+//     the partials of each tile in chunk order (no atomics on data, bitwise reproducible
+//     whichever CTA computed what) and applies the epilogue: SiLU * up; residual, gates and
+//     branch features; or the LM head's per-chunk top-k statistics.
 // Every wait on an mbarrier is bounded: after ~2 s it records JK_ERR_TIMEOUT in the status word,
 // and the CTA drains its copies, frees its tensor memory and returns.
 #include <cuda.h>
@@ -43,13 +44,15 @@ struct tc_params {
   int tiles_per_group;               // ceil(M_rows / 128)
   int kdim;                          // K
   int kb;                            // TMA boxes per stage along K (1 or 2)
-  int kt;                            // ceil(K / (64 * kb))
+  int kt;                            // k steps of a tile: ceil(K / (64 * kb))
+  int ch;                            // k steps of a chunk
+  int n_chunks;                      // chunks of a tile: ceil(kt / ch)
   int n_pad;                         // activation rows, multiple of 16
   int stages;
-  int max_seg;                       // partial slots per CTA
   int R, K_top, n_experts;           // to derive the active experts from `expert`
   int tmem_cols;
   int prefetch;                      // 1: the producer streams weight tiles before the grid-dependency wait
+  int* counter;                      // next work item of this launch (zero when the kernel starts)
 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
@@ -64,12 +67,15 @@ __host__ __device__ inline uint32_t instr_desc_bf16(int n) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Work partition shared by the GEMM kernel and the fix-up kernel
+// Work partition shared by the GEMM kernel and the fix-up kernels.  A work item is one chunk of
+// the k steps of one weight tile of one active group; item i = (group, tile, chunk) in that
+// order.  Its partial tile lands in slot i of the partial buffer, whichever CTA computed it, so
+// the sum the fix-up kernels form (chunks in ascending order) does not depend on the dealing.
 // ---------------------------------------------------------------------------------------------
 struct tc_plan {
   int n_groups;                      // active groups
   int group_src[TC_MAX_GROUPS];      // index into the parameter arrays
-  long long total_units;
+  int total_items;
 };
 
 __device__ __forceinline__ void tc_make_plan(const tc_params& p, const int32_t* expert,
@@ -88,22 +94,32 @@ __device__ __forceinline__ void tc_make_plan(const tc_params& p, const int32_t* 
     if (e < 0 || (active >> e) & 1u) plan->group_src[n++] = g;
   }
   plan->n_groups = n;
-  plan->total_units = (long long)n * p.tiles_per_group * p.kt;
+  plan->total_items = n * p.tiles_per_group * p.n_chunks;
 }
-__device__ __forceinline__ long long tc_span_start(long long total, int cta, int n_cta) {
-  return total * cta / n_cta;
-}
+
+#define TC_ITEM_Q 4                  // item ids in flight between the producer and the epilogue warps
+#define TC_FLAG_FIRST 1
+#define TC_FLAG_LAST 2
+#define TC_FLAG_END 4
 
 struct __align__(1024) tc_smem_tail {
   uint64_t full[TC_MAX_STAGES];
   uint64_t empty[TC_MAX_STAGES];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
+  uint64_t iq_full[TC_ITEM_Q];
+  uint64_t iq_empty[TC_ITEM_Q];
   uint32_t tmem_base;
   int abort_flag;
+  int st_flag[TC_MAX_STAGES];        // first / last k step of its item, or the end of the work
+  int q_item[TC_ITEM_Q];
   tc_plan plan;
 };
 
+// Work is dealt dynamically: a CTA asks a global counter for its next item.  The SMs do not get
+// equal shares of the memory bandwidth at every moment (measured: with equal static shares the
+// slowest CTA of a 110 us launch ended 20 us after the fastest), and this way a slower SM simply
+// takes fewer items.
 template <int TC_KB>
 __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
     const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
@@ -120,6 +136,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&T.full[s], 1); mbar_init(&T.empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&T.acc_full[a], 1); mbar_init(&T.acc_empty[a], 4); }
+    for (int i = 0; i < TC_ITEM_Q; ++i) { mbar_init(&T.iq_full[i], 1); mbar_init(&T.iq_empty[i], 4); }
     T.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -139,11 +156,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = T.tmem_base;
-  const long long total = T.plan.total_units;
-  const long long u0 = tc_span_start(total, blockIdx.x, gridDim.x);
-  const long long u1 = tc_span_start(total, blockIdx.x + 1, gridDim.x);
-  const int units_per_tile = p.kt;
-  const long long first_tile = u0 / units_per_tile;
+  const int total = T.plan.total_items;
   // (the whole producer warp skips this wait when it prefetches: lanes of that warp waiting here
   // would hold back the lane that issues the copies; its other lanes touch no global memory)
   if (!(p.prefetch && warp == 0)) {
@@ -153,82 +166,83 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
 
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
-    int issued = 0;
     bool ok = true;
-    const int n_units = (int)(u1 - u0);
     const uint64_t pol = l2_policy_evict_first();   // weight tiles are read once per call
-    // position of a unit of the span, advanced incrementally (no divisions in the loop)
-    struct cursor {
-      int kt, t, gi, g, arow, brow;
-      const CUtensorMap* ma;
-    };
-    auto cur_load = [&](cursor& c) {
-      c.g = T.plan.group_src[c.gi];
-      c.ma = p.group_amap[c.g] ? &map_a1 : &map_a0;
-      c.brow = p.group_brow0[c.g];
-      c.arow = p.group_arow0[c.g] + c.t * TC_TILE_M;
-    };
-    auto cur_next = [&](cursor& c, bool more) {
-      if (++c.kt == units_per_tile) {
-        c.kt = 0;
-        if (++c.t == p.tiles_per_group) {
-          c.t = 0;
-          ++c.gi;
-          if (more) cur_load(c);
-        }
-        c.arow = p.group_arow0[c.g] + c.t * TC_TILE_M;
-      }
-    };
-    cursor ca;
-    ca.kt = (int)(u0 % units_per_tile);
-    ca.t = (int)(first_tile % p.tiles_per_group);
-    ca.gi = (int)(first_tile / p.tiles_per_group);
-    ca.g = 0; ca.arow = 0; ca.brow = 0; ca.ma = &map_a0;
-    if (n_units > 0) cur_load(ca);
-    int s = 0;
+    int s = 0, issued = 0, qn = 0;
     uint32_t ph = 0;
-    if (p.prefetch) {
-      // The weights do not depend on the kernel that runs before this one: start streaming the
-      // first ring of weight tiles now, and add the activation tiles once that kernel is done.
-      const int npre = n_units < p.stages ? n_units : p.stages;
-      cursor cb = ca;
-      for (int i = 0; i < npre; ++i) {
-        mbar_expect_tx(&T.full[i], (uint32_t)stage_bytes);
-#pragma unroll
-        for (int kb = 0; kb < TC_KB; ++kb)
-          tma_load_2d_hint(smem + (size_t)i * stage_bytes + kb * (TC_TILE_M * TC_BOX_K * 2), ca.ma,
-                           ca.kt * TC_TILE_K + kb * TC_BOX_K, ca.arow, &T.full[i], pol);
-        cur_next(ca, i + 1 < n_units);
-      }
+    // With prefetch the weights of the first item start streaming before the grid-dependency
+    // wait (they do not depend on the kernel before); the activation tiles of those stages
+    // follow once that kernel is done.
+    bool waited = !p.prefetch;
+    int pend_s[TC_MAX_STAGES], pend_k[TC_MAX_STAGES], pend_brow = 0, n_pend = 0;
+    auto settle = [&]() {
       jk_pdl_wait();
       jk_pdl_trigger();
-      for (int i = 0; i < npre; ++i) {
+      for (int i = 0; i < n_pend; ++i) {
+        unsigned char* sb = smem + (size_t)pend_s[i] * stage_bytes + TC_TILE_M * TC_TILE_K * 2;
 #pragma unroll
         for (int kb = 0; kb < TC_KB; ++kb)
-          tma_load_2d(smem + (size_t)i * stage_bytes + TC_TILE_M * TC_TILE_K * 2 +
-                          kb * (p.n_pad * TC_BOX_K * 2),
-                      &map_b, cb.kt * TC_TILE_K + kb * TC_BOX_K, cb.brow, &T.full[i]);
-        cur_next(cb, i + 1 < n_units);
+          tma_load_2d(sb + kb * (p.n_pad * TC_BOX_K * 2), &map_b,
+                      pend_k[i] * TC_TILE_K + kb * TC_BOX_K, pend_brow, &T.full[pend_s[i]]);
       }
-      issued = npre;
-      if (npre == p.stages) { s = 0; ph = 1u; } else { s = npre; }
-    }
-    for (; issued < n_units; ++issued) {
-      if (issued >= p.stages) ok = mbar_wait(&T.empty[s], ph ^ 1u, abort_flag, status);
+      n_pend = 0;
+      waited = true;
+    };
+    while (ok) {
+      const int item = atomicAdd(p.counter, 1);
+      if (item >= total) break;
+      // the epilogue warps learn the item (its partial slot) through a small queue
+      const int qs = qn % TC_ITEM_Q;
+      if (qn >= TC_ITEM_Q)
+        ok = mbar_wait(&T.iq_empty[qs], (uint32_t)(qn / TC_ITEM_Q - 1) & 1u, abort_flag, status);
       if (!ok) break;
-      unsigned char* sa = smem + (size_t)s * stage_bytes;
-      unsigned char* sb = sa + TC_TILE_M * TC_TILE_K * 2;
-      mbar_expect_tx(&T.full[s], (uint32_t)stage_bytes);
+      T.q_item[qs] = item;
+      mbar_arrive(&T.iq_full[qs]);
+      ++qn;
+      const int c = item % p.n_chunks, tt = item / p.n_chunks;
+      const int t = tt % p.tiles_per_group, g = T.plan.group_src[tt / p.tiles_per_group];
+      const CUtensorMap* ma = p.group_amap[g] ? &map_a1 : &map_a0;
+      const int arow = p.group_arow0[g] + t * TC_TILE_M, brow = p.group_brow0[g];
+      const int k0 = c * p.ch, k1 = min(p.kt, k0 + p.ch);
+      for (int k = k0; k < k1 && ok; ++k) {
+        if (issued >= p.stages) ok = mbar_wait(&T.empty[s], ph ^ 1u, abort_flag, status);
+        if (!ok) break;
+        unsigned char* sa = smem + (size_t)s * stage_bytes;
+        unsigned char* sb = sa + TC_TILE_M * TC_TILE_K * 2;
+        T.st_flag[s] = (k == k0 ? TC_FLAG_FIRST : 0) | (k == k1 - 1 ? TC_FLAG_LAST : 0);
+        mbar_expect_tx(&T.full[s], (uint32_t)stage_bytes);   // (an arrive: releases the flag too)
 #pragma unroll
-      for (int kb = 0; kb < TC_KB; ++kb)
-        tma_load_2d_hint(sa + kb * (TC_TILE_M * TC_BOX_K * 2), ca.ma,
-                         ca.kt * TC_TILE_K + kb * TC_BOX_K, ca.arow, &T.full[s], pol);
+        for (int kb = 0; kb < TC_KB; ++kb)
+          tma_load_2d_hint(sa + kb * (TC_TILE_M * TC_BOX_K * 2), ma, k * TC_TILE_K + kb * TC_BOX_K,
+                           arow, &T.full[s], pol);
+        if (waited) {
 #pragma unroll
-      for (int kb = 0; kb < TC_KB; ++kb)
-        tma_load_2d(sb + kb * (p.n_pad * TC_BOX_K * 2), &map_b, ca.kt * TC_TILE_K + kb * TC_BOX_K,
-                    ca.brow, &T.full[s]);
-      if (++s == p.stages) { s = 0; ph ^= 1u; }
-      cur_next(ca, issued + 1 < n_units);
+          for (int kb = 0; kb < TC_KB; ++kb)
+            tma_load_2d(sb + kb * (p.n_pad * TC_BOX_K * 2), &map_b, k * TC_TILE_K + kb * TC_BOX_K,
+                        brow, &T.full[s]);
+        } else {
+          pend_s[n_pend] = s; pend_k[n_pend] = k; pend_brow = brow; ++n_pend;
+        }
+        ++issued;
+        if (++s == p.stages) { s = 0; ph ^= 1u; }
+        if (!waited && (issued == p.stages || k == k1 - 1)) settle();
+      }
+    }
+    if (!waited) settle();
+    if (ok) {
+      // the end of the work, for the epilogue warps and for the MMA thread
+      const int qs = qn % TC_ITEM_Q;
+      if (qn >= TC_ITEM_Q)
+        ok = mbar_wait(&T.iq_empty[qs], (uint32_t)(qn / TC_ITEM_Q - 1) & 1u, abort_flag, status);
+      if (ok) {
+        T.q_item[qs] = -1;
+        mbar_arrive(&T.iq_full[qs]);
+        if (issued >= p.stages) ok = mbar_wait(&T.empty[s], ph ^ 1u, abort_flag, status);
+      }
+      if (ok) {
+        T.st_flag[s] = TC_FLAG_END;
+        mbar_arrive(&T.full[s]);
+      }
     }
     if (!ok) {
       // gave up: let the copies already in flight land before the CTA's memory goes away
@@ -242,58 +256,67 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
   } else if (warp == 1 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
     const uint32_t idesc = instr_desc_bf16(p.n_pad);
-    int seg = 0, s = 0;
+    int seg = 0, s = 0, acc = 0;
     uint32_t fph = 0;
-    bool ok = true;
-    long long tile_end = (first_tile + 1) * units_per_tile;
-    for (long long u = u0; u < u1 && ok; ++seg, tile_end += units_per_tile) {
-      const long long ue = tile_end < u1 ? tile_end : u1;
-      const int acc = seg & 1;
-      if (seg >= 2) ok = mbar_wait(&T.acc_empty[acc], ((uint32_t)(seg >> 1) & 1u) ^ 1u, abort_flag, status);
+    bool ok = true, first = true;
+    uint32_t d_addr = tmem_base;
+    while (ok) {
+      ok = mbar_wait(&T.full[s], fph, abort_flag, status);
       if (!ok) break;
-      tc_fence_after();
-      const uint32_t d_addr = tmem_base + (uint32_t)(acc * p.n_pad);
-      bool first = true;
-      for (; u < ue; ++u) {
-        ok = mbar_wait(&T.full[s], fph, abort_flag, status);
+      const int flag = T.st_flag[s];
+      if (flag & TC_FLAG_END) break;
+      if (flag & TC_FLAG_FIRST) {
+        acc = seg & 1;
+        if (seg >= 2)
+          ok = mbar_wait(&T.acc_empty[acc], ((uint32_t)(seg >> 1) & 1u) ^ 1u, abort_flag, status);
         if (!ok) break;
-        tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t b_addr = a_addr + TC_TILE_M * TC_TILE_K * 2;
-#pragma unroll
-        for (int kb = 0; kb < TC_KB; ++kb) {
-          const uint64_t da = smem_desc_sw128(a_addr + kb * (TC_TILE_M * TC_BOX_K * 2));
-          const uint64_t db = smem_desc_sw128(b_addr + kb * (p.n_pad * TC_BOX_K * 2));
-#pragma unroll
-          for (int k = 0; k < TC_BOX_K / 16; ++k) {
-            // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in the address field
-            tc_mma_bf16(d_addr, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
-                        (first && kb == 0 && k == 0) ? 0u : 1u);
-          }
-        }
-        first = false;
-        tc_commit(&T.empty[s]);          // the stage is free once these MMAs have read it
-        if (++s == p.stages) { s = 0; fph ^= 1u; }
+        d_addr = tmem_base + (uint32_t)(acc * p.n_pad);
+        first = true;
       }
-      if (ok) tc_commit(&T.acc_full[acc]);
+      tc_fence_after();
+      const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+      const uint32_t b_addr = a_addr + TC_TILE_M * TC_TILE_K * 2;
+#pragma unroll
+      for (int kb = 0; kb < TC_KB; ++kb) {
+        const uint64_t da = smem_desc_sw128(a_addr + kb * (TC_TILE_M * TC_BOX_K * 2));
+        const uint64_t db = smem_desc_sw128(b_addr + kb * (p.n_pad * TC_BOX_K * 2));
+#pragma unroll
+        for (int k = 0; k < TC_BOX_K / 16; ++k) {
+          // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in the address field
+          tc_mma_bf16(d_addr, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
+                      (first && kb == 0 && k == 0) ? 0u : 1u);
+        }
+      }
+      first = false;
+      tc_commit(&T.empty[s]);          // the stage is free once these MMAs have read it
+      if (flag & TC_FLAG_LAST) {
+        tc_commit(&T.acc_full[acc]);
+        ++seg;
+      }
+      if (++s == p.stages) { s = 0; fph ^= 1u; }
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;        // the TMEM lanes this warp may read: 32*quarter .. +31
     const int m = quarter * 32 + lane;
-    int seg = 0;
+    int seg = 0, qn = 0;
     bool ok = true;
-    for (long long u = u0; u < u1 && ok; ++seg) {
-      const long long tile = u / units_per_tile;
-      const long long tile_end = (tile + 1) * units_per_tile;
-      u = tile_end < u1 ? tile_end : u1;
+    while (ok) {
+      const int qs = qn % TC_ITEM_Q;
+      ok = mbar_wait(&T.iq_full[qs], (uint32_t)(qn / TC_ITEM_Q) & 1u, abort_flag, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const int item = T.q_item[qs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&T.iq_empty[qs]);
+      ++qn;
+      if (item < 0) break;
       const int acc = seg & 1;
       ok = mbar_wait(&T.acc_full[acc], (uint32_t)(seg >> 1) & 1u, abort_flag, status);
       ok = __all_sync(0xffffffffu, ok);          // the TMEM loads below need the whole warp
       if (!ok) break;
       tc_fence_after();
-      const int slot = blockIdx.x * p.max_seg + (int)(tile - first_tile);
-      float* dst = partial + ((size_t)slot * p.n_pad) * TC_TILE_M + m;
+      float* dst = partial + ((size_t)item * p.n_pad) * TC_TILE_M + m;
       const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.n_pad);
       for (int c = 0; c < p.n_pad; c += 16) {
         uint32_t r[16];
@@ -305,6 +328,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&T.acc_empty[acc]);
+      ++seg;
     }
   }
   tc_fence_before();
@@ -316,105 +340,46 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
 }
 
 // ---------------------------------------------------------------------------------------------
-// Fix-up kernels: every output element is the sum of the partial tiles of the CTAs whose spans
-// touched its tile, added in ascending CTA order (fixed order: bitwise reproducible), followed by
-// the epilogue of the contraction.
+// Fix-up kernels: every output element is the sum of the partial tiles of its tile's chunks,
+// added in ascending chunk order (fixed order: bitwise reproducible), followed by the epilogue
+// of the contraction.  The first thread of each also puts the launch's item counter back to zero.
 // ---------------------------------------------------------------------------------------------
-#define TC_MAX_CONTRIB 8
-
-// Partial-tile slots that add up to `tile`, ascending CTA order.  Returns the count, or -1 if
-// there are more than TC_MAX_CONTRIB (then tc_tile_sum_slow is used).
-__device__ __forceinline__ int tc_tile_slots(const tc_params& p, long long total64, int n_cta,
-                                             long long tile, int* slots) {
-  // 32-bit arithmetic (the host checks total * n_cta < 2^31); span starts are stepped from one
-  // CTA to the next with a quotient/remainder pair instead of one division each.
-  const unsigned total = (unsigned)total64, n = (unsigned)n_cta, kt = (unsigned)p.kt;
-  const unsigned a = (unsigned)tile * kt, b = a + kt;
-  const unsigned q = total / n, r = total - q * n;          // start(c + 1) - start(c) = q or q + 1
-  unsigned c = a * n / total;
-  if (c >= n) c = n - 1;
-  unsigned s0 = total * c / n, rem = total * c - s0 * n;     // start(c) and its remainder
-  // step back while this CTA starts after a
-  while (c > 0 && s0 > a) {
-    --c;
-    if (rem >= r) { rem -= r; s0 -= q; } else { rem = rem + n - r; s0 -= q + 1; }
-  }
-  int cnt = 0;
-  for (; c < n; ++c) {
-    if (s0 >= b) break;
-    unsigned s1 = s0 + q, rem1 = rem + r;
-    if (rem1 >= n) { rem1 -= n; ++s1; }
-    if (s1 > a && s1 != s0) {                                 // overlaps the tile and is not empty
-      if (cnt == TC_MAX_CONTRIB) return -1;
-      slots[cnt++] = (int)(c * (unsigned)p.max_seg + ((unsigned)tile - s0 / kt));
-    }
-    s0 = s1;
-    rem = rem1;
-  }
-  return cnt;
-}
-
-__device__ __forceinline__ float tc_tile_sum_slow(const float* __restrict__ partial,
-                                                  const tc_params& p, long long total, int n_cta,
-                                                  long long tile, int n, int m) {
-  const long long a = tile * p.kt, b = a + p.kt;
-  int c = (int)(a * n_cta / total);
-  while (c + 1 < n_cta && tc_span_start(total, c + 1, n_cta) <= a) ++c;
-  while (c > 0 && tc_span_start(total, c, n_cta) > a) --c;
-  float acc = 0.f;
-  for (; c < n_cta; ++c) {
-    const long long s0 = tc_span_start(total, c, n_cta);
-    if (s0 >= b) break;
-    const long long s1 = tc_span_start(total, c + 1, n_cta);
-    if (s1 <= a || s1 == s0) continue;
-    const int slot = c * p.max_seg + (int)(tile - s0 / p.kt);
-    acc += partial[((size_t)slot * p.n_pad + n) * TC_TILE_M + m];
-  }
-  return acc;
-}
-
-struct tc_slot_list {
-  int n;
-  int slot[TC_MAX_CONTRIB];
-};
-
-__device__ __forceinline__ float tc_sum_list(const float* __restrict__ partial, const tc_params& p,
-                                             const tc_slot_list& L, long long total, int n_cta,
+// tile = (index of the group among the active ones) * tiles_per_group + tile of the group
+__device__ __forceinline__ float tc_tile_sum(const float* __restrict__ partial, const tc_params& p,
                                              long long tile, int n, int m) {
-  if (L.n < 0) return tc_tile_sum_slow(partial, p, total, n_cta, tile, n, m);
+  const float* src = partial + (((size_t)tile * p.n_chunks) * p.n_pad + n) * TC_TILE_M + m;
   float acc = 0.f;
-  for (int i = 0; i < L.n; ++i) acc += partial[((size_t)L.slot[i] * p.n_pad + n) * TC_TILE_M + m];
+  for (int c = 0; c < p.n_chunks; ++c) acc += src[(size_t)c * p.n_pad * TC_TILE_M];
   return acc;
+}
+__device__ __forceinline__ void tc_reset_counter(const tc_params& p) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) *p.counter = 0;
 }
 
 // h[e, n, i] = SiLU(gate) * up for every touched expert (Eq. 3's Expert_j, first half).
 // grid (tiles over I, experts, row slices); groups come in (gate, up) pairs.
-__global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int n_cta, int I, int n_rows,
+__global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int I, int n_rows,
                                                      int Rp, const int32_t* __restrict__ expert,
                                                      const float* __restrict__ partial,
                                                      __nv_bfloat16* __restrict__ hbuf) {
   jk_pdl_wait();
   jk_pdl_trigger();
+  tc_reset_counter(p);
   __shared__ tc_plan plan;
-  __shared__ tc_slot_list lg, lu;
   if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
   __syncthreads();
   const int t = blockIdx.x, go = blockIdx.y, m = threadIdx.x;
   if (2 * go + 1 >= plan.n_groups) return;
-  const long long total = plan.total_units;
   const long long tile_g = (long long)(2 * go) * p.tiles_per_group + t;
   const long long tile_u = tile_g + p.tiles_per_group;
-  if (threadIdx.x == 0) lg.n = tc_tile_slots(p, total, n_cta, tile_g, lg.slot);
-  if (threadIdx.x == 32) lu.n = tc_tile_slots(p, total, n_cta, tile_u, lu.slot);
-  __syncthreads();
   const int i = t * TC_TILE_M + m;
   if (i >= I) return;
   const int e = p.group_expert[plan.group_src[2 * go]];
   __nv_bfloat16* o = hbuf + (size_t)e * Rp * I + i;
 #pragma unroll 4
   for (int n = blockIdx.z; n < n_rows; n += gridDim.z) {
-    const float g = tc_sum_list(partial, p, lg, total, n_cta, tile_g, n, m);
-    const float u = tc_sum_list(partial, p, lu, total, n_cta, tile_u, n, m);
+    const float g = tc_tile_sum(partial, p, tile_g, n, m);
+    const float u = tc_tile_sum(partial, p, tile_u, n, m);
     o[(size_t)n * I] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
   }
 }
@@ -422,27 +387,25 @@ __global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int n_ct
 // y_r = W_down h for the K experts of row r, then Eq. 3 and the branch features:
 //   f = u + sum_r g_r y_r,  b_r = g_r y_r (+ u).   grid (tiles over H, rows).
 __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
-    const tc_params p, int n_cta, int H, const int32_t* __restrict__ expert,
+    const tc_params p, int H, const int32_t* __restrict__ expert,
     const float* __restrict__ gate, const __nv_bfloat16* __restrict__ u, int branch_residual,
     int head_mode, float alpha, float beta, const float* __restrict__ partial,
     __nv_bfloat16* __restrict__ bbuf, __nv_bfloat16* __restrict__ out_feat) {
   jk_pdl_wait();
   jk_pdl_trigger();
+  tc_reset_counter(p);
   __shared__ tc_plan plan;
-  __shared__ tc_slot_list lists[JK_MAX_EXPERTS];
   __shared__ long long tiles[JK_MAX_EXPERTS];
   if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
   __syncthreads();
   const int t = blockIdx.x, r = blockIdx.y, m = threadIdx.x;
   const int K = p.K_top;
-  const long long total = plan.total_units;
   if (threadIdx.x < K) {
     const int e = expert[r * K + threadIdx.x];
     int ga = 0;                       // position of expert e among the active groups
     for (int g = 0; g < plan.n_groups; ++g)
       if (p.group_expert[plan.group_src[g]] == e) ga = g;
     tiles[threadIdx.x] = (long long)ga * p.tiles_per_group + t;
-    lists[threadIdx.x].n = tc_tile_slots(p, total, n_cta, tiles[threadIdx.x], lists[threadIdx.x].slot);
   }
   __syncthreads();
   const int h = t * TC_TILE_M + m;
@@ -451,8 +414,8 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
   float f = uv;
   if (head_mode == 1) {
     // contrastive heads (Eq. 6-7): b_0 = f^moe (+ u), b_1 = beta y_1 - alpha y_2 (+ u)
-    const float y0 = tc_sum_list(partial, p, lists[0], total, n_cta, tiles[0], r, m);
-    const float y1 = tc_sum_list(partial, p, lists[1], total, n_cta, tiles[1], r, m);
+    const float y0 = tc_tile_sum(partial, p, tiles[0], r, m);
+    const float y1 = tc_tile_sum(partial, p, tiles[1], r, m);
     const float g0y = gate[r * K] * y0, g1y = gate[r * K + 1] * y1;
     const float fm = g0y + g1y, fc = beta * y0 - alpha * y1;
     f = (uv + g0y) + g1y;
@@ -460,7 +423,7 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
     bbuf[((size_t)r * K + 1) * H + h] = __float2bfloat16_rn(branch_residual ? fc + uv : fc);
   } else {
     for (int k = 0; k < K; ++k) {
-      const float y = tc_sum_list(partial, p, lists[k], total, n_cta, tiles[k], r, m);
+      const float y = tc_tile_sum(partial, p, tiles[k], r, m);
       const float gy = gate[r * K + k] * y;
       f += gy;
       bbuf[((size_t)r * K + k) * H + h] = __float2bfloat16_rn(branch_residual ? gy + uv : gy);
@@ -472,21 +435,14 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
 // logits = b W_head^T (Eq. 4) assembled from the partial tiles, optionally stored, and the
 // per-chunk top-k statistics of jk_topk.cuh.   grid (chunks, logits rows), JK_TOPK_THREADS threads.
 __global__ void __launch_bounds__(JK_TOPK_THREADS, 2) k_tc_fix_lmhead_topk(
-    const tc_params p, int n_cta, int V, int k_e, int chunks, const float* __restrict__ partial,
+    const tc_params p, int V, int k_e, int chunks, const float* __restrict__ partial,
     float* __restrict__ logits, int rows_per_b, long long stride_b, float* __restrict__ tk_val,
     int32_t* __restrict__ tk_idx, float* __restrict__ tk_ms) {
   jk_pdl_wait();
   jk_pdl_trigger();
+  tc_reset_counter(p);
   constexpr int TILES = JK_TOPK_CHUNK / TC_TILE_M;     // 32 tiles per chunk
-  __shared__ tc_slot_list lists[TILES];
   const int chunk = blockIdx.x, row = blockIdx.y;
-  const long long total = (long long)p.tiles_per_group * p.kt;     // one group, always active
-  if (threadIdx.x < TILES) {
-    const long long tile = (long long)chunk * TILES + threadIdx.x;
-    lists[threadIdx.x].n = tile < p.tiles_per_group
-                               ? tc_tile_slots(p, total, n_cta, tile, lists[threadIdx.x].slot) : 0;
-  }
-  __syncthreads();
   const int base = chunk * JK_TOPK_CHUNK;
   float vals[JK_TOPK_PER];
   float* lrow = logits ? logits + (size_t)(row / rows_per_b) * (size_t)stride_b +
@@ -498,7 +454,7 @@ __global__ void __launch_bounds__(JK_TOPK_THREADS, 2) k_tc_fix_lmhead_topk(
     float v = -INFINITY;
     if (idx < V) {
       const int tl = off / TC_TILE_M, m = off % TC_TILE_M;
-      v = tc_sum_list(partial, p, lists[tl], total, n_cta, (long long)chunk * TILES + tl, row, m);
+      v = tc_tile_sum(partial, p, (long long)chunk * TILES + tl, row, m);
       if (lrow) lrow[idx] = v;
     }
     vals[j] = v;
@@ -543,36 +499,49 @@ static int tc_stages(int n_pad, int kb) {
   return s;
 }
 
-static int tc_max_seg(long long max_units, int n_cta, int kt) {
-  const long long span = (max_units + n_cta - 1) / n_cta;
-  return (int)((span + kt - 1) / kt) + 1;
+// Tiling of one contraction: boxes per stage, k steps of a tile, and the cut of a tile's k steps
+// into chunks (the work items).  Chunks are at least 128 KB of weights long and as many as give
+// every CTA a dozen items when all groups are active; more chunks mean more partial tiles.
+struct tc_tiling { int kb, kt, ch, n_chunks; };
+static tc_tiling tc_tile_plan(int kdim, int n_pad, long long tiles_all_groups, int n_cta) {
+  tc_tiling t;
+  t.kb = tc_stages(n_pad, 2) >= TC_KB_WIDE_MIN_STAGES ? 2 : 1;
+  t.kt = (kdim + t.kb * TC_BOX_K - 1) / (t.kb * TC_BOX_K);
+  const int ch_min = 8 / t.kb;                                  // 8 boxes of 128 x 64 bf16 = 128 KB
+  long long want = (12ll * n_cta + tiles_all_groups - 1) / tiles_all_groups;
+  const int most = t.kt / ch_min > 1 ? t.kt / ch_min : 1;
+  if (want > most) want = most;
+  if (want < 1) want = 1;
+  t.ch = (t.kt + (int)want - 1) / (int)want;
+  t.n_chunks = (t.kt + t.ch - 1) / t.ch;
+  return t;
 }
 
-// n_cta * max_seg <= tiles + 3 * n_cta for any grid size up to TC_MAX_GRID.
-static size_t tc_partial_for(long long units, int kt, int n_pad) {
-  return (size_t)(units / kt + 3 * TC_MAX_GRID) * n_pad * TC_TILE_M * sizeof(float);
+static size_t tc_partial_for(long long tiles_all_groups, int kdim, int n_pad) {
+  // (the grid is the SM count, which the sizing does not know: take the chunk count of the
+  // largest grid, which is the largest chunk count)
+  const tc_tiling t = tc_tile_plan(kdim, n_pad, tiles_all_groups, TC_MAX_GRID);
+  return (size_t)tiles_all_groups * t.n_chunks * n_pad * TC_TILE_M * sizeof(float);
 }
 
-// Worst case over the three contractions.
+// Worst case over the contractions.
 size_t jk_tc_partial_bytes(const jk_config& c) {
   const int R = c.max_batch * c.max_frontier;
   const int np1 = (int)jk_align_up(R, 16), np2 = (int)jk_align_up((size_t)R * c.top_k, 16);
-  const int kt_h = (c.hidden + TC_BOX_K - 1) / TC_BOX_K, kt_i = (c.inter + TC_BOX_K - 1) / TC_BOX_K;
   const long long t_i = (c.inter + TC_TILE_M - 1) / TC_TILE_M, t_h = (c.hidden + TC_TILE_M - 1) / TC_TILE_M,
                   t_v = (c.vocab + TC_TILE_M - 1) / TC_TILE_M;
-  size_t a = tc_partial_for(2ll * c.n_experts * t_i * kt_h, kt_h, np1);
-  size_t b = tc_partial_for((long long)c.n_experts * t_h * kt_i, kt_i, np1);
-  size_t d = tc_partial_for(t_v * kt_h, kt_h, np2);
+  size_t a = tc_partial_for(2ll * c.n_experts * t_i, c.hidden, np1);
+  size_t b = tc_partial_for((long long)c.n_experts * t_h, c.inter, np1);
+  size_t d = tc_partial_for(t_v, c.hidden, np2);
   // the draft layer's reduction, QKV and output projections (one group each)
   const int qd = c.n_q_heads * c.head_dim, qkvd = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
-  const int kt_2h = (2 * c.hidden + TC_BOX_K - 1) / TC_BOX_K, kt_q = (qd + TC_BOX_K - 1) / TC_BOX_K;
   const long long t_qkv = (qkvd + TC_TILE_M - 1) / TC_TILE_M;
-  size_t e1 = tc_partial_for(t_h * kt_2h, kt_2h, np1);
+  size_t e1 = tc_partial_for(t_h, 2 * c.hidden, np1);
   // (jk_verify_qkv sends up to 256 tree tokens at a time through the QKV projection)
   int np_v = (int)jk_align_up((size_t)c.max_batch * c.max_tree, 16);
   if (np_v > 256) np_v = 256;
-  size_t e2 = tc_partial_for(t_qkv * kt_h, kt_h, np_v > np1 ? np_v : np1);
-  size_t e3 = tc_partial_for(t_h * kt_q, kt_q, np1);
+  size_t e2 = tc_partial_for(t_qkv, c.hidden, np_v > np1 ? np_v : np1);
+  size_t e3 = tc_partial_for(t_h, qd, np1);
   size_t m = a > b ? a : b;
   m = m > d ? m : d;
   m = m > e1 ? m : e1;
@@ -651,23 +620,26 @@ static bool tc_map(jk_ctx* ctx, tc_state* s, const void* ptr, uint64_t rows, uin
   return true;
 }
 
-// Launch the streaming GEMM; fills the launch-dependent fields of p and returns the grid size.
+// Launch the streaming GEMM; fills the launch-dependent fields of p.  Four item counters take
+// turns: a launch's counter is put back to zero by its own fix-up kernel, well before the same
+// counter is used again four launches later (a GEMM that prefetches reads its counter while the
+// fix-up of the GEMM before it is still running, so that one cannot share it).
 static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUtensorMap* a0,
                           const CUtensorMap* a1, const CUtensorMap* b, tc_params& p,
-                          const int32_t* expert, int stage_id, int* n_cta_out) {
+                          const int32_t* expert, int stage_id) {
   const jk_ws_layout& L = ctx->lay;
   const int n_cta = tc_grid(ctx);
-  p.kb = tc_stages(p.n_pad, 2) >= TC_KB_WIDE_MIN_STAGES ? 2 : 1;
-  p.kt = (p.kdim + p.kb * TC_BOX_K - 1) / (p.kb * TC_BOX_K);
+  const long long tiles_all = (long long)p.n_groups_max * p.tiles_per_group;
+  const tc_tiling t = tc_tile_plan(p.kdim, p.n_pad, tiles_all, n_cta);
+  p.kb = t.kb; p.kt = t.kt; p.ch = t.ch; p.n_chunks = t.n_chunks;
   p.stages = tc_stages(p.n_pad, p.kb);
-  const long long max_units = (long long)p.n_groups_max * p.tiles_per_group * p.kt;
-  p.max_seg = tc_max_seg(max_units, n_cta, p.kt);
-  if (max_units * TC_MAX_GRID >= (1ll << 31)) return JK_ERR_SHAPE;   // 32-bit span arithmetic
+  if (tiles_all * p.n_chunks >= (1ll << 30)) return JK_ERR_SHAPE;    // item ids are 32-bit
   int cols = 32;
   while (cols < 2 * p.n_pad) cols <<= 1;
   p.tmem_cols = cols;
-  if ((size_t)n_cta * p.max_seg * p.n_pad * TC_TILE_M * sizeof(float) > L.gemm_part_bytes)
+  if ((size_t)tiles_all * p.n_chunks * p.n_pad * TC_TILE_M * sizeof(float) > L.gemm_part_bytes)
     return JK_ERR_WORKSPACE;
+  p.counter = (int*)(ctx->ws + L.gemm_cnt) + (ctx->gemm_seq++ & 3);
   const size_t smem = (size_t)p.stages * tc_stage_bytes(p.n_pad, p.kb) + sizeof(tc_smem_tail) + 1024;
   if (!s->smem_set) {
     JK_CUDA_CHECK(ctx, cudaFuncSetAttribute(k_tc_gemm<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -684,7 +656,6 @@ static int tc_launch_gemm(jk_ctx* ctx, cudaStream_t st, tc_state* s, const CUten
     jk_launch_pdl(k_tc_gemm<1>, dim3(n_cta), dim3(TC_THREADS), smem, st, *a0, *a1, *b, p, expert,
                   (float*)(ctx->ws + L.gemm_part), (int32_t*)(ctx->ws + L.status));
   JK_LAUNCH_CHECK(ctx);
-  *n_cta_out = n_cta;
   return JK_OK;
 }
 
@@ -702,7 +673,6 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   memset(&p, 0, sizeof(p));
   p.R = R; p.K_top = c.top_k; p.n_experts = N;
   const int n_pad = (int)jk_align_up(R, 16);
-  int n_cta = 0;
   // gate / up
   CUtensorMap ag, au, bx;
   if (!tc_map(ctx, s, w->w_gate, (uint64_t)N * I, H, TC_TILE_M, &ag) ||
@@ -718,11 +688,11 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   p.tiles_per_group = (I + TC_TILE_M - 1) / TC_TILE_M;
   p.kdim = H;
   p.n_pad = n_pad;
-  int rc = tc_launch_gemm(ctx, st, s, &ag, &au, &bx, p, expert, JK_ST_GATEUP, &n_cta);
+  int rc = tc_launch_gemm(ctx, st, s, &ag, &au, &bx, p, expert, JK_ST_GATEUP);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_GEMM_FIXUP);
   jk_launch_pdl(k_tc_fix_silu, dim3(p.tiles_per_group, N, R), dim3(128), 0, st, 
-      p, n_cta, I, R, Rp, expert, partial, (__nv_bfloat16*)(ctx->ws + L.hbuf));
+      p, I, R, Rp, expert, partial, (__nv_bfloat16*)(ctx->ws + L.hbuf));
   JK_LAUNCH_CHECK(ctx);
   // down
   CUtensorMap ad, bh;
@@ -736,11 +706,11 @@ int jk_tc_ffn(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R,
   p.tiles_per_group = (H + TC_TILE_M - 1) / TC_TILE_M;
   p.kdim = I;
   p.prefetch = 1;
-  rc = tc_launch_gemm(ctx, st, s, &ad, &ad, &bh, p, expert, JK_ST_DOWN, &n_cta);
+  rc = tc_launch_gemm(ctx, st, s, &ad, &ad, &bh, p, expert, JK_ST_DOWN);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_BRANCH);
   jk_launch_pdl(k_tc_fix_down_branch, dim3(p.tiles_per_group, R), dim3(128), 0, st, 
-      p, n_cta, H, expert, gate, (const __nv_bfloat16*)u, c.branch_residual, c.head_mode,
+      p, H, expert, gate, (const __nv_bfloat16*)u, c.branch_residual, c.head_mode,
       c.contrast_alpha, c.contrast_beta, partial,
       (__nv_bfloat16*)(ctx->ws + L.bbuf), (__nv_bfloat16*)out_feat);
   JK_LAUNCH_CHECK(ctx);
@@ -769,13 +739,12 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
   p.tiles_per_group = (V + TC_TILE_M - 1) / TC_TILE_M;
   p.kdim = H;
   p.n_pad = n_pad;
-  int n_cta = 0;
   p.prefetch = 1;
-  int rc = tc_launch_gemm(ctx, st, s, &ah, &ah, &bb, p, nullptr, JK_ST_LMHEAD, &n_cta);
+  int rc = tc_launch_gemm(ctx, st, s, &ah, &ah, &bb, p, nullptr, JK_ST_LMHEAD);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_TOPK);
   jk_launch_pdl(k_tc_fix_lmhead_topk, dim3(L.topk_chunks, RK), dim3(JK_TOPK_THREADS), 0, st, 
-      p, n_cta, V, c.k_per_expert, L.topk_chunks, (const float*)(ctx->ws + L.gemm_part), logits,
+      p, V, c.k_per_expert, L.topk_chunks, (const float*)(ctx->ws + L.gemm_part), logits,
       rows_per_b, logits_stride_b, (float*)(ctx->ws + L.tk_val), (int32_t*)(ctx->ws + L.tk_idx),
       (float*)(ctx->ws + L.tk_ms));
   JK_LAUNCH_CHECK(ctx);
@@ -788,20 +757,17 @@ int jk_tc_lm_head(jk_ctx* ctx, cudaStream_t st, const jk_draft_weights* w, int R
 // ---------------------------------------------------------------------------------------------
 // grid (tiles over the M output features, rows); one of out_bf16 / out_f32 is written
 __global__ void __launch_bounds__(128) k_tc_fix_linear(
-    const tc_params p, int n_cta, int Mrows, const float* __restrict__ partial,
+    const tc_params p, int Mrows, const float* __restrict__ partial,
     const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ resid,
     long long resid_ld, __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32,
     long long out_ld) {
   jk_pdl_wait();
   jk_pdl_trigger();
-  __shared__ tc_slot_list list;
+  tc_reset_counter(p);
   const int t = blockIdx.x, r = blockIdx.y, m = threadIdx.x;
-  const long long total = (long long)p.tiles_per_group * p.kt;     // one group, always active
-  if (threadIdx.x == 0) list.n = tc_tile_slots(p, total, n_cta, t, list.slot);
-  __syncthreads();
   const int o = t * TC_TILE_M + m;
   if (o >= Mrows) return;
-  float v = tc_sum_list(partial, p, list, total, n_cta, t, r, m);
+  float v = tc_tile_sum(partial, p, t, r, m);
   if (bias) v += __bfloat162float(bias[o]);
   if (resid) v += __bfloat162float(resid[(size_t)r * resid_ld + o]);
   if (out_bf16) out_bf16[(size_t)r * out_ld + o] = __float2bfloat16_rn(v);
@@ -830,11 +796,10 @@ int jk_tc_linear(jk_ctx* ctx, cudaStream_t st, const void* W, int Mrows, int Kdi
   p.kdim = Kdim;
   p.n_pad = n_pad;
   p.prefetch = 1;
-  int n_cta = 0;
-  int rc = tc_launch_gemm(ctx, st, s, &aw, &aw, &bx, p, nullptr, JK_ST_PRE_GEMM, &n_cta);
+  int rc = tc_launch_gemm(ctx, st, s, &aw, &aw, &bx, p, nullptr, JK_ST_PRE_GEMM);
   if (rc != JK_OK) return rc;
   JK_PROF(ctx, st, JK_ST_PRE_FIXUP);
-  jk_launch_pdl(k_tc_fix_linear, dim3(p.tiles_per_group, n_rows), dim3(128), 0, st, p, n_cta, Mrows,
+  jk_launch_pdl(k_tc_fix_linear, dim3(p.tiles_per_group, n_rows), dim3(128), 0, st, p, Mrows,
                 (const float*)(ctx->ws + L.gemm_part), (const __nv_bfloat16*)bias,
                 (const __nv_bfloat16*)resid, resid_ld, (__nv_bfloat16*)out_bf16, out_f32, out_ld);
   JK_LAUNCH_CHECK(ctx);

@@ -6,8 +6,10 @@ one expire there.  What can be checked without a GPU is the protocol itself: eve
 budget; the role whose wait runs out records JK_ERR_TIMEOUT once, raises the CTA's abort flag and
 returns; every other role notices the flag at its next wait and returns too; the common exit path
 (drain the copies in flight, free the tensor memory) is reached by all of them.  The model below
-follows the roles of the streaming GEMM one to one - same barriers, same arrival counts, same
-parities - and the failure is injected on the host by under-filling one arrival count."""
+follows the roles of the streaming GEMM - producer, MMA issuer, four epilogue warps, the stage ring
+and the two accumulators with their arrival counts and parities (the kernel's small queue of item
+ids between producer and epilogue warps follows the same pattern and is left out) - and the
+failure is injected on the host by under-filling one arrival count."""
 import itertools
 
 JK_ERR_TIMEOUT = -8
