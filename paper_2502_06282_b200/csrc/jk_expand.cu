@@ -365,12 +365,7 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
         if (!(taken & (1u << j)) && jk_better(cv[j], ci[j], bv, bi)) { bv = cv[j]; bi = ci[j]; bj = j; }
       float wv = bv;
       int wi = bi;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, wv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, wi, o);
-        if (jk_better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
-      }
+      jk_warp_argbest(wv, wi);
       if (wi == bi && bj >= 0 && wi != INT_MAX) taken |= 1u << bj;
       if (lane == 0) {
         const int flat = lr * k_e + it;

@@ -501,14 +501,16 @@ static int tc_stages(int n_pad, int kb) {
 
 // Tiling of one contraction: boxes per stage, k steps of a tile, and the cut of a tile's k steps
 // into chunks (the work items).  Chunks are at least 128 KB of weights long and as many as give
-// every CTA a dozen items when all groups are active; more chunks mean more partial tiles.
+// every CTA about six items when all groups are active: more chunks balance the CTAs better but
+// mean more partial tiles for the fix-up kernels to add up, and those sit on the critical path
+// (measured at the 7B shape: 3-4 items per CTA 519, 6 items 532, 12 items 531, 24 items 524 steps/s).
 struct tc_tiling { int kb, kt, ch, n_chunks; };
 static tc_tiling tc_tile_plan(int kdim, int n_pad, long long tiles_all_groups, int n_cta) {
   tc_tiling t;
   t.kb = tc_stages(n_pad, 2) >= TC_KB_WIDE_MIN_STAGES ? 2 : 1;
   t.kt = (kdim + t.kb * TC_BOX_K - 1) / (t.kb * TC_BOX_K);
   const int ch_min = 8 / t.kb;                                  // 8 boxes of 128 x 64 bf16 = 128 KB
-  long long want = (12ll * n_cta + tiles_all_groups - 1) / tiles_all_groups;
+  long long want = (6ll * n_cta + tiles_all_groups - 1) / tiles_all_groups;
   const int most = t.kt / ch_min > 1 ? t.kt / ch_min : 1;
   if (want > most) want = most;
   if (want < 1) want = 1;

@@ -16,13 +16,23 @@
 #define JK_TOPK_WARPS (JK_TOPK_THREADS / 32)
 #define JK_TOPK_PER (JK_TOPK_CHUNK / JK_TOPK_THREADS)
 
+// Order-preserving map of a float (finite or -inf) to an unsigned key, and back.  -0 is folded
+// into +0 first, as the comparison of the values themselves does.
+__device__ __forceinline__ unsigned jk_fkey(float v) {
+  const unsigned u = __float_as_uint(v + 0.f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float jk_fkey_inv(unsigned k) {
+  return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+// The warp's best (value descending, index ascending) with two hardware reductions instead of a
+// shuffle tree: the largest key, then the smallest index among the lanes that hold it.
 __device__ __forceinline__ void jk_warp_argbest(float& v, int& i) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, i, o);
-    if (jk_better(ov, oi, v, i)) { v = ov; i = oi; }
-  }
+  const unsigned key = jk_fkey(v);
+  const unsigned kmax = __reduce_max_sync(0xffffffffu, key);
+  const unsigned imin = __reduce_min_sync(0xffffffffu, key == kmax ? (unsigned)i : 0xffffffffu);
+  v = jk_fkey_inv(kmax);
+  i = (int)imin;
 }
 
 // JK_TOPK_THREADS threads; thread t holds entries base + t + j*JK_TOPK_THREADS in vals[j]
