@@ -352,6 +352,35 @@ __device__ __forceinline__ float tc_tile_sum(const float* __restrict__ partial, 
   for (int c = 0; c < p.n_chunks; ++c) acc += src[(size_t)c * p.n_pad * TC_TILE_M];
   return acc;
 }
+// NV such sums at once: the loads of two chunks of all NV sums are in flight together (a loop
+// per sum would pay one trip to the L2 per chunk and sum, one after the other); every sum still
+// adds its chunks in ascending order.  tiles[v] < 0: that sum is skipped (stays 0).
+template <int NV>
+__device__ __forceinline__ void tc_tile_sums(const float* __restrict__ partial, const tc_params& p,
+                                             const long long (&tiles)[NV], int n, int m,
+                                             float (&acc)[NV]) {
+  const size_t stride = (size_t)p.n_pad * TC_TILE_M;
+  const float* src[NV];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    acc[v] = 0.f;
+    src[v] = partial + (((size_t)(tiles[v] < 0 ? 0 : tiles[v]) * p.n_chunks) * p.n_pad + n) * TC_TILE_M + m;
+  }
+  for (int c = 0; c < p.n_chunks; c += 2) {
+    float a[NV], b[NV];
+    const bool two = c + 1 < p.n_chunks;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      a[v] = tiles[v] < 0 ? 0.f : src[v][(size_t)c * stride];
+      b[v] = (tiles[v] < 0 || !two) ? 0.f : src[v][(size_t)(c + 1) * stride];
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      acc[v] += a[v];
+      if (two) acc[v] += b[v];
+    }
+  }
+}
 __device__ __forceinline__ void tc_reset_counter(const tc_params& p) {
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) *p.counter = 0;
 }
@@ -378,8 +407,10 @@ __global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int I, i
   __nv_bfloat16* o = hbuf + (size_t)e * Rp * I + i;
 #pragma unroll 4
   for (int n = blockIdx.z; n < n_rows; n += gridDim.z) {
-    const float g = tc_tile_sum(partial, p, tile_g, n, m);
-    const float u = tc_tile_sum(partial, p, tile_u, n, m);
+    const long long tl[2] = {tile_g, tile_u};
+    float gu[2];
+    tc_tile_sums<2>(partial, p, tl, n, m, gu);
+    const float g = gu[0], u = gu[1];
     o[(size_t)n * I] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
   }
 }
@@ -414,16 +445,25 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
   float f = uv;
   if (head_mode == 1) {
     // contrastive heads (Eq. 6-7): b_0 = f^moe (+ u), b_1 = beta y_1 - alpha y_2 (+ u)
-    const float y0 = tc_tile_sum(partial, p, tiles[0], r, m);
-    const float y1 = tc_tile_sum(partial, p, tiles[1], r, m);
+    const long long tl[2] = {tiles[0], tiles[1]};
+    float yy[2];
+    tc_tile_sums<2>(partial, p, tl, r, m, yy);
+    const float y0 = yy[0], y1 = yy[1];
     const float g0y = gate[r * K] * y0, g1y = gate[r * K + 1] * y1;
     const float fm = g0y + g1y, fc = beta * y0 - alpha * y1;
     f = (uv + g0y) + g1y;
     bbuf[((size_t)r * K) * H + h] = __float2bfloat16_rn(branch_residual ? fm + uv : fm);
     bbuf[((size_t)r * K + 1) * H + h] = __float2bfloat16_rn(branch_residual ? fc + uv : fc);
   } else {
-    for (int k = 0; k < K; ++k) {
-      const float y = tc_tile_sum(partial, p, tiles[k], r, m);
+    long long tl[JK_MAX_EXPERTS];
+    float ys[JK_MAX_EXPERTS];
+#pragma unroll
+    for (int k = 0; k < JK_MAX_EXPERTS; ++k) tl[k] = k < K ? tiles[k] : -1;
+    tc_tile_sums<JK_MAX_EXPERTS>(partial, p, tl, r, m, ys);
+#pragma unroll
+    for (int k = 0; k < JK_MAX_EXPERTS; ++k) {
+      if (k >= K) break;
+      const float y = ys[k];
       const float gy = gate[r * K + k] * y;
       f += gy;
       bbuf[((size_t)r * K + k) * H + h] = __float2bfloat16_rn(branch_residual ? gy + uv : gy);
@@ -447,17 +487,19 @@ __global__ void __launch_bounds__(JK_TOPK_THREADS, 2) k_tc_fix_lmhead_topk(
   float vals[JK_TOPK_PER];
   float* lrow = logits ? logits + (size_t)(row / rows_per_b) * (size_t)stride_b +
                              (size_t)(row % rows_per_b) * V : nullptr;
+  // thread t owns entries t, t + 512, ...: the same column m of JK_TOPK_PER different tiles
+  long long tl[JK_TOPK_PER];
 #pragma unroll
   for (int j = 0; j < JK_TOPK_PER; ++j) {
     const int off = threadIdx.x + j * JK_TOPK_THREADS; // within the chunk
-    const int idx = base + off;
-    float v = -INFINITY;
-    if (idx < V) {
-      const int tl = off / TC_TILE_M, m = off % TC_TILE_M;
-      v = tc_tile_sum(partial, p, (long long)chunk * TILES + tl, row, m);
-      if (lrow) lrow[idx] = v;
-    }
-    vals[j] = v;
+    tl[j] = base + off < V ? (long long)chunk * TILES + off / TC_TILE_M : -1;
+  }
+  tc_tile_sums<JK_TOPK_PER>(partial, p, tl, row, threadIdx.x % TC_TILE_M, vals);
+#pragma unroll
+  for (int j = 0; j < JK_TOPK_PER; ++j) {
+    const int idx = base + threadIdx.x + j * JK_TOPK_THREADS;
+    if (idx < V) { if (lrow) lrow[idx] = vals[j]; }
+    else vals[j] = -INFINITY;
   }
   jk_topk_chunk_select(vals, base, V, k_e, (size_t)row * chunks + chunk, tk_val, tk_idx, tk_ms);
 }
