@@ -215,6 +215,28 @@ def test_expand_planted_ties(name, tensor_path):
     _check_tree(w, pool, bufs, 5)
 
 
+@pytest.mark.parametrize("name,tensor_path", [("tiny", None), ("tiny_bf16", True)])
+def test_expand_many_equal_logits(name, tensor_path):
+    """Three hundred vocabulary rows of the LM head made identical to the root's best token: more
+    entries reach the chunk's selection threshold than its short candidate list holds, so the
+    full selection runs instead, and the tie rule (lower token id first) decides the top-k."""
+    w = synth.WORKLOADS[name]
+    assert w.vocab >= 400
+    wts, us = _inputs(w)
+    _, first = _run_gpu(w, wts, us, tensor_path)
+    t1 = int(host(first.pool["tok"])[0, 0])
+    wts["lm_head"] = wts["lm_head"].copy()
+    wts["lm_head"][40:340] = wts["lm_head"][t1]
+    ctx, bufs = _run_gpu(w, wts, us, tensor_path)
+    lg = host(bufs.logits)[0, 0, 0]
+    assert np.all(lg[40:340] == lg[t1])
+    pool = _check_layers(w, wts, us, bufs)
+    ke = w.k_per_expert
+    want = sorted(set(range(40, 340)) | {t1})[:ke]
+    assert pool["tok"][0, :ke].tolist() == want
+    _check_tree(w, pool, bufs, 5)
+
+
 def test_expand_tensor_path_row_limit_and_fallback():
     """128 activation rows with K = 2 give 256 logits rows, the most the tensor-core GEMM takes
     (two accumulators of 256 columns fill the tensor memory); with K = 3 the same rows give 384,
