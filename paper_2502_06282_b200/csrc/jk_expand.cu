@@ -26,6 +26,16 @@ __global__ void __launch_bounds__(512) k_router(
     const T* __restrict__ u, const T* __restrict__ router, const T* __restrict__ norm_w,
     int H, int N, int K, float eps, int use_norm, T* __restrict__ xn,
     float* __restrict__ out_probs, int32_t* __restrict__ out_expert, float* __restrict__ out_gate) {
+  // The weights do not depend on the kernel before: ask for this thread's pieces of them (into
+  // the L2) ahead of the dependency wait, so that only u is fetched after it.
+  {
+    constexpr int VNP = jk_vec<T>::N;
+    for (int k = threadIdx.x * VNP; k < H; k += blockDim.x * VNP) {
+      if (use_norm && norm_w) asm volatile("prefetch.global.L2 [%0];" ::"l"(norm_w + k));
+      for (int j = 0; j < N; ++j)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(router + (size_t)j * H + k));
+    }
+  }
   jk_pdl_wait();
   jk_pdl_trigger();
   // One pass over the row: the sum of squares and the N centroid dot products of u * gamma are

@@ -83,7 +83,7 @@ __device__ __forceinline__ void tc_make_plan(const tc_params& p, const int32_t* 
   // called by one whole warp; lane 0 writes the plan
   unsigned active = 0;
   for (int i = threadIdx.x & 31; i < p.R * p.K_top; i += 32) {
-    const int e = expert[i];
+    const int e = __ldcg(expert + i);      // (past the L1: some callers read it before their wait)
     if (e >= 0 && e < p.n_experts) active |= 1u << e;
   }
   active = __reduce_or_sync(0xffffffffu, active);
@@ -391,12 +391,14 @@ __global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int I, i
                                                      int Rp, const int32_t* __restrict__ expert,
                                                      const float* __restrict__ partial,
                                                      __nv_bfloat16* __restrict__ hbuf) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
-  tc_reset_counter(p);
+  // The router's output is older than the GEMM this kernel follows (a kernel releases its
+  // successor only after its own wait), so the plan can be made while that GEMM still runs.
   __shared__ tc_plan plan;
   if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
   __syncthreads();
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  tc_reset_counter(p);
   const int t = blockIdx.x, go = blockIdx.y, m = threadIdx.x;
   if (2 * go + 1 >= plan.n_groups) return;
   const long long tile_g = (long long)(2 * go) * p.tiles_per_group + t;
@@ -422,26 +424,31 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
     const float* __restrict__ gate, const __nv_bfloat16* __restrict__ u, int branch_residual,
     int head_mode, float alpha, float beta, const float* __restrict__ partial,
     __nv_bfloat16* __restrict__ bbuf, __nv_bfloat16* __restrict__ out_feat) {
-  jk_pdl_wait();
-  jk_pdl_trigger();
-  tc_reset_counter(p);
+  // Everything but the partial tiles is older than the GEMM this kernel follows (the router's
+  // output, the caller's u): it is fetched, past the L1, while that GEMM still runs.
   __shared__ tc_plan plan;
   __shared__ long long tiles[JK_MAX_EXPERTS];
+  __shared__ float s_gate[JK_MAX_EXPERTS];
   if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
   __syncthreads();
   const int t = blockIdx.x, r = blockIdx.y, m = threadIdx.x;
   const int K = p.K_top;
   if (threadIdx.x < K) {
-    const int e = expert[r * K + threadIdx.x];
+    const int e = __ldcg(expert + r * K + threadIdx.x);
     int ga = 0;                       // position of expert e among the active groups
     for (int g = 0; g < plan.n_groups; ++g)
       if (p.group_expert[plan.group_src[g]] == e) ga = g;
     tiles[threadIdx.x] = (long long)ga * p.tiles_per_group + t;
+    s_gate[threadIdx.x] = __ldcg(gate + r * K + threadIdx.x);
   }
-  __syncthreads();
   const int h = t * TC_TILE_M + m;
+  const unsigned short u_bits = h < H ? __ldcg(reinterpret_cast<const unsigned short*>(u) + (size_t)r * H + h) : 0;
+  __syncthreads();
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  tc_reset_counter(p);
   if (h >= H) return;
-  const float uv = __bfloat162float(u[(size_t)r * H + h]);
+  const float uv = __uint_as_float((unsigned)u_bits << 16);
   float f = uv;
   if (head_mode == 1) {
     // contrastive heads (Eq. 6-7): b_0 = f^moe (+ u), b_1 = beta y_1 - alpha y_2 (+ u)
@@ -449,7 +456,7 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
     float yy[2];
     tc_tile_sums<2>(partial, p, tl, r, m, yy);
     const float y0 = yy[0], y1 = yy[1];
-    const float g0y = gate[r * K] * y0, g1y = gate[r * K + 1] * y1;
+    const float g0y = s_gate[0] * y0, g1y = s_gate[1] * y1;
     const float fm = g0y + g1y, fc = beta * y0 - alpha * y1;
     f = (uv + g0y) + g1y;
     bbuf[((size_t)r * K) * H + h] = __float2bfloat16_rn(branch_residual ? fm + uv : fm);
@@ -464,7 +471,7 @@ __global__ void __launch_bounds__(128) k_tc_fix_down_branch(
     for (int k = 0; k < JK_MAX_EXPERTS; ++k) {
       if (k >= K) break;
       const float y = ys[k];
-      const float gy = gate[r * K + k] * y;
+      const float gy = s_gate[k] * y;
       f += gy;
       bbuf[((size_t)r * K + k) * H + h] = __float2bfloat16_rn(branch_residual ? gy + uv : gy);
     }
