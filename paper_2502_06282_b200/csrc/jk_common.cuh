@@ -135,7 +135,9 @@ int jk_ensure_device_info(jk_ctx* ctx);
 // serialization attribute, a kernel may start while its predecessor is still running; it must
 // call jk_pdl_wait() before it reads or writes global memory that an earlier kernel of the
 // stream touches, and it calls jk_pdl_trigger() only after that wait, so that at most two
-// consecutive kernels overlap and everything older is complete when a kernel starts.
+// consecutive kernels overlap and everything older is complete when a kernel starts.  (One
+// kernel, the SiLU fix-up between the gate/up and the down GEMM, releases its successor before
+// its wait; the reasons why that is sound there are given at that call.)
 __device__ __forceinline__ void jk_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void jk_pdl_trigger() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

@@ -188,8 +188,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_tc_gemm(
       n_pend = 0;
       waited = true;
     };
+    // A CTA's first item is its own number (no trip to the counter before the first copies are
+    // on their way); further items come from the counter, which counts from the grid size up.
+    bool first_item = true;
     while (ok) {
-      const int item = atomicAdd(p.counter, 1);
+      const int item = first_item ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(p.counter, 1);
+      first_item = false;
       if (item >= total) break;
       // the epilogue warps learn the item (its partial slot) through a small queue
       const int qs = qn % TC_ITEM_Q;
@@ -396,8 +400,15 @@ __global__ void __launch_bounds__(128) k_tc_fix_silu(const tc_params p, int I, i
   __shared__ tc_plan plan;
   if (threadIdx.x < 32) tc_make_plan(p, expert, &plan);
   __syncthreads();
-  jk_pdl_wait();
+  // This kernel has more blocks than fit the SMs at once, so its last blocks start late; if the
+  // successor (the down GEMM) were released only after each block's wait, it would be launched
+  // when this kernel is nearly over and could not stream its first weights meanwhile.  It is
+  // released before the wait instead.  That is sound here: ahead of its own wait the down GEMM
+  // reads only weights, the router's output (complete before the gate/up GEMM started) and its
+  // own item counter, and it needs all of an SM's shared memory, so it gets onto an SM only when
+  // the gate/up GEMM's CTA there has left; everything it writes comes after its wait.
   jk_pdl_trigger();
+  jk_pdl_wait();
   tc_reset_counter(p);
   const int t = blockIdx.x, go = blockIdx.y, m = threadIdx.x;
   if (2 * go + 1 >= plan.n_groups) return;
