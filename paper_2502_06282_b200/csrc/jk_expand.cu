@@ -6,6 +6,7 @@
 // jk_gemm_tc.cu (bf16).  Everything around them (router, activation, residuals, top-k, frontier)
 // is shared.
 #include <limits.h>
+#include <type_traits>
 #include <math.h>
 
 #include "jk_common.cuh"
@@ -344,13 +345,15 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
   const int rows = F * K;
   const size_t pb = (size_t)b * pool.stride_b;
   const int nc = chunks * k_e;
-  for (int lr = warp; lr < rows; lr += nw) {
+  // One warp per logits row.  PER = candidates a lane holds (the chunks' partial winners); the
+  // selection loop is instantiated for the smallest PER that covers them.
+  auto merge_row = [&](auto per_tag, int lr) {
+    constexpr int PER = decltype(per_tag)::value;
     const size_t row = (size_t)b * rows + lr;
-    // candidates of this row: the chunks' partial winners (loaded once)
-    float cv[PER_MAX];
-    int ci[PER_MAX];
+    float cv[PER];
+    int ci[PER];
 #pragma unroll
-    for (int j = 0; j < PER_MAX; ++j) {
+    for (int j = 0; j < PER; ++j) {
       const int c = lane + j * 32;
       cv[j] = c < nc ? tk_val[row * nc + c] : -INFINITY;
       ci[j] = c < nc ? tk_idx[row * nc + c] : INT_MAX;
@@ -371,7 +374,7 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
       float bv = -INFINITY;
       int bi = INT_MAX, bj = -1;
 #pragma unroll
-      for (int j = 0; j < PER_MAX; ++j)
+      for (int j = 0; j < PER; ++j)
         if (!(taken & (1u << j)) && jk_better(cv[j], ci[j], bv, bi)) { bv = cv[j]; bi = ci[j]; bj = j; }
       float wv = bv;
       int wi = bi;
@@ -383,6 +386,12 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
         tk[flat] = wi;
       }
     }
+  };
+  for (int lr = warp; lr < rows; lr += nw) {
+    if (nc <= 64) merge_row(std::integral_constant<int, 2>{}, lr);
+    else if (nc <= 128) merge_row(std::integral_constant<int, 4>{}, lr);
+    else if (nc <= 256) merge_row(std::integral_constant<int, 8>{}, lr);
+    else merge_row(std::integral_constant<int, PER_MAX>{}, lr);
   }
   __syncthreads();
   const int n = rows * k_e;
