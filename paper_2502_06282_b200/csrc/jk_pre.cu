@@ -115,15 +115,23 @@ __global__ void __launch_bounds__(256) k_linear(
 
 // Rotary positions (LLaMA convention: pair (i, i + d/2) turns by pos / theta^(2i/d), pos = prefix
 // length + depth of the node), the rotated query kept per slot, K and V appended to the draft
-// layer's cache at row prefix length + slot.  One block per node; the angle is formed in double
-// precision (a position of several thousand times a frequency near one loses the tolerance in
-// fp32).
+// layer's cache at row prefix length + slot.  One block per node; the angle is formed and reduced
+// in double precision (a position of several thousand times a frequency near one loses the
+// tolerance in fp32).
 template <typename T>
 __global__ void __launch_bounds__(256) k_pre_rope_scatter(
     const float* __restrict__ qkv, int F, int Hq, int Hkv, int D, float theta,
     const int32_t* __restrict__ kv_len, const int32_t* __restrict__ slot_depth, int slot_base,
     long long slot_stride, T* __restrict__ q_slots, T* __restrict__ k_cache, T* __restrict__ v_cache,
     long long cache_sb, long long cache_sh, int cache_rows, int32_t* status) {
+  // The frequencies theta^(-2j/d) in double precision, once per block and ahead of the
+  // dependency wait (they depend on nothing); per pair the angle is then one double product,
+  // reduced to [-pi, pi] in double, and only the sine and cosine of the small remainder are
+  // taken in single precision.
+  __shared__ double s_inv[64];                     // head size 64 or 128
+  for (int j = threadIdx.x; j < D / 2; j += blockDim.x)
+    s_inv[j] = pow((double)theta, -2.0 * (double)j / (double)D);
+  __syncthreads();
   jk_pdl_wait();
   jk_pdl_trigger();
   const int r = blockIdx.x, b = r / F, f = r % F;
@@ -140,12 +148,15 @@ __global__ void __launch_bounds__(256) k_pre_rope_scatter(
   const int n_rot = (Hq + Hkv) * half;               // rotated pairs: all q heads, then all k heads
   for (int i = threadIdx.x; i < n_rot; i += blockDim.x) {
     const int head = i / half, j = i % half;
-    const double ang = pos * pow((double)theta, -2.0 * (double)j / (double)D);
-    double sn, cs;
-    sincos(ang, &sn, &cs);
+    const double ang = pos * s_inv[j];
+    const double turns = rint(ang * 0.15915494309189535);            // 1 / (2 pi)
+    double red = fma(-turns, 6.283185307179586, ang);                // 2 pi, leading part
+    red = fma(-turns, 2.4492935982947064e-16, red);                  // 2 pi, the rest
+    float sn, cs;
+    sincosf((float)red, &sn, &cs);
     const float x1 = row[head * D + j], x2 = row[head * D + half + j];
-    const float o1 = (float)((double)x1 * cs - (double)x2 * sn);
-    const float o2 = (float)((double)x2 * cs + (double)x1 * sn);
+    const float o1 = x1 * cs - x2 * sn;
+    const float o2 = x2 * cs + x1 * sn;
     if (head < Hq) {
       T* dst = q_slots + (((size_t)b * slot_stride + slot) * Hq + head) * D;
       dst[j] = jk_from_float<T>(o1);
@@ -253,10 +264,17 @@ static int pre_impl(jk_ctx* ctx, cudaStream_t st, const jk_pre_weights* w, const
                 theta, kv_len, (const int32_t*)s->slot_depth, slot_base, (long long)s->stride_b,
                 (T*)s->q, (T*)k_cache, (T*)v_cache, (long long)sb, (long long)sh, cache_rows, status);
   JK_LAUNCH_CHECK(ctx);
-  JK_PROF(ctx, st, JK_ST_PRE_ROPE);
-  jk_launch_pdl(k_pre_dense<T>, dim3(B * M), dim3(256), 0, st, (const T*)s->q,
-                (const int32_t*)s->slot_parent, (long long)s->stride_b, M, qd, q_dense, par_dense);
-  JK_LAUNCH_CHECK(ctx);
+  // With one sequence the slots of the nodes expanded so far already are a dense [M, Hq, d]
+  // array (and their parents a dense list): the attention call reads them where they are.
+  if (B == 1) {
+    q_dense = (T*)s->q;
+    par_dense = s->slot_parent;
+  } else {
+    JK_PROF(ctx, st, JK_ST_PRE_ROPE);
+    jk_launch_pdl(k_pre_dense<T>, dim3(B * M), dim3(256), 0, st, (const T*)s->q,
+                  (const int32_t*)s->slot_parent, (long long)s->stride_b, M, qd, q_dense, par_dense);
+    JK_LAUNCH_CHECK(ctx);
+  }
   // Attn over the committed prefix and each node's ancestors
   ctx->st_attn = JK_ST_PRE_ATTN;
   ctx->st_combine = JK_ST_PRE_ATTN_COMBINE;
@@ -265,10 +283,15 @@ static int pre_impl(jk_ctx* ctx, cudaStream_t st, const jk_pre_weights* w, const
   ctx->st_attn = JK_ST_ATTN;
   ctx->st_combine = JK_ST_ATTN_COMBINE;
   if (rc != JK_OK) return rc;
+  // u = W_o Attn + h.  With one sequence this pass's rows of the attention output are
+  // contiguous and feed the projection where they are (rows past the last are zero-filled by
+  // the copy engine: the array is declared F rows long).
+  if (B == 1)
+    return linear<T>(ctx, st, tc, w->w_o, H, qd, att + (size_t)slot_base * qd, F, R, nullptr, h, H,
+                     out_u, nullptr, H);
   JK_PROF(ctx, st, JK_ST_PRE_ROPE);
   jk_launch_pdl(k_pre_pick<T>, dim3(R), dim3(256), 0, st, (const T*)att, M, F, slot_base, qd, ao);
   JK_LAUNCH_CHECK(ctx);
-  // u = W_o Attn + h
   return linear<T>(ctx, st, tc, w->w_o, H, qd, ao, Rp, R, nullptr, h, H, out_u, nullptr, H);
 }
 
