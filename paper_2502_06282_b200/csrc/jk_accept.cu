@@ -163,13 +163,49 @@ __global__ void __launch_bounds__(128) k_walk_greedy(
                 status);
 }
 
-// Sampling walk.  One block of 1024 threads per sequence.  p and the q_r start "lazy" (read from
-// the logits with the row's precomputed max and sum) and are written out to pbuf/qbuf the first
-// time a rejection changes them.  Every pass over the vocabulary works on 4 entries per thread
-// per step (16-byte loads; the host checks V % 4 == 0 for this mode).
+// Sampling walk.  A thread-block cluster of WALK_CLUSTER blocks per sequence; block r of the cluster
+// owns the vocabulary range [r * Vc, (r + 1) * Vc).  Every block follows the whole walk (tree
+// bookkeeping, the accept / reject decisions, the path) from the same values, so all of them take
+// the same branches and meet at the same cluster barriers; only the passes over the vocabulary
+// (the residual after a rejection, the prefix sums of the bonus draw) are divided, and their
+// per-block sums are exchanged through the blocks' shared memories and added in block order, which
+// gives every block the same bits.  p and the q_r start "lazy" (read from the logits with the
+// row's precomputed max and sum) and are written out to pbuf/qbuf the first time a rejection
+// changes them; a value another block wrote is read from L2 after the barrier that followed the
+// write.  pbuf and every q_r buffer exist twice and a rejection writes the copy it does not read:
+// a block that is already in the next pass cannot overwrite the entry a slower block still has to
+// read for its decision (the copy written two passes later is only reached through a barrier the
+// slower block has passed after that read).  Every pass works on 4 entries per thread per step
+// (16-byte loads; the host checks V % 4 == 0 for this mode).
+#define WALK_CLUSTER 8                 // portable cluster size
+#define WALK_THREADS 512
 struct walk_vec4 { float v[4]; };
 
-__global__ void __launch_bounds__(1024) k_walk_sample(
+__device__ __forceinline__ uint32_t walk_cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t walk_cluster_size() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+// Release-arrive / acquire-wait on the cluster's barrier: orders the shared-memory stores into
+// other blocks and the global stores made before it against the reads after it.
+__device__ __forceinline__ void walk_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// store two words into the variable at `p` of block `rank` of the cluster
+__device__ __forceinline__ void walk_st_remote(const void* p, uint32_t rank, uint32_t a, uint32_t c) {
+  uint32_t addr;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+               : "=r"(addr) : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(rank));
+  asm volatile("st.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(c) : "memory");
+}
+
+__global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
     int M, int max_depth, int V, int K, int n_slots, float inv_t,
     const void* __restrict__ tl_raw, int tl_bf16, const int32_t* __restrict__ tok,
     const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
@@ -177,19 +213,23 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     const float* __restrict__ draft_logits, const float* __restrict__ u_accept,
     const float* __restrict__ u_bonus, const float* __restrict__ rs_max,
     const float* __restrict__ rs_sum, const float* __restrict__ qs_max,
-    const float* __restrict__ qs_sum, float* __restrict__ pbuf_all, float* __restrict__ qbuf_all,
+    const float* __restrict__ qs_sum, float* pbuf_all, float* qbuf_all,
     walk_out o, int cache_rows, int32_t* status) {
   jk_pdl_wait();      // (its dependent is released when this kernel's CTAs exit: measured faster)
   __shared__ float red[66];
+  __shared__ __align__(8) uint32_t xs[2][WALK_CLUSTER][2];   // [round parity][block][2 words]
   __shared__ int s_parent[JK_MAX_TREE], s_tok[JK_MAX_TREE], s_branch[JK_MAX_TREE];
   __shared__ int kids[JK_MAX_TREE];
   __shared__ int n_kids;
   __shared__ int path[16], path_tok[16];
   __shared__ int s_decision;
   __shared__ int s_found;
-  const int b = blockIdx.x, t = threadIdx.x, nt = blockDim.x;
+  const int C = (int)walk_cluster_size(), rank = (int)walk_cluster_rank();
+  const int b = blockIdx.x / C, t = threadIdx.x, nt = blockDim.x;
   const int lane = t & 31, warp = t >> 5, nw = nt >> 5;
-  float* pbuf = pbuf_all + (size_t)b * V;
+  const int Vc = ((V / 4 + C - 1) / C) * 4;            // this block's share of the vocabulary
+  const int vlo = min(V, rank * Vc), vhi = min(V, vlo + Vc);
+  float* pb2 = pbuf_all + (size_t)b * 2 * V;        // the two copies of p, V apart
   const float* tlf = (const float*)tl_raw;
   const __nv_bfloat16* tlh = (const __nv_bfloat16*)tl_raw;
   if (t < M) {
@@ -199,18 +239,21 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
   }
   __syncthreads();
   int cur = 0, n = 0;
+  int xround = 0;                     // exchanges so far: picks the half of xs[] to use
   bool p_mat = false;                 // p lives in pbuf (scaled by p_scale) instead of the logits
+  int p_par = 0;                      // which copy of pbuf holds it
+  unsigned q_par = 0;                 // bit r: which copy of branch r's buffer is current
   float p_scale = 1.f, p_max = 0.f, p_isum = 1.f;
   size_t tl_row = 0;
-  auto p_at = [&](int v) -> float {
-    if (p_mat) return pbuf[v] * p_scale;
+  auto p_at = [&](int v) -> float {                // any v: another block may have written it
+    if (p_mat) return __ldcg(pb2 + (size_t)p_par * V + v) * p_scale;
     const float x = tl_bf16 ? __bfloat162float(tlh[tl_row * V + v]) : tlf[tl_row * V + v];
     return expf((x - p_max) * inv_t) * p_isum;
   };
-  auto p_at4 = [&](int v) -> walk_vec4 {           // v % 4 == 0
+  auto p_at4 = [&](int v) -> walk_vec4 {           // v % 4 == 0, inside this block's range
     walk_vec4 r;
     if (p_mat) {
-      const float4 x = *reinterpret_cast<const float4*>(pbuf + v);
+      const float4 x = *reinterpret_cast<const float4*>(pb2 + (size_t)p_par * V + v);
       r.v[0] = x.x * p_scale; r.v[1] = x.y * p_scale; r.v[2] = x.z * p_scale; r.v[3] = x.w * p_scale;
     } else {
       float x[4];
@@ -227,8 +270,18 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
     }
     return r;
   };
-  // sum of two values over the block in one round
-  auto block_sum2 = [&](float& a, float& c) {
+  // Every block hands its two words to all blocks of the cluster; after the barrier xs[half][j]
+  // holds block j's pair in every block.  Two halves: a block that is one exchange ahead writes
+  // the other half, and it cannot get two ahead without everybody passing the barrier between.
+  auto exchange = [&](uint32_t a, uint32_t c) -> int {
+    const int half = xround & 1;
+    ++xround;
+    if (t < C) walk_st_remote(&xs[half][rank][0], (uint32_t)t, a, c);
+    walk_cluster_sync();
+    return half;
+  };
+  // sum of two values over the block in one round, then over the cluster in block order
+  auto cluster_sum2 = [&](float& a, float& c) {
     a = jk_warp_sum(a);
     c = jk_warp_sum(c);
     __syncthreads();
@@ -241,8 +294,13 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
       if (lane == 0) { red[32] = x; red[65] = y; }
     }
     __syncthreads();
-    a = red[32];
-    c = red[65];
+    const int half = exchange(__float_as_uint(red[32]), __float_as_uint(red[65]));
+    a = 0.f;
+    c = 0.f;
+    for (int j = 0; j < C; ++j) {
+      a += __uint_as_float(xs[half][j][0]);
+      c += __uint_as_float(xs[half][j][1]);
+    }
   };
   while (true) {
     tl_row = (size_t)b * M + cur;
@@ -277,12 +335,15 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
           break;
         }
         const float* dl = draft_logits + (((size_t)b * n_slots + slot) * K + r) * V;
-        float* qbuf = qbuf_all + ((size_t)b * K + r) * V;
+        float* qb2 = qbuf_all + ((size_t)b * K + r) * 2 * V;
+        const float* qcur = qb2 + (size_t)((q_par >> r) & 1u) * V;
+        float* qnew = qb2 + (size_t)(((q_par >> r) & 1u) ^ 1u) * V;
+        float* pnew = pb2 + (size_t)(p_par ^ 1) * V;
         const bool qm = q_mat[r];
         const float qmx = q_max[r], qis = q_isum[r], qsc = q_scale[r];
         if (t == 0) {
           const float px = p_at(x);
-          const float qx = qm ? qbuf[x] * qsc : expf((dl[x] - qmx) * inv_t) * qis;
+          const float qx = qm ? __ldcg(qcur + x) * qsc : expf((dl[x] - qmx) * inv_t) * qis;
           bool acc;
           if (qx > 0.f) acc = u_accept[(size_t)b * M + c] < fminf(1.f, px / qx);
           else acc = px > 0.f;
@@ -295,10 +356,10 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
         // rejection: p <- max(0, p - q_r) (normalised through p_scale); q_r[x] <- 0, renormalised
         float sp = 0.f, sq = 0.f;
 #pragma unroll 2
-        for (int v = t * 4; v < V; v += nt * 4) {
+        for (int v = vlo + t * 4; v < vhi; v += nt * 4) {
           const walk_vec4 pv = p_at4(v);
           float qv[4];
-          const float4 qr = *reinterpret_cast<const float4*>((qm ? qbuf : dl) + v);
+          const float4 qr = *reinterpret_cast<const float4*>((qm ? qcur : dl) + v);
           if (qm) {
             qv[0] = qr.x * qsc; qv[1] = qr.y * qsc; qv[2] = qr.z * qsc; qv[3] = qr.w * qsc;
           } else {
@@ -313,17 +374,19 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
             sp += res[i];
             sq += qn[i];
           }
-          *reinterpret_cast<float4*>(pbuf + v) = make_float4(res[0], res[1], res[2], res[3]);
-          *reinterpret_cast<float4*>(qbuf + v) = make_float4(qn[0], qn[1], qn[2], qn[3]);
+          *reinterpret_cast<float4*>(pnew + v) = make_float4(res[0], res[1], res[2], res[3]);
+          *reinterpret_cast<float4*>(qnew + v) = make_float4(qn[0], qn[1], qn[2], qn[3]);
         }
-        block_sum2(sp, sq);
+        cluster_sum2(sp, sq);
         q_mat[r] = true;
+        q_par ^= 1u << r;
         q_scale[r] = sq > 0.f ? 1.f / sq : 1.f;
         if (!(sp > 0.f)) {            // residual vanished: keep the node's own p for the bonus
           p_mat = false;
           break;
         }
         p_mat = true;
+        p_par ^= 1;
         p_scale = 1.f / sp;
       }
     }
@@ -335,17 +398,18 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
       continue;
     }
     // bonus token: inverse CDF of the current p at u_bonus[depth]; every thread owns a contiguous
-    // run of `per` entries (a multiple of 4)
+    // run of `per` entries (a multiple of 4) of its block's range
     const int dcur = depth[(size_t)b * M + cur];
     const float ub = u_bonus[(size_t)b * (max_depth + 1) + min(max(dcur, 0), max_depth)];
-    const int per = ((V + nt - 1) / nt + 3) / 4 * 4;
-    const int v0 = min(V, t * per), v1 = min(V, v0 + per);
+    const int per = ((Vc + nt - 1) / nt + 3) / 4 * 4;
+    const int v0 = min(vhi, vlo + t * per), v1 = min(vhi, v0 + per);
     float loc = 0.f;
     for (int v = v0; v < v1; v += 4) {
       const walk_vec4 pv = p_at4(v);
       loc += (pv.v[0] + pv.v[1]) + (pv.v[2] + pv.v[3]);
     }
-    // inclusive scan of the runs' sums: shuffles inside a warp, the 32 warp totals by warp 0
+    // inclusive scan of the runs' sums: shuffles inside a warp, the warp totals by warp 0, the
+    // blocks' totals in block order
     float incl = loc;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -368,17 +432,28 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
       if (lane == 31) red[32] = wi;
     }
     __syncthreads();
-    incl += red[33 + warp];
-    const float total = red[32];
+    float base = 0.f, total = 0.f;         // what lies before this block; the whole sum
+    {
+      const int half = exchange(__float_as_uint(red[32]), 0u);
+      for (int j = 0; j < C; ++j) {
+        if (j == rank) base = total;
+        total += __uint_as_float(xs[half][j][0]);
+      }
+    }
+    incl += red[33 + warp] + base;
     const float thr = ub * total;
-    // `before` is exactly the previous thread's inclusive value, so the runs' intervals
-    // [before, incl) join without gaps and some run claims every threshold below the total.
+    // `before` is exactly the previous thread's inclusive value (for a block's first thread the
+    // previous block's last, which is set to the sum of the blocks' totals up to it), so the
+    // runs' intervals [before, incl) join without gaps and some run claims every threshold below
+    // the total.
+    if (t == nt - 1) incl = base + red[32];
+    __syncthreads();                       // red[0..nw) was read above by warp 0 only
     if (lane == 31) red[warp] = incl;
     __syncthreads();
     const float up = __shfl_up_sync(0xffffffffu, incl, 1);
-    const float before = lane ? up : (warp ? red[warp - 1] : 0.f);
+    const float before = lane ? up : (warp ? red[warp - 1] : base);
     // The crossing lies in this thread's run; rounding can let more than one run claim the
-    // threshold (the scan need not be monotone to the last bit) and atomicMin keeps the first.
+    // threshold (the scan need not be monotone to the last bit) and the minimum keeps the first.
     const bool mine = before <= thr && incl > thr;
     if (mine) {
       float run = before;
@@ -395,16 +470,26 @@ __global__ void __launch_bounds__(1024) k_walk_sample(
       if (last_pos >= 0) atomicMin(&s_found, last_pos);
     }
     __syncthreads();
-    if (s_found == INT_MAX) {            // no run passed the threshold: last token with p > 0
-      __syncthreads();
-      if (t == 0) s_found = -1;
-      __syncthreads();
-      for (int v = v1 - 1; v >= v0; --v)
-        if (p_at(v) > 0.f) { atomicMax(&s_found, v); break; }
-      __syncthreads();
+    // the block's last token with p > 0 rides along: it is the answer when no run of any block
+    // passed the threshold
+    if (t == 0) s_decision = -1;
+    __syncthreads();
+    int found;
+    {
+      const int half0 = exchange((uint32_t)s_found, 0u);
+      found = INT_MAX;
+      for (int j = 0; j < C; ++j) found = min(found, (int)xs[half0][j][0]);
     }
-    if (t == 0)
-      walk_finish(o, b, max_depth, n, path, path_tok, max(s_found, 0), cache_rows, M, status);
+    if (found == INT_MAX) {
+      for (int v = v1 - 1; v >= v0; --v)
+        if (p_at(v) > 0.f) { atomicMax(&s_decision, v); break; }
+      __syncthreads();
+      const int half1 = exchange((uint32_t)s_decision, 0u);
+      found = -1;
+      for (int j = 0; j < C; ++j) found = max(found, (int)xs[half1][j][0]);
+    }
+    if (t == 0 && rank == 0)
+      walk_finish(o, b, max_depth, n, path, path_tok, max(found, 0), cache_rows, M, status);
     return;
   }
 }
@@ -502,7 +587,7 @@ extern "C" int jk_accept_and_compact(
     jk_launch_pdl(k_walk_greedy, dim3(batch), dim3(128), 0, st, tree_size, c.max_depth, c.vocab, tok, parent, rs_arg, o,
                                          cache_rows, status);
   } else {
-    jk_launch_pdl(k_walk_sample, dim3(batch), dim3(1024), 0, st, 
+    jk_launch_pdl_cluster(k_walk_sample, dim3(batch * WALK_CLUSTER), dim3(WALK_THREADS), WALK_CLUSTER, 0, st,
         tree_size, c.max_depth, c.vocab, c.top_k, n_slots, inv_t, target_logits,
         tl_dtype == JK_BF16, tok, parent, depth, branch, qslot, draft_logits, u_accept, u_bonus,
         rs_max, rs_sum, (const float*)(ws + L.qs_max), (const float*)(ws + L.qs_sum),

@@ -76,8 +76,8 @@ static void build_layout(const jk_config& c, jk_ws_layout* L) {
   L->rs_arg = take(BM * 4);
   L->rs_max = take(BM * 4);
   L->rs_sum = take(BM * 4);
-  L->pbuf = take((size_t)c.max_batch * c.vocab * 4);
-  L->qbuf = take((size_t)c.max_batch * c.top_k * c.vocab * 4);
+  L->pbuf = take((size_t)c.max_batch * 2 * c.vocab * 4);              // two copies each: a
+  L->qbuf = take((size_t)c.max_batch * c.top_k * 2 * c.vocab * 4);    // rejection writes the other
   L->p_old = take((size_t)c.max_batch * 4);
   const size_t qrows = (size_t)c.max_batch * c.max_depth * c.max_frontier * c.top_k;
   L->qs_arg = take(qrows * 4);

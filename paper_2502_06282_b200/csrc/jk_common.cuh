@@ -37,8 +37,8 @@ struct jk_ws_layout {
   size_t rs_arg;        // i32 [B, M]        per tree node: top-1 token of the target row
   size_t rs_max;        // f32 [B, M]
   size_t rs_sum;        // f32 [B, M]
-  size_t pbuf;          // f32 [B, V]
-  size_t qbuf;          // f32 [B, K, V]
+  size_t pbuf;          // f32 [B, 2, V]
+  size_t qbuf;          // f32 [B, K, 2, V]
   size_t p_old;         // i32 [B]
   size_t qs_arg;        // i32 [B, S, K]     top-1 of every stored draft row (written, not read)
   size_t qs_max;        // f32 [B, S, K]     max of every stored draft logits row
@@ -156,6 +156,28 @@ static inline cudaError_t jk_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// The same launch with the grid grouped into thread-block clusters of `cluster_x` blocks.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t jk_launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                                                unsigned cluster_x, size_t smem, cudaStream_t st,
+                                                Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cluster_x;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
