@@ -197,12 +197,14 @@ __device__ __forceinline__ void walk_cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// store two words into the variable at `p` of block `rank` of the cluster
-__device__ __forceinline__ void walk_st_remote(const void* p, uint32_t rank, uint32_t a, uint32_t c) {
+// store four words into the variable at `p` (16-byte aligned) of block `rank` of the cluster
+__device__ __forceinline__ void walk_st_remote(const void* p, uint32_t rank, uint32_t a, uint32_t c,
+                                               uint32_t d, uint32_t e) {
   uint32_t addr;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
                : "=r"(addr) : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(rank));
-  asm volatile("st.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(c) : "memory");
+  asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};"
+               ::"r"(addr), "r"(a), "r"(c), "r"(d), "r"(e) : "memory");
 }
 
 __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
@@ -217,8 +219,12 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
     walk_out o, int cache_rows, int32_t* status) {
   jk_pdl_wait();      // (its dependent is released when this kernel's CTAs exit: measured faster)
   __shared__ float red[66];
-  __shared__ __align__(8) uint32_t xs[2][WALK_CLUSTER][2];   // [round parity][block][2 words]
+  __shared__ __align__(16) uint32_t xs[2][WALK_CLUSTER][4];  // [exchange parity][block][4 words]
   __shared__ int s_parent[JK_MAX_TREE], s_tok[JK_MAX_TREE], s_branch[JK_MAX_TREE];
+  __shared__ int s_qslot[JK_MAX_TREE], s_depth[JK_MAX_TREE];
+  __shared__ float s_uacc[JK_MAX_TREE], s_rmax[JK_MAX_TREE], s_risum[JK_MAX_TREE];
+  __shared__ float s_qmax[JK_MAX_EXPERTS], s_qisum[JK_MAX_EXPERTS], s_qscale[JK_MAX_EXPERTS];
+  __shared__ float s_fwd[2];          // the next child's token in this pass: new p, new q_r
   __shared__ int kids[JK_MAX_TREE];
   __shared__ int n_kids;
   __shared__ int path[16], path_tok[16];
@@ -232,10 +238,16 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
   float* pb2 = pbuf_all + (size_t)b * 2 * V;        // the two copies of p, V apart
   const float* tlf = (const float*)tl_raw;
   const __nv_bfloat16* tlh = (const __nv_bfloat16*)tl_raw;
-  if (t < M) {
-    s_parent[t] = parent[(size_t)b * M + t];
-    s_tok[t] = tok[(size_t)b * M + t];
-    s_branch[t] = branch[(size_t)b * M + t];
+  if (t < M) {                        // everything the walk reads per node, once
+    const size_t i = (size_t)b * M + t;
+    s_parent[t] = parent[i];
+    s_tok[t] = tok[i];
+    s_branch[t] = branch[i];
+    s_qslot[t] = qslot[i];
+    s_depth[t] = depth[i];
+    s_uacc[t] = u_accept[i];
+    s_rmax[t] = rs_max[i];
+    s_risum[t] = 1.f / rs_sum[i];
   }
   __syncthreads();
   int cur = 0, n = 0;
@@ -243,6 +255,7 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
   bool p_mat = false;                 // p lives in pbuf (scaled by p_scale) instead of the logits
   int p_par = 0;                      // which copy of pbuf holds it
   unsigned q_par = 0;                 // bit r: which copy of branch r's buffer is current
+  unsigned q_mat = 0;                 // bit r: q_r lives in its buffer (scaled by s_qscale[r])
   float p_scale = 1.f, p_max = 0.f, p_isum = 1.f;
   size_t tl_row = 0;
   auto p_at = [&](int v) -> float {                // any v: another block may have written it
@@ -270,62 +283,52 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
     }
     return r;
   };
-  // Every block hands its two words to all blocks of the cluster; after the barrier xs[half][j]
-  // holds block j's pair in every block.  Two halves: a block that is one exchange ahead writes
+  // branch r's draft probability of token v as it stands (any v)
+  auto q_at = [&](int r, int v, const float* dl_r, const float* qcur_r) -> float {
+    if ((q_mat >> r) & 1u) return __ldcg(qcur_r + v) * s_qscale[r];
+    return expf((dl_r[v] - s_qmax[r]) * inv_t) * s_qisum[r];
+  };
+  // Every block hands its four words to all blocks of the cluster; after the barrier xs[half][j]
+  // holds block j's words in every block.  Two halves: a block that is one exchange ahead writes
   // the other half, and it cannot get two ahead without everybody passing the barrier between.
-  auto exchange = [&](uint32_t a, uint32_t c) -> int {
+  auto exchange = [&](uint32_t a, uint32_t c, uint32_t d, uint32_t e) -> int {
     const int half = xround & 1;
     ++xround;
-    if (t < C) walk_st_remote(&xs[half][rank][0], (uint32_t)t, a, c);
+    if (t < C) walk_st_remote(&xs[half][rank][0], (uint32_t)t, a, c, d, e);
     walk_cluster_sync();
     return half;
-  };
-  // sum of two values over the block in one round, then over the cluster in block order
-  auto cluster_sum2 = [&](float& a, float& c) {
-    a = jk_warp_sum(a);
-    c = jk_warp_sum(c);
-    __syncthreads();
-    if (lane == 0) { red[warp] = a; red[33 + warp] = c; }
-    __syncthreads();
-    if (warp == 0) {
-      float x = lane < nw ? red[lane] : 0.f, y = lane < nw ? red[33 + lane] : 0.f;
-      x = jk_warp_sum(x);
-      y = jk_warp_sum(y);
-      if (lane == 0) { red[32] = x; red[65] = y; }
-    }
-    __syncthreads();
-    const int half = exchange(__float_as_uint(red[32]), __float_as_uint(red[65]));
-    a = 0.f;
-    c = 0.f;
-    for (int j = 0; j < C; ++j) {
-      a += __uint_as_float(xs[half][j][0]);
-      c += __uint_as_float(xs[half][j][1]);
-    }
   };
   while (true) {
     tl_row = (size_t)b * M + cur;
     p_mat = false;
-    p_max = rs_max[tl_row];
-    p_isum = 1.f / rs_sum[tl_row];
-    // children of cur in child order (= ascending node index)
-    if (t == 0) {
+    q_mat = 0;
+    p_max = s_rmax[cur];
+    p_isum = s_risum[cur];
+    const int slot = s_qslot[cur];
+    const bool expandable = n < max_depth && slot >= 0 && slot < n_slots;
+    // children of cur in child order (= ascending node index); the branches' (max, 1/sum)
+    if (warp == 0) {
       int c = 0;
-      for (int i = 1; i < M; ++i)
-        if (s_parent[i] == cur) kids[c++] = i;
-      n_kids = c;
+      for (int i0 = 0; i0 < M; i0 += 32) {
+        const int i = i0 + lane;
+        const bool k = i >= 1 && i < M && s_parent[i] == cur;
+        const unsigned m = __ballot_sync(0xffffffffu, k);
+        if (k) kids[c + __popc(m & ((1u << lane) - 1u))] = i;
+        c += __popc(m);
+      }
+      if (lane == 0) n_kids = c;
+    } else if (warp == 1 && lane < K && expandable) {
+      const size_t qrow = ((size_t)b * n_slots + slot) * K + lane;
+      s_qmax[lane] = qs_max[qrow];
+      s_qisum[lane] = 1.f / qs_sum[qrow];
+      s_qscale[lane] = 1.f;
     }
     __syncthreads();
     const int nk = n_kids;
-    const int slot = qslot[(size_t)b * M + cur];
     int accepted = -1;
-    if (nk > 0 && n < max_depth && slot >= 0 && slot < n_slots) {
-      // per-branch draft distributions: lazy (row max, 1/sum) until a rejection touches them
-      float q_max[JK_MAX_EXPERTS], q_isum[JK_MAX_EXPERTS], q_scale[JK_MAX_EXPERTS];
-      bool q_mat[JK_MAX_EXPERTS];
-      for (int r = 0; r < K; ++r) {
-        const size_t qrow = ((size_t)b * n_slots + slot) * K + r;
-        q_max[r] = qs_max[qrow]; q_isum[r] = 1.f / qs_sum[qrow]; q_scale[r] = 1.f; q_mat[r] = false;
-      }
+    if (nk > 0 && expandable) {
+      bool fwd = false;               // this child's decision came with the last pass's sums
+      float fwd_p = 0.f, fwd_q = 0.f;
       for (int ci = 0; ci < nk; ++ci) {
         const int c = kids[ci];
         const int x = s_tok[c];
@@ -339,21 +342,40 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
         const float* qcur = qb2 + (size_t)((q_par >> r) & 1u) * V;
         float* qnew = qb2 + (size_t)(((q_par >> r) & 1u) ^ 1u) * V;
         float* pnew = pb2 + (size_t)(p_par ^ 1) * V;
-        const bool qm = q_mat[r];
-        const float qmx = q_max[r], qis = q_isum[r], qsc = q_scale[r];
-        if (t == 0) {
-          const float px = p_at(x);
-          const float qx = qm ? __ldcg(qcur + x) * qsc : expf((dl[x] - qmx) * inv_t) * qis;
-          bool acc;
-          if (qx > 0.f) acc = u_accept[(size_t)b * M + c] < fminf(1.f, px / qx);
-          else acc = px > 0.f;
-          s_decision = acc ? 1 : 0;
+        int dec;
+        if (fwd) {                    // the same arithmetic on the same values in every thread
+          const float px = fwd_p, qx = fwd_q;
+          dec = qx > 0.f ? (s_uacc[c] < fminf(1.f, px / qx)) : (px > 0.f);
+        } else {
+          if (t == 0) {
+            const float px = p_at(x);
+            const float qx = q_at(r, x, dl, qcur);
+            s_decision = qx > 0.f ? (s_uacc[c] < fminf(1.f, px / qx)) : (px > 0.f);
+          }
+          __syncthreads();            // (the next write of s_decision lies behind another barrier)
+          dec = s_decision;
         }
-        __syncthreads();
-        const int dec = s_decision;
-        __syncthreads();
         if (dec) { accepted = c; break; }
-        // rejection: p <- max(0, p - q_r) (normalised through p_scale); q_r[x] <- 0, renormalised
+        // rejection: p <- max(0, p - q_r) (normalised through p_scale); q_r[x] <- 0, renormalised.
+        // The next child's token (xn, branch rn) is watched for in the pass: its new p and, when
+        // it comes from the same branch, its new q_r travel with the sums, so that its decision
+        // needs no further load.  Another branch's q is not touched by this pass: read it now.
+        const bool qm = (q_mat >> r) & 1u;
+        const float qmx = s_qmax[r], qis = s_qisum[r], qsc = s_qscale[r];
+        int xn = -1, rn = -1;
+        if (ci + 1 < nk) {
+          xn = s_tok[kids[ci + 1]];
+          rn = s_branch[kids[ci + 1]];
+          if (xn < 0 || xn >= V || rn < 0 || rn >= K) xn = -1;
+        }
+        float q_other = 0.f;
+        if (xn >= 0 && rn != r) {
+          const float* dln = draft_logits + (((size_t)b * n_slots + slot) * K + rn) * V;
+          const float* qcn = qbuf_all + (((size_t)b * K + rn) * 2 + ((q_par >> rn) & 1u)) * V;
+          q_other = q_at(rn, xn, dln, qcn);
+        }
+        if (t == 0) { s_fwd[0] = 0.f; s_fwd[1] = 0.f; }
+        __syncthreads();
         float sp = 0.f, sq = 0.f;
 #pragma unroll 2
         for (int v = vlo + t * 4; v < vhi; v += nt * 4) {
@@ -373,14 +395,35 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
             qn[i] = (v + i == x) ? 0.f : qv[i];
             sp += res[i];
             sq += qn[i];
+            if (v + i == xn) { s_fwd[0] = res[i]; s_fwd[1] = qn[i]; }
           }
           *reinterpret_cast<float4*>(pnew + v) = make_float4(res[0], res[1], res[2], res[3]);
           *reinterpret_cast<float4*>(qnew + v) = make_float4(qn[0], qn[1], qn[2], qn[3]);
         }
-        cluster_sum2(sp, sq);
-        q_mat[r] = true;
+        // sums over the block in one round, then over the cluster in block order
+        sp = jk_warp_sum(sp);
+        sq = jk_warp_sum(sq);
+        if (lane == 0) { red[warp] = sp; red[33 + warp] = sq; }
+        __syncthreads();
+        if (warp == 0) {
+          float a = lane < nw ? red[lane] : 0.f, y = lane < nw ? red[33 + lane] : 0.f;
+          a = jk_warp_sum(a);
+          y = jk_warp_sum(y);
+          if (lane == 0) { red[32] = a; red[65] = y; }
+        }
+        __syncthreads();
+        const int half = exchange(__float_as_uint(red[32]), __float_as_uint(red[65]),
+                                  __float_as_uint(s_fwd[0]), __float_as_uint(s_fwd[1]));
+        sp = 0.f;
+        sq = 0.f;
+        for (int j = 0; j < C; ++j) {
+          sp += __uint_as_float(xs[half][j][0]);
+          sq += __uint_as_float(xs[half][j][1]);
+        }
+        q_mat |= 1u << r;
         q_par ^= 1u << r;
-        q_scale[r] = sq > 0.f ? 1.f / sq : 1.f;
+        const float qsc_new = sq > 0.f ? 1.f / sq : 1.f;
+        s_qscale[r] = qsc_new;        // every thread stores the same bits
         if (!(sp > 0.f)) {            // residual vanished: keep the node's own p for the bonus
           p_mat = false;
           break;
@@ -388,6 +431,12 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
         p_mat = true;
         p_par ^= 1;
         p_scale = 1.f / sp;
+        fwd = xn >= 0;
+        if (fwd) {
+          const int owner = xn / Vc;  // the block whose range holds xn
+          fwd_p = __uint_as_float(xs[half][owner][2]) * p_scale;
+          fwd_q = rn == r ? __uint_as_float(xs[half][owner][3]) * qsc_new : q_other;
+        }
       }
     }
     if (accepted >= 0) {
@@ -399,7 +448,7 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
     }
     // bonus token: inverse CDF of the current p at u_bonus[depth]; every thread owns a contiguous
     // run of `per` entries (a multiple of 4) of its block's range
-    const int dcur = depth[(size_t)b * M + cur];
+    const int dcur = s_depth[cur];
     const float ub = u_bonus[(size_t)b * (max_depth + 1) + min(max(dcur, 0), max_depth)];
     const int per = ((Vc + nt - 1) / nt + 3) / 4 * 4;
     const int v0 = min(vhi, vlo + t * per), v1 = min(vhi, v0 + per);
@@ -416,7 +465,7 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
       const float y = __shfl_up_sync(0xffffffffu, incl, off);
       if (lane >= off) incl += y;
     }
-    if (t == 0) s_found = INT_MAX;
+    if (t == 0) { s_found = INT_MAX; s_decision = -1; }
     __syncthreads();                       // red[] is free (the last block sum has been read)
     if (lane == 31) red[warp] = incl;
     __syncthreads();
@@ -434,7 +483,7 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
     __syncthreads();
     float base = 0.f, total = 0.f;         // what lies before this block; the whole sum
     {
-      const int half = exchange(__float_as_uint(red[32]), 0u);
+      const int half = exchange(__float_as_uint(red[32]), 0u, 0u, 0u);
       for (int j = 0; j < C; ++j) {
         if (j == rank) base = total;
         total += __uint_as_float(xs[half][j][0]);
@@ -454,6 +503,8 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
     const float before = lane ? up : (warp ? red[warp - 1] : base);
     // The crossing lies in this thread's run; rounding can let more than one run claim the
     // threshold (the scan need not be monotone to the last bit) and the minimum keeps the first.
+    // The block's last token with p > 0 rides along: it is the answer when no run of any block
+    // passed the threshold.
     const bool mine = before <= thr && incl > thr;
     if (mine) {
       float run = before;
@@ -470,13 +521,9 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
       if (last_pos >= 0) atomicMin(&s_found, last_pos);
     }
     __syncthreads();
-    // the block's last token with p > 0 rides along: it is the answer when no run of any block
-    // passed the threshold
-    if (t == 0) s_decision = -1;
-    __syncthreads();
     int found;
     {
-      const int half0 = exchange((uint32_t)s_found, 0u);
+      const int half0 = exchange((uint32_t)s_found, 0u, 0u, 0u);
       found = INT_MAX;
       for (int j = 0; j < C; ++j) found = min(found, (int)xs[half0][j][0]);
     }
@@ -484,7 +531,7 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk_sample(
       for (int v = v1 - 1; v >= v0; --v)
         if (p_at(v) > 0.f) { atomicMax(&s_decision, v); break; }
       __syncthreads();
-      const int half1 = exchange((uint32_t)s_decision, 0u);
+      const int half1 = exchange((uint32_t)s_decision, 0u, 0u, 0u);
       found = -1;
       for (int j = 0; j < C; ++j) found = max(found, (int)xs[half1][j][0]);
     }
