@@ -453,7 +453,20 @@ __global__ void __launch_bounds__(1024) k_expand_finish(
 
 // ------------------------------------------------------------------------------------------
 // Tree finalisation: top (M-1) of the pool, ascending generation order, ancestor bitsets.
+//
+// Which candidates are kept is the rank of each under (score descending, generation index
+// ascending).  Ranking all of a large pool against all of it is the long part of the kernel, so a
+// pool of more than FIN_SMALL candidates is first cut down: it is divided into FIN_CHUNKS runs,
+// the (M-1)-th largest of the runs' maxima is a lower bound T of the (M-1)-th largest score (the
+// M-1 maxima at or above it are M-1 different candidates), everything below T is dropped unseen
+// and only the candidates at or above T are ranked against one another.  If fewer than M-1 runs
+// are occupied, if more than FIN_CAND candidates reach T (many equal scores) or if a score is
+// NaN, every candidate is ranked against the whole pool as in a small one; the result is the
+// same set either way.
 // ------------------------------------------------------------------------------------------
+#define FIN_SMALL 256
+#define FIN_CHUNKS 128
+#define FIN_CAND 256
 __global__ void __launch_bounds__(1024) k_tree_finalize(
     jk_pool pool, int pool_n, const int32_t* __restrict__ root_tok, int M,
     int32_t* __restrict__ tok, int32_t* __restrict__ parent, int32_t* __restrict__ depth,
@@ -463,14 +476,29 @@ __global__ void __launch_bounds__(1024) k_tree_finalize(
   jk_pdl_trigger();
   __shared__ float sc[JK_MAX_POOL];
   __shared__ short newid[JK_MAX_POOL];      // 0 = dropped, else node index
+  __shared__ unsigned char keepf[JK_MAX_POOL];
   __shared__ int par_s[JK_MAX_TREE];
-  __shared__ int scan[1024];
+  __shared__ int wsum[32];
   __shared__ int keep_s[JK_MAX_TREE];
+  __shared__ float cmax[FIN_CHUNKS];
+  __shared__ int cand[FIN_CAND];
+  __shared__ float s_thr;
+  __shared__ int s_ncand, s_full;
   const int b = blockIdx.x;
   const size_t pb = (size_t)b * pool.stride_b;
-  const int t = threadIdx.x;
-  for (int g = t; g < pool_n; g += blockDim.x) sc[g] = pool.score[pb + g];
+  const int t = threadIdx.x, nt = blockDim.x, lane = t & 31, warp = t >> 5;
   const int m1 = M - 1;
+  const int cs = (pool_n + FIN_CHUNKS - 1) / FIN_CHUNKS;      // candidates per run
+  const bool cut = !static_keep && nt == FIN_CHUNKS * 8 && pool_n > FIN_SMALL &&
+                   (pool_n + cs - 1) / cs >= m1 && m1 >= 1;
+  if (t == 0) { s_ncand = 0; s_full = cut ? 0 : 1; s_thr = 0.f; }
+  __syncthreads();
+  for (int g = t; g < pool_n; g += nt) {
+    const float v = pool.score[pb + g];
+    sc[g] = v;
+    keepf[g] = 0;
+    if (v != v) s_full = 1;
+  }
   if (static_keep && t < m1) {
     // the predefined shape's list: ascending generation indices inside the pool
     const int g = static_keep[t];
@@ -479,33 +507,104 @@ __global__ void __launch_bounds__(1024) k_tree_finalize(
     keep_s[t] = g;
   }
   __syncthreads();
+  if (static_keep) {
+    if (t < m1) {
+      const int g = keep_s[t];
+      if (g >= 0 && g < pool_n) keepf[g] = 1;
+    }
+  } else {
+    if (cut) {
+      // the runs' maxima, then the (M-1)-th largest of them: 8 threads rank one maximum
+      for (int c = t; c < FIN_CHUNKS; c += nt) {
+        float m = -INFINITY;
+        for (int g = c * cs; g < min(pool_n, (c + 1) * cs); ++g) m = fmaxf(m, sc[g]);
+        cmax[c] = m;
+      }
+      __syncthreads();
+      {
+        const int c = t >> 3, part = t & 7;       // 1024 threads = FIN_CHUNKS * 8
+        int rank = 0;
+        if (c < FIN_CHUNKS) {
+          const float v = cmax[c];
+          for (int j = part; j < FIN_CHUNKS; j += 8) rank += jk_better(cmax[j], j, v, c) ? 1 : 0;
+        }
+        rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+        rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+        rank += __shfl_xor_sync(0xffffffffu, rank, 4);
+        if (c < FIN_CHUNKS && part == 0 && rank == m1 - 1) s_thr = cmax[c];
+      }
+      __syncthreads();
+      const float thr = s_thr;
+      for (int g = t; g < pool_n; g += nt) {
+        if (sc[g] >= thr) {
+          const int pos = atomicAdd(&s_ncand, 1);
+          if (pos < FIN_CAND) cand[pos] = g;
+        }
+      }
+      __syncthreads();
+      if (s_ncand > FIN_CAND) s_full = 1;         // (every thread that sees it stores the same)
+      __syncthreads();
+    }
+    if (!s_full) {
+      // rank the candidates at or above the bound against one another: 4 threads each
+      const int nc = s_ncand;
+      const int i = t >> 2, part = t & 3;         // 1024 threads = FIN_CAND * 4
+      int rank = 0, g = 0;
+      if (i < nc) {
+        g = cand[i];
+        const float v = sc[g];
+        for (int j = part; j < nc; j += 4) {
+          const int gj = cand[j];
+          rank += jk_better(sc[gj], gj, v, g) ? 1 : 0;
+        }
+      }
+      rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+      rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+      if (i < nc && part == 0 && rank < m1) keepf[g] = 1;
+    } else {
+      // every candidate against the whole pool; a candidate is shared by as many threads (a
+      // power of two up to 32) as the block has to spare
+      int tpe = 1;
+      while (tpe < 32 && pool_n * tpe * 2 <= nt) tpe <<= 1;
+      for (int g0 = 0; g0 < pool_n; g0 += nt / tpe) {
+        const int g = g0 + t / tpe, part = t % tpe;
+        int rank = 0;
+        if (g < pool_n) {
+          const float v = sc[g];
+          for (int j = part; j < pool_n; j += tpe) rank += jk_better(sc[j], j, v, g) ? 1 : 0;
+        }
+        for (int o = 1; o < tpe; o <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+        if (g < pool_n && part == 0 && rank < m1) keepf[g] = 1;
+      }
+    }
+  }
+  __syncthreads();
   // each thread owns a contiguous slice so that the prefix sum runs in generation order
-  const int per = (pool_n + blockDim.x - 1) / blockDim.x;
+  const int per = (pool_n + nt - 1) / nt;
   const int g0 = t * per, g1 = min(pool_n, g0 + per);
   int cnt = 0;
-  unsigned keepmask = 0;                     // per <= 4 for pool_n <= 4096
-  for (int g = g0; g < g1; ++g) {
-    bool keep = false;
-    if (static_keep) {
-      for (int j = 0; j < m1; ++j) keep |= keep_s[j] == g;
-    } else {
-      const float v = sc[g];
-      int rank = 0;
-      for (int j = 0; j < pool_n; ++j) rank += jk_better(sc[j], j, v, g) ? 1 : 0;
-      keep = rank < m1;
-    }
-    if (keep) { keepmask |= 1u << (g - g0); ++cnt; }
+  for (int g = g0; g < g1; ++g) cnt += keepf[g];
+  int incl = cnt;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += y;
   }
-  scan[t] = cnt;
+  if (lane == 31) wsum[warp] = incl;
   __syncthreads();
-  for (int off = 1; off < (int)blockDim.x; off <<= 1) {
-    int v = t >= off ? scan[t - off] : 0;
-    __syncthreads();
-    scan[t] += v;
-    __syncthreads();
+  if (warp == 0) {
+    const int w = lane < (nt >> 5) ? wsum[lane] : 0;
+    int wi = w;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, wi, off);
+      if (lane >= off) wi += y;
+    }
+    wsum[lane] = wi - w;                     // kept candidates before this warp
   }
-  int id = 1 + scan[t] - cnt;
-  for (int g = g0; g < g1; ++g) newid[g] = (keepmask >> (g - g0)) & 1u ? (short)(id++) : (short)0;
+  __syncthreads();
+  int id = 1 + wsum[warp] + incl - cnt;
+  for (int g = g0; g < g1; ++g) newid[g] = keepf[g] ? (short)(id++) : (short)0;
   __syncthreads();
   const size_t ob = (size_t)b * M;
   if (t == 0) {

@@ -389,3 +389,78 @@ def test_expand_llama2_70b_shape_four_experts():
         wts_dev[name] = t
         wts[name] = _LazyExperts(w, name)
     _sampled_rows(w, [[(0, 0)], [(0, 4)]], wts=wts, wts_dev=wts_dev)
+
+
+# ------------------------------------------------------------ jk_tree_finalize on hand-made pools
+def _made_pool(rng, fs, K, ke, levels=None):
+    """A pool with the structure the draft produces (parents before children, a child never above
+    its parent, the next frontier = the best of a layer), scores in fp32.  `levels`: quantise the
+    increments to that many values, which makes many scores equal."""
+    tok, score, parent, qslot, branch = [], [], [], [], []
+    frontier = [(-1, np.float32(0.0))]
+    slot = 1
+    for l, F in enumerate(fs):
+        assert len(frontier) == F
+        first = len(tok)
+        for pg, ps in frontier:
+            for r in range(K):
+                inc = np.sort(rng.exponential(1.0, ke))
+                if levels:
+                    inc = np.ceil(inc * levels) / levels
+                for j in range(ke):
+                    tok.append(int(rng.integers(0, 64)))
+                    score.append(np.float32(ps - np.float32(inc[j])))
+                    parent.append(pg)
+                    qslot.append(-1)
+                    branch.append(r)
+        if l + 1 < len(fs):
+            layer = np.asarray(score[first:], np.float32)
+            sel = orc.frontier_select(layer, fs[l + 1])
+            frontier = []
+            for s_ in sel:
+                qslot[first + int(s_)] = slot
+                slot += 1
+                frontier.append((first + int(s_), layer[int(s_)]))
+    return {"tok": np.asarray(tok, np.int32), "score": np.asarray(score, np.float32),
+            "parent": np.asarray(parent, np.int32), "qslot": np.asarray(qslot, np.int32),
+            "branch": np.asarray(branch, np.int32)}
+
+
+@pytest.mark.parametrize("fs,ke,M,levels", [
+    ([1, 10, 10, 10, 10, 10], 5, 60, None),      # 510 candidates: the bound cuts the pool down
+    ([1, 10, 10, 10, 10, 10], 5, 60, 2),         # many equal scores: more reach the bound than fit
+    ([1, 10, 10, 10, 10, 10], 5, 128, None),     # 127 kept of 510
+    ([1, 10, 20, 20, 20, 20], 5, 100, None),     # 910 candidates in 114 runs of 8, 99 kept
+    ([1, 10, 20, 20, 20, 20], 5, 128, None),     # the same pool, 127 kept: ranked whole
+    ([1, 12, 12], 6, 100, None),                 # 300 candidates in runs of 3: 100 runs for 99 kept
+    ([1, 6, 6, 6], 5, 40, None),                 # 190 candidates: ranked whole
+    ([1, 5, 5], 13, 128, None),                  # 286 candidates in 96 runs, 127 kept: ranked whole
+])
+def test_tree_finalize_made_pools(fs, ke, M, levels):
+    K, B = 2, 3
+    rng = np.random.default_rng(len(fs) * 1000 + ke * 10 + M)
+    pools = [_made_pool(rng, fs, K, ke, levels) for _ in range(B)]
+    pool_n = len(pools[0]["tok"])
+    w = synth.scaled(synth.WORKLOADS["tiny"], batch=B, tree_size=M, k_per_expert=ke,
+                     depth=len(fs), width=max(fs))
+    ctx = jk.Context.for_workload(w, frontier_sizes=fs)
+    pool = {k: dev(np.stack([p[k] for p in pools])) for k in pools[0]}
+    i32 = dict(dtype=torch.int32, device="cuda")
+    tree = {k: torch.full((B, M), -7, **i32) for k in ("tok", "parent", "depth", "branch", "qslot")}
+    anc = torch.zeros(B, M, 2, dtype=torch.int64, device="cuda")
+    root = torch.arange(5, 5 + B, **i32)
+    ctx.tree_finalize(B, pool, pool_n, root, M, tree["tok"], tree["parent"], tree["depth"],
+                      tree["branch"], tree["qslot"], anc)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    for b in range(B):
+        p = pools[b]
+        t = orc.tree_finalize(p["tok"], p["score"], p["parent"], p["qslot"], 5 + b, M,
+                              pool_branch=p["branch"])
+        for key in ("tok", "parent", "depth", "branch", "qslot"):
+            assert host(tree[key])[b].tolist() == t[key].tolist(), (b, key)
+        am = orc.ancestor_mask(t["parent"])
+        bits = host(anc)[b].astype(np.uint64)
+        for i in range(M):
+            got = [(int(bits[i, c // 64]) >> (c % 64)) & 1 for c in range(M)]
+            assert got == am[i].astype(int).tolist()
