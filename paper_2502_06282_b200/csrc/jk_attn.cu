@@ -157,10 +157,12 @@ __global__ void __launch_bounds__(256) k_attn_combine(
   if (row >= n_out) return;
   const float* po = part_o + row * D + lane * DPL;      // slice s is s * n_out * D further
   const size_t sstride = n_out * D;
-  auto load_batch = [&](int s0, float (&v)[8][DPL]) {   // eight independent vector loads in flight
+  constexpr int NB = 12;                                // slices per batch of loads
+  auto load_batch = [&](int s0, float (&v)[NB][DPL]) {  // NB independent vector loads in flight
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int s = s0 + j < n_split ? s0 + j : n_split - 1;
+    for (int j = 0; j < NB; ++j) {
+      if (s0 + j >= n_split) continue;                  // (never read below)
+      const int s = s0 + j;
       if (DPL == 4) {
         const float4 x = *reinterpret_cast<const float4*>(po + (size_t)s * sstride);
         v[j][0] = x.x; v[j][1] = x.y; v[j][DPL - 2] = x.z; v[j][DPL - 1] = x.w;
@@ -171,7 +173,7 @@ __global__ void __launch_bounds__(256) k_attn_combine(
     }
   };
   // the first batch of partial outputs is asked for before anything waits on the (max, sum) pairs
-  float v[8][DPL];
+  float v[NB][DPL];
   load_batch(0, v);
   // lane s holds (max, sum) of slice s (n_split <= 32); one load round for all slices
   float ms = -INFINITY, ls = 0.f;
@@ -186,10 +188,10 @@ __global__ void __launch_bounds__(256) k_attn_combine(
   float acc[DPL];
 #pragma unroll
   for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
-  for (int s0 = 0; s0 < n_split; s0 += 8) {
+  for (int s0 = 0; s0 < n_split; s0 += NB) {
     if (s0 > 0) load_batch(s0, v);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < NB; ++j) {
       const float w = __shfl_sync(0xffffffffu, w_lane, (s0 + j) & 31);
       if (s0 + j < n_split && w != 0.f) {
 #pragma unroll
