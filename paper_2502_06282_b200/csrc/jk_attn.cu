@@ -145,7 +145,10 @@ __global__ void __launch_bounds__(256) k_tree_attn(
 }
 
 // Merge the key-range slices: out = sum_s e^{m_s - m} o_s / sum_s e^{m_s - m} l_s.  One warp per row.
-template <typename T, int D>
+// NB slices are loaded per round: 8, or 12 when there are more than 8 slices (9 at the 7B shape: a
+// second round is a second trip to L2 on a call that is a chain of such trips; 20 per round costs
+// the occupancy that keeps the 240 blocks in one wave and measured slower).
+template <typename T, int D, int NB>
 __global__ void __launch_bounds__(256) k_attn_combine(
     const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_split,
     size_t n_out, T* __restrict__ out) {
@@ -157,7 +160,6 @@ __global__ void __launch_bounds__(256) k_attn_combine(
   if (row >= n_out) return;
   const float* po = part_o + row * D + lane * DPL;      // slice s is s * n_out * D further
   const size_t sstride = n_out * D;
-  constexpr int NB = 12;                                // slices per batch of loads
   auto load_batch = [&](int s0, float (&v)[NB][DPL]) {  // NB independent vector loads in flight
 #pragma unroll
     for (int j = 0; j < NB; ++j) {
@@ -236,7 +238,7 @@ static int attn_impl(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, 
   JK_LAUNCH_CHECK(ctx);
   const size_t n_out = (size_t)B * M * c.n_q_heads;
   JK_PROF(ctx, st, ctx->st_combine);
-  k_attn_combine<T, D><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
+  k_attn_combine<T, D, 8><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
                                                                     n_out, (T*)out);
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
@@ -255,12 +257,17 @@ int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_o
   const float* part_ml = (const float*)(ctx->ws + L.attn_ml);
   JK_PROF(ctx, st, ctx->st_combine);
   const dim3 grid((unsigned)((n_out + 7) / 8));
-  if (ctx->cfg.head_dim == 128)
-    jk_launch_pdl(k_attn_combine<__nv_bfloat16, 128>, grid, dim3(256), 0, st, part_o, part_ml,
-                  n_split, n_out, (__nv_bfloat16*)out);
-  else
-    jk_launch_pdl(k_attn_combine<__nv_bfloat16, 64>, grid, dim3(256), 0, st, part_o, part_ml,
-                  n_split, n_out, (__nv_bfloat16*)out);
+#define JK_COMBINE(DD, NBB)                                                                    \
+  jk_launch_pdl(k_attn_combine<__nv_bfloat16, DD, NBB>, grid, dim3(256), 0, st, part_o, part_ml, \
+                n_split, n_out, (__nv_bfloat16*)out)
+  if (ctx->cfg.head_dim == 128) {
+    if (n_split <= 8) JK_COMBINE(128, 8);
+    else JK_COMBINE(128, 12);
+  } else {
+    if (n_split <= 8) JK_COMBINE(64, 8);
+    else JK_COMBINE(64, 12);
+  }
+#undef JK_COMBINE
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
 }
@@ -372,7 +379,7 @@ static int attn_static_impl(jk_ctx* ctx, cudaStream_t st, int dev, unsigned char
       (const T*)q, (const T*)kc, (const T*)vc, sb, sh, cache_rows, kv_len, parent, scale, M,
       c.n_q_heads, c.n_kv_heads, n_split, n_qblk, part_o, part_ml, status);
   JK_LAUNCH_CHECK(ctx);
-  k_attn_combine<T, D><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
+  k_attn_combine<T, D, 8><<<(unsigned)((n_out + 7) / 8), 256, 0, st>>>(part_o, part_ml, n_split,
                                                                     n_out, (T*)out);
   JK_LAUNCH_CHECK(ctx);
   return JK_OK;
