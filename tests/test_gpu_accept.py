@@ -129,11 +129,14 @@ def _near_tie(trace, ua):
     return False
 
 
-@pytest.mark.parametrize("kind,alpha,agree", [("random", 0.8, 0.0), ("random", 0.0, 0.0),
-                                              ("chain", 0.8, 1.0), ("star", 0.8, 0.5),
-                                              ("random", 1.0, 1.0)])
-def test_sampling_accept(kind, alpha, agree):
-    w = synth.scaled(synth.WORKLOADS["tiny"], batch=4, vocab=2000, seed=1234)
+# vocab 2000: the eight blocks of the walk's cluster own 252 entries each but the last (236);
+# vocab 36: five blocks own 8, 8, 8, 8, 4 entries and three own none
+@pytest.mark.parametrize("kind,alpha,agree,vocab", [("random", 0.8, 0.0, 2000), ("random", 0.0, 0.0, 2000),
+                                                    ("chain", 0.8, 1.0, 2000), ("star", 0.8, 0.5, 2000),
+                                                    ("random", 1.0, 1.0, 2000), ("random", 0.8, 0.3, 36),
+                                                    ("star", 0.5, 0.6, 36)])
+def test_sampling_accept(kind, alpha, agree, vocab):
+    w = synth.scaled(synth.WORKLOADS["tiny"], batch=4, vocab=vocab, seed=1234)
     if kind == "chain":
         w = synth.scaled(w, depth=w.tree_size - 1)
     tree, n_slots = _tree_arrays(w, kind, 21)
