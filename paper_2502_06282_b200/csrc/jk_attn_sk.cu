@@ -721,6 +721,127 @@ __global__ void __launch_bounds__(256) k_attn_combine_sk(
     out[row * D + lane * DPL + t] = __float2bfloat16_rn(acc[t] * inv);
 }
 
+// The same merge with two rows per warp (16 lanes per row, D / 16 values per lane): half as many
+// warps, so that the rows of a large call (9600 at the 13B shape with batch 4, more than the
+// 64 warps per SM the device holds) fit in one wave.  A lane keeps the (max, sum) of slices
+// lane and lane + 16 of its row.
+template <int D>
+__global__ void __launch_bounds__(256, 5) k_attn_combine_sk2(
+    const float* __restrict__ part_o, const float* __restrict__ part_ml,
+    const int32_t* __restrict__ kv_len, int B, int M, int Hq, int Hkv, int n_cta, int max_split,
+    int min_units, int cache_rows, __nv_bfloat16* __restrict__ out) {
+  __shared__ int s_tiles[JK_MAX_ROWS];
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  for (int i = threadIdx.x; i < B; i += blockDim.x) {
+    const int P = kv_len[i];         // not written by the attention kernel: read before the wait
+    const bool bad = P < 0 || P + M > cache_rows;
+    s_tiles[i] = bad ? 1 : (P + M + ASK_KEYS - 1) / ASK_KEYS;
+    if (bad) s_bad = 1;
+  }
+  __syncthreads();
+  jk_pdl_wait();
+  jk_pdl_trigger();
+  if (s_bad) return;
+  constexpr int DPL = D / 16;        // values per lane
+  constexpr int NP = DPL / 4;        // 16-byte pieces per lane
+  constexpr int NBS = NP == 2 ? 3 : 4;   // slices per round of loads (48 registers a thread)
+  const int lane = threadIdx.x & 31, hl = lane & 15;
+  const size_t n_out = (size_t)B * M * Hq;
+  const size_t row_w = (size_t)blockIdx.x * 16 + (size_t)(threadIdx.x >> 5) * 2;
+  if (row_w >= n_out) return;        // both rows of the warp are past the end
+  const bool live = row_w + (lane >> 4) < n_out;
+  const size_t row = live ? row_w + (lane >> 4) : n_out - 1;
+  const int G = Hq / Hkv;
+  const int n_qblk = (G * M + ASK_ROWS - 1) / ASK_ROWS;
+  const int items_per_b = Hkv * n_qblk;
+  const ask_plan pl = ask_make_plan(s_tiles, B, items_per_b, n_cta, max_split, min_units);
+  const int head = (int)(row % Hq);
+  const int node = (int)((row / Hq) % M);
+  const int b = (int)(row / ((size_t)Hq * M));
+  uint32_t base = 0;
+  for (int i = 0; i < b; ++i) base += (uint32_t)s_tiles[i] * (uint32_t)items_per_b;
+  const uint32_t Tb = (uint32_t)s_tiles[b];
+  const uint32_t item = (uint32_t)((head / G) * n_qblk + ((head % G) * M + node) / ASK_ROWS);
+  const uint32_t start = base + item * Tb;
+  const int n_split = (int)(ask_owner(start + Tb - 1u, pl) - ask_owner(start, pl)) + 1;
+  const int n_loop = max(n_split, __shfl_xor_sync(0xffffffffu, n_split, 16));
+  // [slice][item][16-byte piece][row of the block][4]: see the attention kernel's epilogue
+  const size_t gitem = (size_t)b * items_per_b + item;
+  const int lrow = ((head % G) * M + node) % ASK_ROWS;
+  const size_t n_items = (size_t)B * items_per_b;
+  const float* po = part_o + gitem * ((size_t)ASK_ROWS * D) +
+                    ((size_t)(hl * NP) * ASK_ROWS + lrow) * 4;
+  const size_t sstride = n_items * ((size_t)ASK_ROWS * D);
+  auto load_batch = [&](int s0, float4 (&v)[NBS][NP]) {   // NBS * NP independent vector loads in flight
+#pragma unroll
+    for (int j = 0; j < NBS; ++j) {
+      const int s = s0 + j < n_split ? s0 + j : n_split - 1;
+#pragma unroll
+      for (int k = 0; k < NP; ++k)
+        v[j][k] = *reinterpret_cast<const float4*>(po + (size_t)s * sstride + (size_t)k * ASK_ROWS * 4);
+    }
+  };
+  // the first batch of partial outputs is asked for before anything waits on the (max, sum) pairs
+  float4 v[NBS][NP];
+  load_batch(0, v);
+  float ms_a = -INFINITY, ls_a = 0.f, ms_b = -INFINITY, ls_b = 0.f;
+  if (hl < n_split) {
+    const float4 x = *reinterpret_cast<const float4*>(
+        part_ml + (((size_t)hl * n_items + gitem) * ASK_ROWS + lrow) * 4);
+    ms_a = x.x;
+    ls_a = x.y + x.z;
+  }
+  if (hl + 16 < n_split) {
+    const float4 x = *reinterpret_cast<const float4*>(
+        part_ml + (((size_t)(hl + 16) * n_items + gitem) * ASK_ROWS + lrow) * 4);
+    ms_b = x.x;
+    ls_b = x.y + x.z;
+  }
+  float m = fmaxf(ms_a, ms_b);
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float w_a = (ms_a == -INFINITY) ? 0.f : __expf(ms_a - m);
+  const float w_b = (ms_b == -INFINITY) ? 0.f : __expf(ms_b - m);
+  float l = w_a * ls_a + w_b * ls_b;
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  float acc[DPL];
+#pragma unroll
+  for (int t = 0; t < DPL; ++t) acc[t] = 0.f;
+  for (int s0 = 0; s0 < n_loop; s0 += NBS) {
+    if (s0 > 0) load_batch(s0, v);
+#pragma unroll
+    for (int j = 0; j < NBS; ++j) {
+      const int sl = (s0 + j) & 31;
+      const int src = (lane & 16) | (sl & 15);
+      const float wa = __shfl_sync(0xffffffffu, w_a, src);
+      const float wb = __shfl_sync(0xffffffffu, w_b, src);
+      const float w = sl < 16 ? wa : wb;
+      if (s0 + j < n_split && w != 0.f) {
+#pragma unroll
+        for (int k = 0; k < NP; ++k) {
+          acc[4 * k] += w * v[j][k].x; acc[4 * k + 1] += w * v[j][k].y;
+          acc[4 * k + 2] += w * v[j][k].z; acc[4 * k + 3] += w * v[j][k].w;
+        }
+      }
+    }
+  }
+  if (!live) return;
+  const float inv = 1.f / l;
+  __nv_bfloat16* dst = out + row * D + hl * DPL;
+#pragma unroll
+  for (int k = 0; k < NP; ++k) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[4 * k] * inv, acc[4 * k + 1] * inv);
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(acc[4 * k + 2] * inv, acc[4 * k + 3] * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst + 4 * k) = pk;
+  }
+}
+
 // jk_attn_tc.cu: tensor maps of the two caches
 int jk_attn_tc_maps(jk_ctx* ctx, const void* kc, const void* vc, int64_t sb, int64_t sh,
                     int cache_rows, CUtensorMap* mk, CUtensorMap* mv);
@@ -784,7 +905,17 @@ int jk_attn_sk(jk_ctx* ctx, cudaStream_t st, int B, int M, const void* q, const 
   JK_LAUNCH_CHECK(ctx);
   const size_t n_out = (size_t)B * M * c.n_q_heads;
   JK_PROF(ctx, st, ctx->st_combine);
-  if (D == 128)
+  // more rows than the device holds warps at once: two rows per warp keep the merge in one wave
+  const bool two = n_out > (size_t)ctx->sm_count * 48;
+  if (D == 128 && two)
+    jk_launch_pdl(k_attn_combine_sk2<128>, dim3((unsigned)((n_out + 15) / 16)), dim3(256), 0, st,
+                  (const float*)part_o, (const float*)part_ml, kv_len, B, M, c.n_q_heads,
+                  c.n_kv_heads, n_cta, ms, min_units, cache_rows, (__nv_bfloat16*)out);
+  else if (D == 64 && two)
+    jk_launch_pdl(k_attn_combine_sk2<64>, dim3((unsigned)((n_out + 15) / 16)), dim3(256), 0, st,
+                  (const float*)part_o, (const float*)part_ml, kv_len, B, M, c.n_q_heads,
+                  c.n_kv_heads, n_cta, ms, min_units, cache_rows, (__nv_bfloat16*)out);
+  else if (D == 128)
     jk_launch_pdl(k_attn_combine_sk<128>, dim3((unsigned)((n_out + 7) / 8)), dim3(256), 0, st,
                   (const float*)part_o, (const float*)part_ml, kv_len, B, M, c.n_q_heads,
                   c.n_kv_heads, n_cta, ms, min_units, cache_rows, (__nv_bfloat16*)out);

@@ -68,6 +68,9 @@ def test_attn_tiny_every_tensor_core_kernel(kind, kernel):
     (900, 33, 16, 16, 64, 3),     # the same with head size 64
     (8192, 128, 8, 2, 128, 2),    # the longest prefix and largest tree of the sweep: 65 key tiles
     (4096, 64, 8, 8, 64, 8),      # batch 8, ragged lengths, head size 64
+    (512, 60, 32, 8, 64, 4),      # 7680 output rows, head size 64: the persistent kernel's merge
+                                  # takes two rows per warp
+    (200, 57, 45, 45, 128, 3),    # 7695 rows (odd: the last warp of that merge has one live row)
 ])
 def test_attn_shapes(dtype, P, M, Hq, Hkv, d, B):
     w = synth.scaled(synth.WORKLOADS["tiny"], name="attn", dtype=dtype, prefix=P, tree_size=M,
