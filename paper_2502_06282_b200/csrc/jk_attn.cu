@@ -145,9 +145,11 @@ __global__ void __launch_bounds__(256) k_tree_attn(
 }
 
 // Merge the key-range slices: out = sum_s e^{m_s - m} o_s / sum_s e^{m_s - m} l_s.  One warp per row.
-// NB slices are loaded per round: 8, or 12 when there are more than 8 slices (9 at the 7B shape: a
-// second round is a second trip to L2 on a call that is a chain of such trips; 20 per round costs
-// the occupancy that keeps the 240 blocks in one wave and measured slower).
+// NB slices are loaded per round: 8, 10 or 12 by the number of slices (9 at the 7B shape: a second
+// round is a second trip to L2 on a call that is a chain of such trips).  Up to 10 per round the
+// kernel stays within 64 registers, so that two of its blocks leave room on an SM for a CTA of
+// the next call's attention kernel, which starts its prologue and its prefix copies there while
+// the merge runs; 20 per round costs the occupancy that keeps the blocks in one wave.
 template <typename T, int D, int NB>
 __global__ void __launch_bounds__(256) k_attn_combine(
     const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_split,
@@ -262,9 +264,11 @@ int jk_attn_combine_launch(jk_ctx* ctx, cudaStream_t st, int n_split, size_t n_o
                 n_split, n_out, (__nv_bfloat16*)out)
   if (ctx->cfg.head_dim == 128) {
     if (n_split <= 8) JK_COMBINE(128, 8);
+    else if (n_split <= 10) JK_COMBINE(128, 10);
     else JK_COMBINE(128, 12);
   } else {
     if (n_split <= 8) JK_COMBINE(64, 8);
+    else if (n_split <= 10) JK_COMBINE(64, 10);
     else JK_COMBINE(64, 12);
   }
 #undef JK_COMBINE
